@@ -1,0 +1,195 @@
+/*
+ * mcsd.h - C ABI of the B200 (sm_100a) multi-candidate speculative-decoding
+ * verification library (libmcsd.so).
+ *
+ * One call verifies a batch of draft token trees that share one topology:
+ * for every tree node it forms the target and draft next-token distributions
+ * (temperature softmax over the full vocabulary), runs the k-candidate
+ * rejection loop of Algorithm 1 (candidates drawn with replacement) or
+ * Algorithm 2 (without replacement), and then walks every tree from the root
+ * along accepted children (Section 3, "Multi-Candidate Speculative Decoding")
+ * to return the accepted tokens, the endpoint ("bonus") token and the
+ * distribution that token was drawn from.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global-memory pointers on the current device;
+ *     "host" pointers are ordinary CPU memory.  Nothing is allocated, freed or
+ *     retained by the library except where an entry point says so; all device
+ *     work is enqueued on desc->stream and the call returns without
+ *     synchronising.
+ *   - Tree layout: node 0 is the root (the last committed token); nodes are in
+ *     generation (level) order, parent[n] < n, the children of a node are
+ *     contiguous and are tested in ascending index, which is the order the draft
+ *     model sampled them in (loop "for i = 1..k" of Algorithms 1 and 2); the
+ *     nodes that have children are exactly 0 .. n_internal-1.  Every k-config
+ *     tree k_1 x k_2 x ... (Section 4.3) has this form.
+ *   - Randomness is supplied by the caller: uniforms[b][n][0] is the r of the
+ *     acceptance test of node n as a candidate of its parent, uniforms[b][n][1]
+ *     is the uniform used to draw the endpoint token if the walk stops at n.
+ *     Uniforms are expected in the open interval (0, 1).
+ *   - Endpoint draw: inverse CDF in token order, the smallest x with
+ *     sum_{y<=x} P(y) > u * sum_y P(y); tokens of probability 0 are never drawn.
+ *   - Temperature 0 selects the argmax rule (Section 4.4): a candidate is
+ *     accepted iff it equals the target argmax (lowest index on ties) and the
+ *     endpoint token is the target argmax of the node where the walk stops;
+ *     draft logits are not read.
+ *   - Return value: MCSD_OK (0) or a negative MCSD_ERR_* code; on an error
+ *     nothing has been enqueued.  Faults that only the device can see (token out
+ *     of range, zero mass, expired bounded wait) set MCSD_STATUS_* bits in
+ *     out_status[b]; kernels never trap and every wait in them is bounded.
+ */
+#ifndef MCSD_H_
+#define MCSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MCSD_VERSION 100
+
+/* logit element types (both logit tensors share one) */
+#define MCSD_DTYPE_F32 0
+#define MCSD_DTYPE_BF16 1
+#define MCSD_DTYPE_F16 2
+
+/* replacement_mode */
+#define MCSD_MODE_WITH_REPLACEMENT 0    /* Algorithm 1 */
+#define MCSD_MODE_WITHOUT_REPLACEMENT 1 /* Algorithm 2 */
+
+/* limits */
+#define MCSD_MAX_NODES 512     /* nodes per tree, root included            */
+#define MCSD_MAX_CHILDREN 32   /* candidates per node (the paper uses <= 32) */
+#define MCSD_MAX_VOCAB 65536   /* vocabulary size                          */
+
+/* return codes */
+#define MCSD_OK 0
+#define MCSD_ERR_NULL (-1)        /* a required pointer is NULL                       */
+#define MCSD_ERR_SHAPE (-2)       /* batch/n_nodes/n_internal/vocab out of range      */
+#define MCSD_ERR_DTYPE (-3)
+#define MCSD_ERR_MODE (-4)
+#define MCSD_ERR_TEMPERATURE (-5) /* negative, NaN or infinite                        */
+#define MCSD_ERR_TREE (-6)        /* tree_parent breaks the layout contract           */
+#define MCSD_ERR_STRIDE (-7)      /* row stride smaller than vocab                    */
+#define MCSD_ERR_WORKSPACE (-8)   /* workspace missing, misaligned or too small       */
+#define MCSD_ERR_CUDA (-9)        /* a CUDA runtime call or kernel launch failed      */
+#define MCSD_ERR_UNSUPPORTED (-10)/* beyond MCSD_MAX_*                                */
+
+/* bits of out_status[b] */
+#define MCSD_STATUS_DEGENERATE 1 /* residual mass was 0 after a rejection; residual kept */
+#define MCSD_STATUS_BAD_TOKEN 2  /* a candidate token outside [0, vocab): rejected       */
+#define MCSD_STATUS_NO_MASS 4    /* endpoint draw from a distribution of mass 0 / NaN    */
+#define MCSD_STATUS_TIMEOUT 8    /* a bounded on-chip wait expired; results invalid      */
+
+typedef struct mcsd_desc {
+    int32_t batch;      /* B: number of trees                                         */
+    int32_t n_nodes;    /* N+1: nodes per tree, root included                         */
+    int32_t n_internal; /* nodes that have children (= rows of draft_logits per tree) */
+    int32_t vocab;      /* V                                                          */
+    int32_t dtype;      /* MCSD_DTYPE_*                                               */
+    int32_t reserved;   /* must be 0                                                  */
+    int64_t ld_target;  /* elements between consecutive rows of target_logits, >= V   */
+    int64_t ld_draft;   /* same for draft_logits                                      */
+    void *stream;       /* cudaStream_t the work is enqueued on (0 = default stream)  */
+    void *workspace;    /* device scratch, 256-byte aligned, caller-owned; at least   */
+    size_t workspace_bytes; /* mcsd_workspace_bytes() bytes; contents are overwritten */
+    /* Optional per-node outputs (device), NULL to skip; when NULL the library keeps
+     * the first two in the workspace:                                              */
+    int32_t *node_accept; /* [B][n_nodes] accepted child of each node, or -1          */
+    int32_t *node_bonus;  /* [B][n_nodes] endpoint token of each node that can end a
+                             walk (leaf, or all candidates rejected), else -1       */
+    float *node_ratio;    /* [B][n_nodes] p/q seen by the test of each draft node; -1
+                             for a forced rejection; untouched if never tested      */
+    int32_t *out_status;  /* [B] MCSD_STATUS_* bits (device), NULL to skip            */
+} mcsd_desc;
+
+/*
+ * The whole verification step (Algorithms 1 and 2 at every node, then the walk
+ * of Section 3).  Equivalent to mcsd_verify_nodes followed by mcsd_verify_walk.
+ *
+ *   target_logits  device [B][n_nodes][ld_target]   logits of the target model at
+ *                  the root and after every draft node
+ *   draft_logits   device [B][n_internal][ld_draft] logits of the draft model at
+ *                  every node that has children; may be NULL when temperature == 0
+ *   tree_parent    HOST   [n_nodes] parent[0] = -1; shared by the whole batch
+ *   cand_tokens    device [B][n_nodes] token carried by each draft node; entry 0
+ *                  of a tree is ignored
+ *   uniforms       device [B][n_nodes][2] float32, see "Randomness" above; may be
+ *                  NULL when temperature == 0
+ *   temperature    0 = argmax rule; > 0 = softmax(logits / temperature), both models
+ *   replacement_mode  MCSD_MODE_*
+ *   out_accept_len device [B] number of accepted draft tokens, 0 .. gamma
+ *   out_tokens     device [B][gamma+1] accepted tokens, then the endpoint token,
+ *                  then -1; gamma = depth of the tree
+ *   out_residual   device [B][vocab] float32, the distribution the endpoint token
+ *                  was drawn from (final residual p of the stopping node, its
+ *                  target distribution for a leaf, one-hot at temperature 0);
+ *                  NULL to skip
+ * Rows whose base address and stride are multiples of 16 bytes take the bulk-copy
+ * (TMA) path; any other layout is accepted and takes a slower plain-load path.
+ */
+int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                float temperature, int replacement_mode, int32_t *out_accept_len,
+                int32_t *out_tokens, float *out_residual);
+
+/*
+ * Stage 1: the per-node part (softmax statistics of both models, the rejection
+ * loop of Algorithm 1 / 2, the endpoint token of every node that can end a
+ * walk).  Fills node_accept / node_bonus (in the workspace when the descriptor
+ * leaves them NULL) and the per-node statistics kept in the workspace.
+ * Arguments as in mcsd_verify.
+ */
+int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                      float temperature, int replacement_mode);
+
+/*
+ * Stage 2: the walk of Section 3 from the root along accepted children, using
+ * what stage 1 left in the workspace of the same descriptor, and the residual
+ * distribution of the node where each walk stops (recomputed from that node's
+ * two logit rows and stored statistics).  Arguments as in mcsd_verify.
+ */
+int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, float temperature,
+                     int32_t *out_accept_len, int32_t *out_tokens, float *out_residual);
+
+/*
+ * The same step for callers whose data lives in HOST memory: every pointer below
+ * is a host pointer.  The library allocates device buffers for a slice of the
+ * batch, copies the slice in, verifies it and copies the results back, slice
+ * after slice on two internal streams so that copies overlap the kernels; it
+ * frees everything and synchronises before it returns.  Only batch, n_nodes,
+ * n_internal, vocab, dtype, ld_target and ld_draft of the descriptor are read;
+ * node_* outputs are not produced.  out_status (host, [B]) may be NULL.
+ * Host buffers in page-locked memory make the copies asynchronous.
+ */
+int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int replacement_mode, int32_t *out_accept_len,
+                     int32_t *out_tokens, float *out_residual, int32_t *out_status);
+
+/* Bytes of device workspace mcsd_verify needs for this descriptor (batch and
+ * n_nodes are read); 0 if the descriptor is NULL or its shape is invalid. */
+size_t mcsd_workspace_bytes(const mcsd_desc *desc);
+
+/* Depth (gamma) of a tree given as a host parent array, or a negative MCSD_ERR_*
+ * code if the array breaks the layout contract.  out_tokens has gamma+1 columns. */
+int mcsd_tree_depth(const int32_t *tree_parent, int32_t n_nodes);
+
+/* Number of kernel launches the last successful mcsd_verify / stage call on this
+ * host thread enqueued (for launch accounting in benchmarks). */
+int mcsd_last_launch_count(void);
+
+/* Static description of a return code. */
+const char *mcsd_status_string(int code);
+
+/* MCSD_VERSION the library was built from. */
+int mcsd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MCSD_H_ */

@@ -1,0 +1,189 @@
+"""Comparison rules between the CPU oracle and another implementation's outputs.
+
+TEST INFRASTRUCTURE (same standing as the oracle itself).  Works on numpy arrays
+only; imports nothing from the CUDA package.
+
+Rules
+  * Acceptance decisions are compared node by node and must be identical, except
+    that a node whose first differing test has |u - rho_oracle| < NEAR_TIE is
+    counted as a flipped near-tie and the rest of that node is skipped.
+  * Every test the oracle performed with |u - rho| < NEAR_TIE is counted as a
+    near-tie decision; these must stay below NEAR_TIE_SHARE of all decisions.
+  * A sequence whose oracle path crosses a flipped node is excluded from the path
+    and residual comparison (and counted).  All other sequences must have the same
+    accepted length and accepted tokens.
+  * Endpoint tokens are draws by inverse CDF; a different token is tolerated only
+    if it has positive oracle probability and u lies within NEAR_TIE (in CDF
+    units) of that token's oracle CDF interval.  Such cases are counted.
+  * Residual distributions agree within `residual_tol` max abs error.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import numpy as np
+
+from . import verify as oracle_verify, softmax as oracle_softmax, mcss as oracle_mcss
+
+NEAR_TIE = 1e-5
+NEAR_TIE_SHARE = 1e-4
+RESIDUAL_TOL = {"fp32": 1e-5, "bf16": 2e-3, "fp16": 2e-3}
+
+
+@dataclass
+class ParityReport:
+    n_sequences: int = 0
+    n_tests: int = 0                 # acceptance tests the oracle performed (all nodes)
+    n_near_tie: int = 0              # of those, |u - rho| < NEAR_TIE
+    n_flipped: int = 0               # nodes whose decision differs inside the near-tie band
+    n_excluded_sequences: int = 0    # sequences whose oracle path crosses a flipped node
+    n_bonus_tolerated: int = 0       # endpoint tokens that differ within the CDF tolerance
+    n_nodes_compared: int = 0
+    max_residual_err: float = 0.0
+    failures: List[str] = field(default_factory=list)
+
+    @property
+    def ok(self) -> bool:
+        return not self.failures
+
+    def summary(self) -> dict:
+        return {"sequences": self.n_sequences, "tests": self.n_tests, "near_ties": self.n_near_tie,
+                "flipped": self.n_flipped, "excluded_sequences": self.n_excluded_sequences,
+                "bonus_tolerated": self.n_bonus_tolerated, "max_residual_err": self.max_residual_err,
+                "failures": len(self.failures)}
+
+
+def _children(parent):
+    n = parent.shape[0]
+    first = np.full(n, -1, dtype=np.int64)
+    count = np.zeros(n, dtype=np.int64)
+    for c in range(1, n):
+        p = parent[c]
+        if count[p] == 0:
+            first[p] = c
+        count[p] += 1
+    return first, count
+
+
+def _bonus_tolerated(P: np.ndarray, g: int, u: float) -> bool:
+    if g < 0 or g >= P.shape[0] or not (P[g] > 0):
+        return False
+    cdf = np.cumsum(P) / P.sum()
+    lo = cdf[g - 1] if g > 0 else 0.0
+    return lo - NEAR_TIE <= u <= cdf[g] + NEAR_TIE
+
+
+def _node_residual(target_b, draft_b, parent, cand_b, unif_b, n, first, count, T, mode):
+    """Oracle residual of a single node (only used to judge a differing endpoint token)."""
+    p = oracle_softmax(target_b[n], T)
+    k = int(count[n])
+    if k == 0:
+        return p
+    q = oracle_softmax(draft_b[n], T)
+    ch = np.arange(first[n], first[n] + k)
+    r = oracle_mcss(p, q, cand_b[ch], unif_b[ch, 0].astype(np.float64), mode)
+    return r.p
+
+
+def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: str, *,
+            accept_len, tokens, residual=None, node_accept=None, node_bonus=None, status=None,
+            oracle_result=None, max_failures: int = 20) -> ParityReport:
+    """target/draft: float32 numpy (exact widening of the rounded logits); the keyword arrays are
+    the outputs under test (numpy)."""
+    parent = np.asarray(parent, dtype=np.int32)
+    ref = oracle_result if oracle_result is not None else oracle_verify(
+        target, draft if T > 0 else None, parent, cand, unif, T, mode)
+    B, n_nodes = cand.shape
+    first, count = _children(parent)
+    rep = ParityReport(n_sequences=B)
+    tol = RESIDUAL_TOL[dtype_name]
+
+    def fail(msg):
+        if len(rep.failures) < max_failures:
+            rep.failures.append(msg)
+
+    # decisions the oracle made, and how many sat inside the near-tie band
+    tested = ~np.isnan(ref.node_ratio)
+    tested[:, 0] = False
+    rep.n_tests = int(tested.sum())
+    if T > 0:
+        u0 = unif[:, :, 0].astype(np.float64)
+        near = tested & (ref.node_ratio >= 0) & (np.abs(u0 - ref.node_ratio) < NEAR_TIE)
+        rep.n_near_tie = int(near.sum())
+        if rep.n_near_tie > NEAR_TIE_SHARE * max(rep.n_tests, 1):
+            fail(f"{rep.n_near_tie} near-tie decisions out of {rep.n_tests} exceed the allowed share")
+
+    flipped = np.zeros((B, n_nodes), dtype=bool)
+    if node_accept is not None:
+        diff = np.argwhere(node_accept != ref.node_accept)
+        for b, n in diff:
+            ao, ag = int(ref.node_accept[b, n]), int(node_accept[b, n])
+            cands = [c for c in (ao, ag) if c >= 0]
+            i_star = min(cands)
+            in_range = first[n] <= i_star < first[n] + count[n]
+            rho = ref.node_ratio[b, i_star] if in_range else np.nan
+            u = float(unif[b, i_star, 0]) if in_range else np.nan
+            if T > 0 and in_range and rho >= 0 and abs(u - rho) < NEAR_TIE:
+                flipped[b, n] = True
+            else:
+                fail(f"seq {b} node {n}: accepted child {ag}, oracle {ao} (u={u}, rho={rho})")
+        rep.n_flipped = int(flipped.sum())
+        rep.n_nodes_compared = B * n_nodes
+
+    if node_bonus is not None:
+        both_stop = (ref.node_accept < 0) & ~flipped
+        if node_accept is not None:
+            both_stop &= node_accept < 0
+        diff = np.argwhere(both_stop & (node_bonus != ref.node_bonus))
+        for b, n in diff:
+            g = int(node_bonus[b, n])
+            okk = False
+            if T > 0:
+                P = _node_residual(target[b], None if draft is None else draft[b], parent, cand[b], unif[b], n,
+                                   first, count, T, mode)
+                okk = _bonus_tolerated(P, g, float(unif[b, n, 1]))
+            if okk:
+                rep.n_bonus_tolerated += 1
+            else:
+                fail(f"seq {b} node {n}: endpoint token {g}, oracle {int(ref.node_bonus[b, n])}")
+        acc_nodes = (ref.node_accept >= 0) & ~flipped
+        if node_accept is not None:
+            acc_nodes &= node_accept >= 0
+        bad = np.argwhere(acc_nodes & (node_bonus != -1))
+        for b, n in bad[:max_failures]:
+            fail(f"seq {b} node {n}: endpoint token set on a node that accepted a candidate")
+
+    # sequence level
+    for b in range(B):
+        n, path_flipped = 0, bool(flipped[b, 0])
+        while ref.node_accept[b, n] >= 0:
+            n = int(ref.node_accept[b, n])
+            path_flipped |= bool(flipped[b, n])
+        if path_flipped:
+            rep.n_excluded_sequences += 1
+            continue
+        L = int(ref.accept_len[b])
+        if int(accept_len[b]) != L:
+            fail(f"seq {b}: accepted length {int(accept_len[b])}, oracle {L}")
+            continue
+        if not np.array_equal(tokens[b, :L], ref.tokens[b, :L]):
+            fail(f"seq {b}: accepted tokens {tokens[b, :L].tolist()}, oracle {ref.tokens[b, :L].tolist()}")
+            continue
+        if not (tokens[b, L + 1:] == -1).all():
+            fail(f"seq {b}: padding after the endpoint token is not -1")
+        g, o = int(tokens[b, L]), int(ref.tokens[b, L])
+        if g != o:
+            if T > 0 and _bonus_tolerated(ref.residual[b], g, float(unif[b, n, 1])):
+                if node_bonus is None:
+                    rep.n_bonus_tolerated += 1
+            else:
+                fail(f"seq {b}: endpoint token {g}, oracle {o}")
+        if residual is not None:
+            err = float(np.abs(residual[b].astype(np.float64) - ref.residual[b]).max())
+            rep.max_residual_err = max(rep.max_residual_err, err)
+            if not err <= tol:
+                fail(f"seq {b}: residual max abs error {err:.3e} > {tol:.1e}")
+        if status is not None and int(status[b]) != int(ref.status[b]):
+            fail(f"seq {b}: status {int(status[b])}, oracle {int(ref.status[b])}")
+    return rep

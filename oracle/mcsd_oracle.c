@@ -219,7 +219,7 @@ static int32_t verify_node(int32_t n, int32_t n_nodes, int32_t n_internal, int32
              * 1 for a match and 0 otherwise */
             int32_t match = cand_b[first + i] == a;
             if (ratio_b) ratio_b[first + i] = match ? 1.0 : 0.0;
-            if (match) return first + i;
+            if (match) { *bonus = -1; return first + i; }
         }
         return -1;
     }

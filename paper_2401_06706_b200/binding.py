@@ -1,0 +1,258 @@
+"""Thin Python binding of libmcsd.so: argument marshalling only.
+
+Every step of the verification runs inside the CUDA library; this module turns
+torch tensors into raw pointers, fills the descriptor and raises on a non-zero
+return code.  It fails loudly when the library is missing: there is no CPU or
+eager fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmcsd.so")
+
+MCSD_DTYPE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
+STATUS_DEGENERATE, STATUS_BAD_TOKEN, STATUS_NO_MASS, STATUS_TIMEOUT = 1, 2, 4, 8
+MAX_NODES, MAX_CHILDREN, MAX_VOCAB = 512, 32, 65536
+
+EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host",
+           "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
+           "mcsd_version")
+
+
+class McsdDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_nodes", ctypes.c_int32), ("n_internal", ctypes.c_int32),
+                ("vocab", ctypes.c_int32), ("dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("ld_target", ctypes.c_int64), ("ld_draft", ctypes.c_int64),
+                ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t),
+                ("node_accept", ctypes.c_void_p), ("node_bonus", ctypes.c_void_p),
+                ("node_ratio", ctypes.c_void_p), ("out_status", ctypes.c_void_p)]
+
+
+class McsdError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"libmcsd error {code}: {text}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None):
+    """dlopen libmcsd.so and declare its signatures.  Raises if it has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise RuntimeError(f"{p} is missing: build it with `python -m paper_2401_06706_b200.build` "
+                           "(there is no fallback path)")
+    lib = ctypes.CDLL(p)
+    vp, i32, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float
+    dp = ctypes.POINTER(McsdDesc)
+    lib.mcsd_verify.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
+    lib.mcsd_verify.restype = ctypes.c_int
+    lib.mcsd_verify_nodes.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int]
+    lib.mcsd_verify_nodes.restype = ctypes.c_int
+    lib.mcsd_verify_walk.argtypes = [dp, vp, vp, vp, vp, f32, vp, vp, vp]
+    lib.mcsd_verify_walk.restype = ctypes.c_int
+    lib.mcsd_verify_host.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp, vp]
+    lib.mcsd_verify_host.restype = ctypes.c_int
+    lib.mcsd_workspace_bytes.argtypes = [dp]
+    lib.mcsd_workspace_bytes.restype = ctypes.c_size_t
+    lib.mcsd_tree_depth.argtypes = [vp, i32]
+    lib.mcsd_tree_depth.restype = ctypes.c_int
+    lib.mcsd_last_launch_count.argtypes = []
+    lib.mcsd_last_launch_count.restype = ctypes.c_int
+    lib.mcsd_status_string.argtypes = [ctypes.c_int]
+    lib.mcsd_status_string.restype = ctypes.c_char_p
+    lib.mcsd_version.argtypes = []
+    lib.mcsd_version.restype = ctypes.c_int
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().mcsd_status_string(int(code)).decode()
+
+
+def _check(code: int):
+    if code != 0:
+        raise McsdError(code, status_string(code))
+
+
+def mcsd_version() -> int:
+    return int(load_library().mcsd_version())
+
+
+def mcsd_tree_depth(parent) -> int:
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    rc = load_library().mcsd_tree_depth(parent.ctypes.data, parent.shape[0])
+    _check(rc if rc < 0 else 0)
+    return rc
+
+
+def mcsd_last_launch_count() -> int:
+    return int(load_library().mcsd_last_launch_count())
+
+
+def _n_internal(parent: np.ndarray) -> int:
+    has = np.zeros(parent.shape[0], dtype=bool)
+    if parent.shape[0] > 1:
+        has[parent[1:][parent[1:] >= 0]] = True
+    return int(has.sum())
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _row_stride(t: torch.Tensor) -> int:
+    """Elements between consecutive rows of a [B, rows, V] tensor whose rows are contiguous and
+    whose leading dimensions collapse to one stride."""
+    assert t.dim() == 3 and (t.shape[2] == 1 or t.stride(2) == 1), "vocabulary axis must be contiguous"
+    ld = t.stride(1) if t.shape[1] > 1 else max(t.shape[2], t.stride(1))
+    if t.shape[0] > 1:
+        assert t.stride(0) == ld * t.shape[1], "batch stride must equal rows * row stride"
+    return int(ld)
+
+
+@dataclass
+class VerifyOutput:
+    accept_len: torch.Tensor            # [B] int32
+    tokens: torch.Tensor                # [B, gamma+1] int32
+    residual: Optional[torch.Tensor]    # [B, V] float32
+    status: torch.Tensor                # [B] int32
+    node_accept: Optional[torch.Tensor] = None
+    node_bonus: Optional[torch.Tensor] = None
+    node_ratio: Optional[torch.Tensor] = None
+
+
+class Verifier:
+    """Holds the descriptor and device buffers for one (batch, tree, vocab, dtype) shape so that
+    repeated calls allocate nothing."""
+
+    def __init__(self, batch: int, parent, vocab: int, dtype: torch.dtype, device="cuda", *,
+                 want_residual: bool = True, node_outputs: bool = False, ld_target: Optional[int] = None,
+                 ld_draft: Optional[int] = None):
+        self.lib = load_library()
+        self.parent = np.ascontiguousarray(parent, dtype=np.int32)
+        self.device = torch.device(device)
+        self.batch, self.vocab, self.dtype = int(batch), int(vocab), dtype
+        self.n_nodes = int(self.parent.shape[0])
+        self.n_internal = _n_internal(self.parent)
+        gamma = self.lib.mcsd_tree_depth(self.parent.ctypes.data, self.n_nodes)
+        _check(gamma if gamma < 0 else 0)
+        self.gamma = gamma
+        self.desc = McsdDesc()
+        d = self.desc
+        d.batch, d.n_nodes, d.n_internal, d.vocab = self.batch, self.n_nodes, self.n_internal, self.vocab
+        d.dtype = MCSD_DTYPE[dtype]
+        d.ld_target = int(ld_target if ld_target is not None else vocab)
+        d.ld_draft = int(ld_draft if ld_draft is not None else vocab)
+        ws = int(self.lib.mcsd_workspace_bytes(ctypes.byref(d)))
+        if ws == 0:
+            _check(-2)
+        self.workspace = torch.empty(ws + 256, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        d.workspace = (base + 255) // 256 * 256
+        d.workspace_bytes = ws
+        i32 = dict(dtype=torch.int32, device=self.device)
+        self.accept_len = torch.empty(self.batch, **i32)
+        self.tokens = torch.empty((self.batch, self.gamma + 1), **i32)
+        self.residual = (torch.empty((self.batch, self.vocab), dtype=torch.float32, device=self.device)
+                         if want_residual else None)
+        self.status = torch.zeros(self.batch, **i32)
+        d.out_status = self.status.data_ptr()
+        self.node_accept = self.node_bonus = self.node_ratio = None
+        if node_outputs:
+            self.node_accept = torch.empty((self.batch, self.n_nodes), **i32)
+            self.node_bonus = torch.empty((self.batch, self.n_nodes), **i32)
+            self.node_ratio = torch.full((self.batch, self.n_nodes), float("nan"), dtype=torch.float32,
+                                         device=self.device)
+            d.node_accept = self.node_accept.data_ptr()
+            d.node_bonus = self.node_bonus.data_ptr()
+            d.node_ratio = self.node_ratio.data_ptr()
+
+    def _bind(self, target, draft):
+        assert target.dtype == self.dtype and target.shape == (self.batch, self.n_nodes, self.vocab)
+        self.desc.ld_target = _row_stride(target)
+        if draft is not None:
+            assert draft.dtype == self.dtype and draft.shape == (self.batch, self.n_internal, self.vocab)
+            self.desc.ld_draft = _row_stride(draft) if self.n_internal else self.vocab
+        self.desc.stream = torch.cuda.current_stream(self.device).cuda_stream
+
+    def _out(self) -> VerifyOutput:
+        return VerifyOutput(self.accept_len, self.tokens, self.residual, self.status, self.node_accept,
+                            self.node_bonus, self.node_ratio)
+
+    def mcsd_verify(self, target, draft, cand, unif, temperature: float, mode: int) -> VerifyOutput:
+        self._bind(target, draft)
+        if self.node_ratio is not None:
+            self.node_ratio.fill_(float("nan"))
+        _check(self.lib.mcsd_verify(ctypes.byref(self.desc), _ptr(target), _ptr(draft), self.parent.ctypes.data,
+                                    _ptr(cand), _ptr(unif), float(temperature), int(mode),
+                                    _ptr(self.accept_len), _ptr(self.tokens), _ptr(self.residual)))
+        return self._out()
+
+    def mcsd_verify_nodes(self, target, draft, cand, unif, temperature: float, mode: int) -> None:
+        self._bind(target, draft)
+        _check(self.lib.mcsd_verify_nodes(ctypes.byref(self.desc), _ptr(target), _ptr(draft),
+                                          self.parent.ctypes.data, _ptr(cand), _ptr(unif), float(temperature),
+                                          int(mode)))
+
+    def mcsd_verify_walk(self, target, draft, cand, temperature: float) -> VerifyOutput:
+        self._bind(target, draft)
+        _check(self.lib.mcsd_verify_walk(ctypes.byref(self.desc), _ptr(target), _ptr(draft),
+                                         self.parent.ctypes.data, _ptr(cand), float(temperature),
+                                         _ptr(self.accept_len), _ptr(self.tokens), _ptr(self.residual)))
+        return self._out()
+
+
+def mcsd_verify(target, draft, parent, cand, unif, temperature: float, mode: int, *,
+                want_residual: bool = True, node_outputs: bool = False) -> VerifyOutput:
+    """One-shot convenience wrapper: device tensors in, device tensors out."""
+    B, _, V = target.shape
+    v = Verifier(B, parent, V, target.dtype, target.device, want_residual=want_residual,
+                 node_outputs=node_outputs)
+    return v.mcsd_verify(target, draft, cand, unif, temperature, mode)
+
+
+def mcsd_verify_host(target, draft, parent, cand, unif, temperature: float, mode: int, *,
+                     want_residual: bool = True, out: Optional[dict] = None) -> VerifyOutput:
+    """Host tensors (CPU, ideally pinned) in, host tensors out; all copies happen inside the library."""
+    lib = load_library()
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    B, n_nodes, V = target.shape
+    assert not target.is_cuda and target.is_contiguous()
+    d = McsdDesc()
+    d.batch, d.n_nodes, d.n_internal, d.vocab = B, n_nodes, _n_internal(parent), V
+    d.dtype = MCSD_DTYPE[target.dtype]
+    d.ld_target = V
+    d.ld_draft = V
+    gamma = lib.mcsd_tree_depth(parent.ctypes.data, n_nodes)
+    _check(gamma if gamma < 0 else 0)
+    if out is None:
+        out = {}
+    pin = torch.cuda.is_available()
+    accept_len = out.get("accept_len", torch.empty(B, dtype=torch.int32, pin_memory=pin))
+    tokens = out.get("tokens", torch.empty((B, gamma + 1), dtype=torch.int32, pin_memory=pin))
+    residual = out.get("residual", torch.empty((B, V), dtype=torch.float32, pin_memory=pin)) if want_residual else None
+    status = out.get("status", torch.zeros(B, dtype=torch.int32, pin_memory=pin))
+    _check(lib.mcsd_verify_host(ctypes.byref(d), _ptr(target), _ptr(draft), parent.ctypes.data, _ptr(cand),
+                                _ptr(unif), float(temperature), int(mode), _ptr(accept_len), _ptr(tokens),
+                                _ptr(residual), _ptr(status)))
+    return VerifyOutput(accept_len, tokens, residual, status)

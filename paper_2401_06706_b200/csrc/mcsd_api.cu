@@ -1,0 +1,556 @@
+// Host side of libmcsd.so: argument validation, tree plan, launch configuration
+// and the extern "C" entry points declared in mcsd.h.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "mcsd_device.cuh"
+
+namespace mcsd {
+namespace {
+
+thread_local int g_last_launches = 0;
+
+struct TreePlan {
+    int gamma = 0;
+    uint16_t child_first[MCSD_MAX_NODES];
+    uint8_t child_count[MCSD_MAX_NODES];
+};
+
+// Checks the layout contract (level order, contiguous children, internal nodes
+// first) and fills the per-node child ranges.  Returns MCSD_OK or an error code.
+int plan_tree(const int32_t *parent, int n_nodes, int n_internal, TreePlan *plan)
+{
+    if (!parent) return MCSD_ERR_NULL;
+    if (n_nodes < 1) return MCSD_ERR_SHAPE;
+    if (n_nodes > MCSD_MAX_NODES) return MCSD_ERR_UNSUPPORTED;
+    if (parent[0] != -1) return MCSD_ERR_TREE;
+    std::vector<int> depth(n_nodes, 0);
+    std::memset(plan->child_first, 0, sizeof(plan->child_first));
+    std::memset(plan->child_count, 0, sizeof(plan->child_count));
+    int gamma = 0;
+    for (int n = 1; n < n_nodes; ++n) {
+        const int p = parent[n];
+        if (p < 0 || p >= n) return MCSD_ERR_TREE;
+        if (p < parent[n - 1]) return MCSD_ERR_TREE;  // level order <=> parents never decrease
+        if (plan->child_count[p] == 0) plan->child_first[p] = static_cast<uint16_t>(n);
+        if (plan->child_count[p] >= MCSD_MAX_CHILDREN) return MCSD_ERR_UNSUPPORTED;
+        ++plan->child_count[p];
+        depth[n] = depth[p] + 1;
+        if (depth[n] > gamma) gamma = depth[n];
+    }
+    if (n_internal >= 0) {
+        for (int n = 0; n < n_nodes; ++n)
+            if ((plan->child_count[n] > 0) != (n < n_internal)) return MCSD_ERR_TREE;
+    }
+    plan->gamma = gamma;
+    return MCSD_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Workspace {
+    int32_t *node_accept;
+    int32_t *node_bonus;
+    NodeStats *stats;
+    int32_t *status;
+    size_t bytes;
+};
+
+Workspace carve(void *base, long long n_items, int batch)
+{
+    Workspace w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        unsigned char *p = base ? static_cast<unsigned char *>(base) + off : nullptr;
+        off += align_up(bytes, 256);
+        return p;
+    };
+    w.node_accept = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
+    w.node_bonus = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
+    w.stats = reinterpret_cast<NodeStats *>(take(sizeof(NodeStats) * n_items));
+    w.status = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
+    w.bytes = off;
+    return w;
+}
+
+int check_desc(const mcsd_desc *d)
+{
+    if (!d) return MCSD_ERR_NULL;
+    if (d->batch < 0 || d->n_nodes < 1 || d->vocab < 1 || d->n_internal < 0 ||
+        d->n_internal > d->n_nodes)
+        return MCSD_ERR_SHAPE;
+    if (d->n_nodes > MCSD_MAX_NODES || d->vocab > MCSD_MAX_VOCAB) return MCSD_ERR_UNSUPPORTED;
+    if (static_cast<long long>(d->batch) * d->n_nodes > 0x7fffffffLL) return MCSD_ERR_UNSUPPORTED;
+    if (d->dtype != MCSD_DTYPE_F32 && d->dtype != MCSD_DTYPE_BF16 && d->dtype != MCSD_DTYPE_F16)
+        return MCSD_ERR_DTYPE;
+    if (d->ld_target < d->vocab) return MCSD_ERR_STRIDE;
+    return MCSD_OK;
+}
+
+int check_workspace(const mcsd_desc *d)
+{
+    const Workspace need = carve(nullptr, static_cast<long long>(d->batch) * d->n_nodes, d->batch);
+    if (!d->workspace) return MCSD_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d->workspace) % 256 != 0) return MCSD_ERR_WORKSPACE;
+    if (d->workspace_bytes < need.bytes) return MCSD_ERR_WORKSPACE;
+    return MCSD_OK;
+}
+
+int elem_bytes(int dtype) { return dtype == MCSD_DTYPE_F32 ? 4 : 2; }
+
+bool rows_aligned16(const void *base, long long ld, int dtype)
+{
+    return reinterpret_cast<uintptr_t>(base) % 16 == 0 && (ld * elem_bytes(dtype)) % 16 == 0;
+}
+
+// ---- node-kernel variants ---------------------------------------------------
+using NodeKernel = void (*)(const NodeParams);
+constexpr int kEptChoices[3] = {8, 16, 32};
+
+template <int DT, bool DIRECT>
+NodeKernel pick_ept(int ept)
+{
+    switch (ept) {
+    case 8: return node_kernel<DT, 8, DIRECT>;
+    case 16: return node_kernel<DT, 16, DIRECT>;
+    default: return node_kernel<DT, 32, DIRECT>;
+    }
+}
+NodeKernel pick_node_kernel(int dtype, int ept, bool direct)
+{
+    switch (dtype) {
+    case MCSD_DTYPE_F32: return direct ? pick_ept<MCSD_DTYPE_F32, true>(ept) : pick_ept<MCSD_DTYPE_F32, false>(ept);
+    case MCSD_DTYPE_BF16: return direct ? pick_ept<MCSD_DTYPE_BF16, true>(ept) : pick_ept<MCSD_DTYPE_BF16, false>(ept);
+    default: return direct ? pick_ept<MCSD_DTYPE_F16, true>(ept) : pick_ept<MCSD_DTYPE_F16, false>(ept);
+    }
+}
+
+int env_int(const char *name, int fallback)
+{
+    const char *v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : fallback;
+}
+
+struct NodeConfig {
+    int cluster, ept, slice;
+    bool direct;
+};
+
+// Smallest (cluster size x elements per thread) that holds one vocabulary row,
+// larger per-thread share first so that fewer CTAs have to agree per node.
+// MCSD_CLUSTER / MCSD_EPT / MCSD_DIRECT override the choice (tuning and tests).
+int choose_config(int vocab, int dtype, bool aligned, NodeConfig *cfg)
+{
+    const int vec = 16 / elem_bytes(dtype);
+    int best_c = 0, best_e = 0;
+    long long best_cap = -1;
+    const int force_c = env_int("MCSD_CLUSTER", 0), force_e = env_int("MCSD_EPT", 0);
+    for (int c = 1; c <= kMaxCluster; c *= 2) {
+        if (force_c && c != force_c) continue;
+        for (int ei = 2; ei >= 0; --ei) {
+            const int e = kEptChoices[ei];
+            if (force_e && e != force_e) continue;
+            const long long slice = align_up((vocab + c - 1) / c, vec);
+            if (slice > static_cast<long long>(kThreads) * e) continue;
+            const long long cap = static_cast<long long>(c) * e;
+            if (best_cap < 0 || cap < best_cap) { best_cap = cap; best_c = c; best_e = e; }
+        }
+    }
+    if (best_cap < 0) return MCSD_ERR_UNSUPPORTED;
+    cfg->cluster = best_c;
+    cfg->ept = best_e;
+    cfg->slice = static_cast<int>(align_up((vocab + best_c - 1) / best_c, vec));
+    cfg->direct = !aligned || env_int("MCSD_DIRECT", 0) != 0;
+    return MCSD_OK;
+}
+
+// Clusters that can be resident at once, cached per (device, kernel, cluster size).
+struct OccKey { int dev; NodeKernel fn; int cluster; int clusters; };
+std::mutex g_occ_mutex;
+std::vector<OccKey> g_occ;
+
+int resident_clusters(NodeKernel fn, int cluster, size_t smem, cudaStream_t stream)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    {
+        std::lock_guard<std::mutex> lock(g_occ_mutex);
+        for (const OccKey &k : g_occ)
+            if (k.dev == dev && k.fn == fn && k.cluster == cluster) return k.clusters;
+    }
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+        return -1;
+    // ask for the largest shared-memory carveout so that as many CTAs as the register
+    // budget allows can hold their staging buffers at once
+    cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    int n_sm = 0;
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(static_cast<unsigned>(cluster * n_sm * 4));
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, fn, &lc) != cudaSuccess || clusters < 1) {
+        cudaGetLastError();
+        return -1;
+    }
+    std::lock_guard<std::mutex> lock(g_occ_mutex);
+    g_occ.push_back({dev, fn, cluster, clusters});
+    return clusters;
+}
+
+struct Call {
+    const mcsd_desc *d;
+    TreePlan plan;
+    Workspace ws;
+    int32_t *node_accept, *node_bonus, *status;
+    cudaStream_t stream;
+};
+
+int prepare(const mcsd_desc *d, const int32_t *parent, Call *c)
+{
+    int rc = check_desc(d);
+    if (rc != MCSD_OK) return rc;
+    rc = plan_tree(parent, d->n_nodes, d->n_internal, &c->plan);
+    if (rc != MCSD_OK) return rc;
+    rc = check_workspace(d);
+    if (rc != MCSD_OK) return rc;
+    c->d = d;
+    c->ws = carve(d->workspace, static_cast<long long>(d->batch) * d->n_nodes, d->batch);
+    c->node_accept = d->node_accept ? d->node_accept : c->ws.node_accept;
+    c->node_bonus = d->node_bonus ? d->node_bonus : c->ws.node_bonus;
+    c->status = d->out_status ? d->out_status : c->ws.status;
+    c->stream = static_cast<cudaStream_t>(d->stream);
+    return MCSD_OK;
+}
+
+int check_common(const mcsd_desc *d, const void *target, const void *draft, const int32_t *cand,
+                 const float *unif, float T, int mode, bool need_unif)
+{
+    if (!target || !cand) return MCSD_ERR_NULL;
+    if (!(T >= 0.f) || std::isinf(T)) return MCSD_ERR_TEMPERATURE;
+    if (mode != MCSD_MODE_WITH_REPLACEMENT && mode != MCSD_MODE_WITHOUT_REPLACEMENT) return MCSD_ERR_MODE;
+    if (T > 0.f) {
+        if (need_unif && !unif) return MCSD_ERR_NULL;
+        if (d->n_internal > 0) {
+            if (!draft) return MCSD_ERR_NULL;
+            if (d->ld_draft < d->vocab) return MCSD_ERR_STRIDE;
+        }
+    }
+    return MCSD_OK;
+}
+
+int launch_nodes(const Call &c, const void *target, const void *draft, const int32_t *cand,
+                 const float *unif, float T, int mode)
+{
+    const mcsd_desc *d = c.d;
+    const long long n_items = static_cast<long long>(d->batch) * d->n_nodes;
+    if (n_items == 0) return MCSD_OK;
+    if (cudaMemsetAsync(c.status, 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
+        return MCSD_ERR_CUDA;
+
+    if (T == 0.f) {
+        ArgmaxParams p = {};
+        p.target = target; p.cand = cand;
+        p.node_accept = c.node_accept; p.node_bonus = c.node_bonus; p.node_ratio = d->node_ratio;
+        p.ld_t = d->ld_target;
+        p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
+        p.n_rows = static_cast<int32_t>(n_items);
+        p.vector_ok = rows_aligned16(target, d->ld_target, d->dtype) ? 1 : 0;
+        std::memcpy(p.child_first, c.plan.child_first, sizeof(p.child_first));
+        std::memcpy(p.child_count, c.plan.child_count, sizeof(p.child_count));
+        int dev = 0, n_sm = 148;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        const long long cap = static_cast<long long>(n_sm) * 8;   // 8 resident CTAs of 256 threads per SM
+        const unsigned grid = static_cast<unsigned>(n_items < cap ? n_items : cap);
+        switch (d->dtype) {
+        case MCSD_DTYPE_F32: argmax_kernel<MCSD_DTYPE_F32><<<grid, kThreads, 0, c.stream>>>(p); break;
+        case MCSD_DTYPE_BF16: argmax_kernel<MCSD_DTYPE_BF16><<<grid, kThreads, 0, c.stream>>>(p); break;
+        default: argmax_kernel<MCSD_DTYPE_F16><<<grid, kThreads, 0, c.stream>>>(p); break;
+        }
+        if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+        g_last_launches += 1;
+        return MCSD_OK;
+    }
+
+    const bool aligned = rows_aligned16(target, d->ld_target, d->dtype) &&
+        (d->n_internal == 0 || rows_aligned16(draft, d->ld_draft, d->dtype));
+    NodeConfig cfg;
+    int rc = choose_config(d->vocab, d->dtype, aligned, &cfg);
+    if (rc != MCSD_OK) return rc;
+    NodeKernel fn = pick_node_kernel(d->dtype, cfg.ept, cfg.direct);
+    const size_t smem = cfg.direct ? 0 : static_cast<size_t>(2) * kThreads * cfg.ept * elem_bytes(d->dtype);
+    const int resident = resident_clusters(fn, cfg.cluster, smem, c.stream);
+    if (resident < 1) return MCSD_ERR_CUDA;
+    const long long n_clusters = n_items < resident ? n_items : resident;
+
+    NodeParams p = {};
+    p.target = target; p.draft = draft; p.cand = cand; p.unif = unif;
+    p.node_accept = c.node_accept; p.node_bonus = c.node_bonus; p.node_ratio = d->node_ratio;
+    p.stats = c.ws.stats; p.status = c.status;
+    p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
+    p.B = d->batch; p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
+    p.slice = cfg.slice;
+    p.n_items = static_cast<int32_t>(n_items);
+    p.mode = mode;
+    p.scale = static_cast<float>(1.4426950408889634 / static_cast<double>(T));
+    std::memcpy(p.child_first, c.plan.child_first, sizeof(p.child_first));
+    std::memcpy(p.child_count, c.plan.child_count, sizeof(p.child_count));
+
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(static_cast<unsigned>(n_clusters * cfg.cluster));
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = c.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cfg.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
+        cudaGetLastError();
+        return MCSD_ERR_CUDA;
+    }
+    g_last_launches += 1;
+    return MCSD_OK;
+}
+
+int launch_walk(const Call &c, const void *target, const void *draft, const int32_t *cand, float T,
+                int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
+{
+    const mcsd_desc *d = c.d;
+    if (d->batch == 0) return MCSD_OK;
+    WalkParams p = {};
+    p.target = target; p.draft = draft; p.cand = cand;
+    p.node_accept = c.node_accept; p.node_bonus = c.node_bonus; p.stats = c.ws.stats;
+    p.out_accept_len = out_accept_len; p.out_tokens = out_tokens; p.out_residual = out_residual;
+    p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
+    p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab; p.gamma = c.plan.gamma;
+    p.scale = T > 0.f ? static_cast<float>(1.4426950408889634 / static_cast<double>(T)) : 0.f;
+    const unsigned gx = out_residual ? static_cast<unsigned>((d->vocab + kThreads * 4 - 1) / (kThreads * 4)) : 1u;
+    const dim3 grid(gx, static_cast<unsigned>(d->batch));
+    switch (d->dtype) {
+    case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32><<<grid, kThreads, 0, c.stream>>>(p); break;
+    case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16><<<grid, kThreads, 0, c.stream>>>(p); break;
+    default: walk_kernel<MCSD_DTYPE_F16><<<grid, kThreads, 0, c.stream>>>(p); break;
+    }
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches += 1;
+    return MCSD_OK;
+}
+
+}  // namespace
+}  // namespace mcsd
+
+using namespace mcsd;
+
+extern "C" {
+
+int mcsd_version(void) { return MCSD_VERSION; }
+
+const char *mcsd_status_string(int code)
+{
+    switch (code) {
+    case MCSD_OK: return "ok";
+    case MCSD_ERR_NULL: return "a required pointer is NULL";
+    case MCSD_ERR_SHAPE: return "batch, n_nodes, n_internal or vocab out of range";
+    case MCSD_ERR_DTYPE: return "unknown logit dtype";
+    case MCSD_ERR_MODE: return "unknown replacement mode";
+    case MCSD_ERR_TEMPERATURE: return "temperature is negative, NaN or infinite";
+    case MCSD_ERR_TREE: return "tree_parent breaks the layout contract";
+    case MCSD_ERR_STRIDE: return "row stride smaller than vocab";
+    case MCSD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MCSD_ERR_CUDA: return "a CUDA runtime call or kernel launch failed";
+    case MCSD_ERR_UNSUPPORTED: return "size beyond the library limits";
+    default: return "unknown code";
+    }
+}
+
+size_t mcsd_workspace_bytes(const mcsd_desc *desc)
+{
+    if (check_desc(desc) != MCSD_OK) return 0;
+    return carve(nullptr, static_cast<long long>(desc->batch) * desc->n_nodes, desc->batch).bytes;
+}
+
+int mcsd_tree_depth(const int32_t *tree_parent, int32_t n_nodes)
+{
+    TreePlan plan;
+    const int rc = plan_tree(tree_parent, n_nodes, -1, &plan);
+    return rc == MCSD_OK ? plan.gamma : rc;
+}
+
+int mcsd_last_launch_count(void) { return g_last_launches; }
+
+int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                      float temperature, int replacement_mode)
+{
+    Call c;
+    int rc = prepare(desc, tree_parent, &c);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0) return MCSD_OK;
+    rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
+                      replacement_mode, true);
+    if (rc != MCSD_OK) return rc;
+    return launch_nodes(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, replacement_mode);
+}
+
+int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, float temperature,
+                     int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
+{
+    Call c;
+    int rc = prepare(desc, tree_parent, &c);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0) return MCSD_OK;
+    rc = check_common(desc, target_logits, draft_logits, cand_tokens, nullptr, temperature,
+                      MCSD_MODE_WITH_REPLACEMENT, false);
+    if (rc != MCSD_OK) return rc;
+    if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
+    return launch_walk(c, target_logits, draft_logits, cand_tokens, temperature, out_accept_len,
+                       out_tokens, out_residual);
+}
+
+int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                float temperature, int replacement_mode, int32_t *out_accept_len,
+                int32_t *out_tokens, float *out_residual)
+{
+    Call c;
+    int rc = prepare(desc, tree_parent, &c);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0) return MCSD_OK;
+    rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
+                      replacement_mode, true);
+    if (rc != MCSD_OK) return rc;
+    if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
+    rc = launch_nodes(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, replacement_mode);
+    if (rc != MCSD_OK) return rc;
+    return launch_walk(c, target_logits, draft_logits, cand_tokens, temperature, out_accept_len,
+                       out_tokens, out_residual);
+}
+
+int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int replacement_mode, int32_t *out_accept_len,
+                     int32_t *out_tokens, float *out_residual, int32_t *out_status)
+{
+    int rc = check_desc(desc);
+    if (rc != MCSD_OK) return rc;
+    TreePlan plan;
+    rc = plan_tree(tree_parent, desc->n_nodes, desc->n_internal, &plan);
+    if (rc != MCSD_OK) return rc;
+    rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
+                      replacement_mode, true);
+    if (rc != MCSD_OK) return rc;
+    if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
+    const int B = desc->batch;
+    if (B == 0) return MCSD_OK;
+
+    const size_t es = elem_bytes(desc->dtype);
+    const bool use_draft = temperature > 0.f && desc->n_internal > 0;
+    const size_t t_seq = static_cast<size_t>(desc->n_nodes) * desc->ld_target * es;
+    const size_t d_seq = use_draft ? static_cast<size_t>(desc->n_internal) * desc->ld_draft * es : 0;
+    const size_t c_seq = sizeof(int32_t) * desc->n_nodes, u_seq = sizeof(float) * 2 * desc->n_nodes;
+    const size_t tok_seq = sizeof(int32_t) * (plan.gamma + 1), res_seq = sizeof(float) * desc->vocab;
+    // sequences per slice: about 256 MiB of logits, at least 1, at most ceil(B/2) so that
+    // two slices exist to overlap whenever B > 1
+    size_t per = (size_t(256) << 20) / (t_seq + d_seq ? t_seq + d_seq : 1);
+    if (per < 1) per = 1;
+    if (per > static_cast<size_t>((B + 1) / 2)) per = static_cast<size_t>((B + 1) / 2);
+    const int chunk = static_cast<int>(per);
+
+    struct Slot {
+        cudaStream_t stream = nullptr;
+        unsigned char *t = nullptr, *d = nullptr;
+        int32_t *cand = nullptr, *len = nullptr, *tok = nullptr, *status = nullptr;
+        float *unif = nullptr, *res = nullptr;
+        void *ws = nullptr;
+    } slot[2];
+    mcsd_desc cd = *desc;
+    cd.batch = chunk;
+    cd.node_accept = nullptr; cd.node_bonus = nullptr; cd.node_ratio = nullptr;
+    const size_t ws_bytes = mcsd_workspace_bytes(&cd);
+    bool ok = true;
+    auto chk = [&](cudaError_t e) { if (e != cudaSuccess) ok = false; return e == cudaSuccess; };
+    for (int s = 0; s < 2 && ok; ++s) {
+        Slot &sl = slot[s];
+        chk(cudaStreamCreateWithFlags(&sl.stream, cudaStreamNonBlocking));
+        chk(cudaMalloc(&sl.t, t_seq * chunk));
+        if (use_draft) chk(cudaMalloc(&sl.d, d_seq * chunk));
+        chk(cudaMalloc(&sl.cand, c_seq * chunk));
+        chk(cudaMalloc(&sl.unif, u_seq * chunk));
+        chk(cudaMalloc(&sl.len, sizeof(int32_t) * chunk));
+        chk(cudaMalloc(&sl.tok, tok_seq * chunk));
+        chk(cudaMalloc(&sl.status, sizeof(int32_t) * chunk));
+        if (out_residual) chk(cudaMalloc(&sl.res, res_seq * chunk));
+        chk(cudaMalloc(&sl.ws, ws_bytes));
+    }
+    int launches = 0;
+    for (int b0 = 0, i = 0; b0 < B && ok && rc == MCSD_OK; b0 += chunk, ++i) {
+        Slot &sl = slot[i & 1];
+        const int nb = (B - b0 < chunk) ? B - b0 : chunk;
+        const unsigned char *ht = static_cast<const unsigned char *>(target_logits) + t_seq * b0;
+        chk(cudaMemcpyAsync(sl.t, ht, t_seq * nb, cudaMemcpyHostToDevice, sl.stream));
+        if (use_draft) {
+            const unsigned char *hd = static_cast<const unsigned char *>(draft_logits) + d_seq * b0;
+            chk(cudaMemcpyAsync(sl.d, hd, d_seq * nb, cudaMemcpyHostToDevice, sl.stream));
+        }
+        chk(cudaMemcpyAsync(sl.cand, cand_tokens + static_cast<size_t>(b0) * desc->n_nodes, c_seq * nb,
+                            cudaMemcpyHostToDevice, sl.stream));
+        if (uniforms)
+            chk(cudaMemcpyAsync(sl.unif, uniforms + static_cast<size_t>(b0) * 2 * desc->n_nodes, u_seq * nb,
+                                cudaMemcpyHostToDevice, sl.stream));
+        cd.batch = nb;
+        cd.stream = sl.stream;
+        cd.workspace = sl.ws;
+        cd.workspace_bytes = ws_bytes;
+        cd.out_status = sl.status;
+        if (ok)
+            rc = mcsd_verify(&cd, sl.t, sl.d, tree_parent, sl.cand, uniforms ? sl.unif : nullptr, temperature,
+                             replacement_mode, sl.len, sl.tok, sl.res);
+        launches += g_last_launches;
+        chk(cudaMemcpyAsync(out_accept_len + b0, sl.len, sizeof(int32_t) * nb, cudaMemcpyDeviceToHost, sl.stream));
+        chk(cudaMemcpyAsync(out_tokens + static_cast<size_t>(b0) * (plan.gamma + 1), sl.tok, tok_seq * nb,
+                            cudaMemcpyDeviceToHost, sl.stream));
+        if (out_residual)
+            chk(cudaMemcpyAsync(out_residual + static_cast<size_t>(b0) * desc->vocab, sl.res, res_seq * nb,
+                                cudaMemcpyDeviceToHost, sl.stream));
+        if (out_status)
+            chk(cudaMemcpyAsync(out_status + b0, sl.status, sizeof(int32_t) * nb, cudaMemcpyDeviceToHost, sl.stream));
+    }
+    for (int s = 0; s < 2; ++s) {
+        Slot &sl = slot[s];
+        if (sl.stream) { chk(cudaStreamSynchronize(sl.stream)); }
+    }
+    for (int s = 0; s < 2; ++s) {
+        Slot &sl = slot[s];
+        cudaFree(sl.t); cudaFree(sl.d); cudaFree(sl.cand); cudaFree(sl.unif); cudaFree(sl.len);
+        cudaFree(sl.tok); cudaFree(sl.status); cudaFree(sl.res); cudaFree(sl.ws);
+        if (sl.stream) cudaStreamDestroy(sl.stream);
+    }
+    g_last_launches = launches;
+    if (rc != MCSD_OK) return rc;
+    if (!ok) { cudaGetLastError(); return MCSD_ERR_CUDA; }
+    return MCSD_OK;
+}
+
+}  // extern "C"

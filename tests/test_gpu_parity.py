@@ -1,0 +1,248 @@
+"""Parity of the CUDA library (called through its C ABI) with the CPU oracle on the same
+seeded inputs.  Tolerances: accept decisions and tokens bit-exact except near-ties
+|u - rho| < 1e-5 (counted, <= 0.01 % of decisions); residual max abs error <= 1e-5 for fp32
+logits and <= 2e-3 for bf16/fp16 logits."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2401_06706_b200 import binding, synth
+from gpu_util import assert_parity, run_library, to_np
+
+pytestmark = pytest.mark.gpu
+
+NAMED = synth.named_workloads()
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    binding.load_library()
+
+
+@pytest.mark.parametrize("name", ["cfg1_tiny", "cfg2_b8_with", "cfg2_b8_without", "cfg3_greedy", "cfg4_opt"])
+def test_named_configurations_full_parity(name):
+    inp = synth.make_inputs(NAMED[name], "cuda")
+    _, out = run_library(inp)
+    rep = assert_parity(inp, out)
+    assert rep.n_tests > 0 and rep.n_excluded_sequences == 0
+    print(name, rep.summary())
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16", "fp16"])
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("vocab,kconfig", [
+    (7, "2x2"), (8, "3"), (96, "1x1x1"), (1000, "4x2"), (2048, "2x2x2"), (2049, "2"),
+    (8200, "8x1"), (32000, "2x2"), (32008, "4"), (50272, "2x2"), (65536, "2"),
+])
+def test_shapes_spanning_tiles_and_ragged_tails(vocab, kconfig, mode, dtype):
+    if mode == 1 and vocab < 16 and max(synth.parse_kconfig(kconfig)) > 3:
+        pytest.skip("not enough distinct tokens")
+    w = synth.Workload(f"edge_{vocab}_{kconfig}", 5, vocab, kconfig, dtype, "normal", 2.5, 0.9, 1.2, 1.0,
+                       mode, 1234 + vocab)
+    inp = synth.make_inputs(w, "cuda")
+    _, out = run_library(inp)
+    assert_parity(inp, out)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("vocab", [1001, 32001, 50257])
+def test_unaligned_rows_take_the_plain_load_path(vocab, dtype):
+    """A contiguous tensor whose row length is not a multiple of 16 bytes."""
+    w = synth.Workload("unaligned", 3, vocab, "3x2", dtype, "normal", 2.5, 1.0, 1.0, 0.9, 1, 77 + vocab)
+    inp = synth.make_inputs(w, "cuda")
+    assert (vocab * inp.target.element_size()) % 16 != 0
+    _, out = run_library(inp)
+    assert_parity(inp, out)
+
+
+def test_padded_row_stride():
+    w = synth.Workload("strided", 4, 5000, "2x2", "fp16", "normal", 2.5, 1.0, 1.0, 1.0, 0, 4242)
+    inp = synth.make_inputs(w, "cuda")
+    ld = 5120
+    st = inp.stats
+    tpad = torch.full((4, st["n_nodes"], ld), 30.0, dtype=torch.float16, device="cuda")
+    dpad = torch.full((4, st["n_internal"], ld), 30.0, dtype=torch.float16, device="cuda")
+    tpad[:, :, :5000] = inp.target
+    dpad[:, :, :5000] = inp.draft
+    v = binding.Verifier(4, inp.parent, 5000, torch.float16, "cuda", node_outputs=True)
+    out = v.mcsd_verify(tpad[:, :, :5000], dpad[:, :, :5000], inp.cand, inp.unif, 1.0, 0)
+    torch.cuda.synchronize()
+    assert v.desc.ld_target == ld
+    assert_parity(inp, out)
+
+
+@pytest.mark.parametrize("cluster,ept", [(1, 32), (2, 16), (4, 8), (8, 8), (8, 32), (2, 32)])
+def test_forced_cluster_shapes(cluster, ept, monkeypatch):
+    """Every cluster size / per-thread share computes the same thing."""
+    monkeypatch.setenv("MCSD_CLUSTER", str(cluster))
+    monkeypatch.setenv("MCSD_EPT", str(ept))
+    vocab = min(cluster * ept * 256 - 24, 9000)
+    w = synth.Workload("forced", 6, vocab, "4x2x1", "fp32", "normal", 2.5, 1.0, 1.0, 1.0, 1, 31 + cluster + ept)
+    inp = synth.make_inputs(w, "cuda")
+    _, out = run_library(inp)
+    assert_parity(inp, out)
+
+
+def test_direct_path_matches_bulk_copy_path(monkeypatch):
+    w = synth.Workload("direct", 6, 32000, "4x2", "bf16", "normal", 2.5, 0.8, 1.5, 1.0, 0, 99)
+    inp = synth.make_inputs(w, "cuda")
+    _, a = run_library(inp)
+    a_acc, a_bon, a_res = to_np(a.node_accept), to_np(a.node_bonus), to_np(a.residual)
+    monkeypatch.setenv("MCSD_DIRECT", "1")
+    _, b = run_library(inp)
+    assert np.array_equal(a_acc, to_np(b.node_accept)) and np.array_equal(a_bon, to_np(b.node_bonus))
+    assert np.array_equal(a_res, to_np(b.residual))
+    assert_parity(inp, b)
+
+
+def test_root_only_tree_and_empty_batch():
+    w = synth.Workload("root_only", 9, 4096, "", "fp32", "normal", 2.0, 1.0, 1.0, 1.0, 0, 5)
+    inp = synth.make_inputs(w, "cuda")
+    assert inp.stats["n_nodes"] == 1 and inp.draft is None
+    _, out = run_library(inp)
+    rep = assert_parity(inp, out)
+    assert (to_np(out.accept_len) == 0).all()
+    v = binding.Verifier(0, inp.parent, 4096, torch.float32, "cuda")
+    out0 = v.mcsd_verify(inp.target[:0], None, inp.cand[:0], inp.unif[:0], 1.0, 0)
+    torch.cuda.synchronize()
+    assert out0.accept_len.numel() == 0
+
+
+def test_wide_and_deep_trees():
+    for kc, seed in (("32", 1), ("16x2", 2), ("1x1x1x1x1x1x1x1", 3), ("4x4x2x2x1", 4)):
+        w = synth.Workload("tree_" + kc, 3, 3000, kc, "fp32", "normal", 2.5, 1.0, 2.0, 1.0, 1, 600 + seed)
+        inp = synth.make_inputs(w, "cuda")
+        _, out = run_library(inp)
+        assert_parity(inp, out)
+
+
+def test_temperatures():
+    for T in (0.3, 0.7, 1.0, 1.7):
+        w = synth.Workload("temp", 8, 6000, "3x2x1", "fp16", "gumbel", 2.0, 1.0, 1.2, T, 1, int(T * 100))
+        inp = synth.make_inputs(w, "cuda")
+        _, out = run_library(inp)
+        assert_parity(inp, out)
+
+
+def test_degenerate_inputs_set_status_and_never_hang():
+    w = synth.Workload("degenerate", 6, 4000, "3x2", "fp32", "normal", 2.0, 1.0, 1.0, 1.0, 1, 808)
+    inp = synth.make_inputs(w, "cuda")
+    # sequence 0: an out-of-range candidate as first child of the root (forced rejection)
+    inp.cand[0, 1] = 4000
+    # sequence 1: duplicate siblings in the without-replacement mode
+    inp.cand[1, 2] = inp.cand[1, 1]
+    # sequence 2: -inf logits on half of the draft row of the root (probability 0 is legal)
+    inp.draft[2, 0, ::2] = float("-inf")
+    # sequence 3: target equals draft at the root: candidates are accepted unless u is ~1
+    inp.draft[3, 0] = inp.target[3, 0]
+    # sequence 4: a negative candidate
+    inp.cand[4, 3] = -5
+    _, out = run_library(inp)
+    rep = assert_parity(inp, out)
+    st = to_np(out.status)
+    assert st[0] & binding.STATUS_BAD_TOKEN
+    assert not (st & binding.STATUS_TIMEOUT).any()
+
+
+def test_argmax_ties_take_the_lowest_index():
+    w = synth.Workload("ties", 16, 3001, "4x2", "fp16", "normal", 3.0, 1.0, 2.0, 0.0, 0, 321)
+    inp = synth.make_inputs(w, "cuda")
+    # quantise hard so that every row has many equal maxima
+    inp.target.copy_((inp.target.float() / 4).round().clamp(-1, 1).to(torch.float16))
+    first, count = synth.children_ranges(inp.parent)
+    amax = inp.target.float().cpu().numpy().argmax(axis=-1)          # numpy returns the first maximum
+    inp.cand[:, 1] = torch.from_numpy(amax[:, 0]).to(inp.cand)        # make the root accept child 1
+    _, out = run_library(inp)
+    assert_parity(inp, out)
+    assert (to_np(out.accept_len) >= 1).all()
+
+
+def test_staged_entry_points_equal_the_fused_call():
+    w = NAMED["cfg2_b8_without"]
+    inp = synth.make_inputs(w, "cuda")
+    v, out = run_library(inp)
+    ref = (to_np(out.accept_len).copy(), to_np(out.tokens).copy(), to_np(out.residual).copy())
+    v2 = binding.Verifier(w.batch, inp.parent, w.vocab, torch.bfloat16, "cuda")
+    v2.mcsd_verify_nodes(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+    o2 = v2.mcsd_verify_walk(inp.target, inp.draft, inp.cand, w.temperature)
+    torch.cuda.synchronize()
+    assert np.array_equal(ref[0], to_np(o2.accept_len)) and np.array_equal(ref[1], to_np(o2.tokens))
+    assert np.array_equal(ref[2], to_np(o2.residual))
+    assert binding.mcsd_last_launch_count() == 1
+
+
+def test_repeated_calls_are_bit_identical():
+    inp = synth.make_inputs(NAMED["cfg4_opt"], "cuda")
+    v, out = run_library(inp)
+    first = [to_np(x).copy() for x in (out.accept_len, out.tokens, out.residual, out.node_accept, out.node_bonus)]
+    for _ in range(3):
+        out = v.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, 0.7, 1)
+        torch.cuda.synchronize()
+        again = [to_np(x) for x in (out.accept_len, out.tokens, out.residual, out.node_accept, out.node_bonus)]
+        for a, b in zip(first, again):
+            assert np.array_equal(a, b, equal_nan=True)
+
+
+def test_host_buffer_entry_point():
+    for name in ("cfg2_b8_with", "cfg3_greedy"):
+        w = NAMED[name]
+        inp = synth.make_inputs(w, "cuda")
+        _, dev = run_library(inp, node_outputs=False)
+        host = binding.mcsd_verify_host(inp.target.cpu().pin_memory(),
+                                        None if inp.draft is None else inp.draft.cpu().pin_memory(),
+                                        inp.parent, inp.cand.cpu().pin_memory(), inp.unif.cpu().pin_memory(),
+                                        w.temperature, w.mode)
+        assert np.array_equal(to_np(dev.accept_len), host.accept_len.numpy())
+        assert np.array_equal(to_np(dev.tokens), host.tokens.numpy())
+        assert np.array_equal(to_np(dev.residual), host.residual.numpy())
+
+
+@pytest.mark.parametrize("idx", [0, 37, 95, 141, 150, 208, 262, 299])
+def test_sweep_points_sampled(idx):
+    """Points of the throughput sweep (both dtypes, small and large batches); parity on 16
+    sequences of each, the library running the whole batch in the launch shape the bench times."""
+    w = synth.sweep_workloads()[idx]
+    if w.batch > 64:
+        w = synth.Workload(w.name, 64, w.vocab, w.kconfig, w.dtype, w.target_dist, w.target_scale,
+                           w.draft_gain, w.draft_sigma, w.temperature, w.mode, w.seed)
+    inp = synth.make_inputs(w, "cuda")
+    _, out = run_library(inp)
+    assert_parity(inp, out, 0, min(16, w.batch))
+
+
+@pytest.mark.skipif(os.environ.get("MCSD_SKIP_LARGE") == "1", reason="large case disabled")
+def test_largest_configuration_sampled_parity_and_properties():
+    """B = 512, 4x4x2x2x1, fp32 (19.5 GB of logits), in the launch shape the bench times: oracle
+    parity on sampled sequences, structural properties on all of them."""
+    w = NAMED["cfg5_largest"]
+    inp = synth.make_inputs(w, "cuda")
+    _, out = run_library(inp)
+    for b0 in (0, 255, 500):
+        assert_parity(inp, out, b0, b0 + 6)
+    acc, bon = to_np(out.node_accept), to_np(out.node_bonus)
+    tok, ln = to_np(out.tokens), to_np(out.accept_len)
+    first, count = synth.children_ranges(inp.parent)
+    parent = inp.parent
+    cand = to_np(inp.cand)
+    assert (to_np(out.status) == 0).all()
+    for n in range(parent.shape[0]):
+        a = acc[:, n]
+        ok = (a == -1) | ((a >= first[n]) & (a < first[n] + count[n]))
+        assert ok.all()
+        assert ((bon[:, n] >= 0) == (a == -1)).all()
+    assert ((bon >= -1) & (bon < w.vocab)).all()
+    for b in range(w.batch):
+        n = 0
+        for i in range(ln[b]):
+            n = acc[b, n]
+            assert tok[b, i] == cand[b, n]
+        assert acc[b, n] == -1 and tok[b, ln[b]] == bon[b, n] and (tok[b, ln[b] + 1:] == -1).all()
+    res = out.residual
+    s = res.sum(dim=1)
+    assert float((s - 1).abs().max()) < 1e-4 and float(res.min()) >= 0.0
+    end = torch.from_numpy(tok[np.arange(w.batch), ln]).to(res.device).long()
+    assert bool((res.gather(1, end[:, None]) > 0).all())       # the endpoint token has positive mass
+    assert 0.5 < ln.mean() < 4.5
