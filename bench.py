@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the MCSD verification step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole hot path (per-node softmax statistics, rejection loop,
+endpoint tokens, tree walk, terminal residual) over one batch of synthetic trees whose
+logits are already resident in HBM.  The default workload is the largest point of the
+throughput sweep (batch 512, k-config 4x4x2x2x1, vocabulary 32000, fp32 logits, 19.5 GB of
+logits), which is the configuration the bandwidth target is quoted on.  Prints ONE JSON
+line (rank 0).  With --impl reference the CPU oracle is timed on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2401_06706_b200 import synth
+
+METRIC = "verified_tree_nodes_per_sec"
+UNIT = "nodes/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+# ----------------------------------------------------------------------------- helpers
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def recorded_traffic(workload_name: str, units: int):
+    """DRAM bytes per launch of the node kernel from the committed ncu capture, scaled by the
+    number of tree nodes when the capture ran a smaller batch of the same workload."""
+    path = os.path.join(ROOT, "profiles", "node_kernel_traffic.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f)[workload_name]
+        return float(rec["dram_bytes_per_launch"]) * units / float(rec["units_per_launch"])
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.15] or [r for (_, r) in self.rows]
+        for row in rows:
+            parts = [p.strip() for p in row.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def pick_workload(name: str) -> synth.Workload:
+    named = synth.named_workloads()
+    if name in named:
+        return named[name]
+    for w in synth.sweep_workloads():
+        if w.name == name:
+            return w
+    raise SystemExit(f"unknown workload {name!r}; named: {sorted(named)}")
+
+
+def shard_for_rank(w: synth.Workload, rank: int, world: int) -> synth.Workload:
+    """Weak scaling: every rank verifies its own batch of the same shape (sequences are
+    independent, so there is no data-path collective); seeds differ per rank."""
+    from dataclasses import replace
+    return replace(w, seed=w.seed + 7919 * rank) if world > 1 else w
+
+
+def oracle_sample(inp: synth.Inputs, n_seq: int):
+    """Times the CPU oracle, as it stands, on the first n_seq sequences."""
+    import oracle
+    w = inp.workload
+    n_seq = min(n_seq, w.batch)
+    t, d, c, u = inp.host_f32(0, n_seq)
+    oracle.verify(t[:1], None if d is None or w.temperature == 0 else d[:1], inp.parent, c[:1], u[:1],
+                  w.temperature, w.mode, want_residual=True)          # loads the library
+    t0 = time.perf_counter()
+    res = oracle.verify(t, d if w.temperature > 0 else None, inp.parent, c, u, w.temperature, w.mode)
+    dt = time.perf_counter() - t0
+    nodes = n_seq * inp.stats["n_draft"]
+    return {"value": nodes / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {n_seq} of {w.batch} sequences of the same inputs, {dt:.2f} s wall, all-node form, "
+                      f"OpenMP over sequences"}, res
+
+
+# ----------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    w = pick_workload(args.workload)
+    n_seq = min(w.batch, args.oracle_seqs)
+    from dataclasses import replace
+    sample = replace(w, batch=n_seq)
+    inp = synth.make_inputs(sample, "cpu")
+    t, d, c, u = inp.host_f32()
+    dd = d if w.temperature > 0 else None
+    for _ in range(max(args.warmup, 1)):
+        oracle.verify(t[:2], None if dd is None else dd[:2], inp.parent, c[:2], u[:2], w.temperature, w.mode)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.verify(t, dd, inp.parent, c, u, w.temperature, w.mode)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n_seq * inp.stats["n_draft"] / dt
+    desc = f"{n_seq} sequences of workload {w.name} per step (bounded sample of its {w.batch}), generated on the CPU"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w, inp.stats, sample_batch=n_seq),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w: synth.Workload, st, **extra):
+    cfg = {"workload": w.name, "batch": w.batch, "vocab": w.vocab, "kconfig": w.kconfig,
+           "logit_dtype": w.dtype, "draft_nodes_per_tree": st["n_draft"], "target_rows_per_tree": st["n_nodes"],
+           "draft_rows_per_tree": st["n_internal"], "temperature": w.temperature,
+           "replacement_mode": "without" if w.mode == 1 else "with", "target_dist": w.target_dist,
+           "target_scale": w.target_scale, "draft_gain": w.draft_gain, "draft_sigma": w.draft_sigma,
+           "seed": w.seed}
+    cfg.update(extra)
+    return cfg
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+def run_cuda(args):
+    from paper_2401_06706_b200 import binding
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        dist = None
+        torch.cuda.set_device(0)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    binding.load_library()       # raises if the CUDA library is missing: no fallback
+
+    w = shard_for_rank(pick_workload(args.workload), rank, world)
+    inp = synth.make_inputs(w, dev)
+    st = inp.stats
+    ver = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[w.dtype], dev)
+    draft = inp.draft if w.temperature > 0 else None
+    nodes_per_step = w.batch * st["n_draft"]
+
+    def step(events=None):
+        if events is None:
+            ver.mcsd_verify(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
+            return
+        e0, e1 = events
+        e0.record()
+        ver.mcsd_verify_nodes(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
+        e1.record()
+        ver.mcsd_verify_walk(inp.target, draft, inp.cand, w.temperature)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    launches_per_step = 0
+    ver.mcsd_verify_nodes(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
+    launches_per_step += binding.mcsd_last_launch_count()
+    ver.mcsd_verify_walk(inp.target, draft, inp.cand, w.temperature)
+    launches_per_step += binding.mcsd_last_launch_count()
+    torch.cuda.synchronize()
+
+    # timed region: K steps between barriers and synchronisations, CUDA events on the
+    # launching stream; the node kernel of every step is bracketed by its own events
+    node_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_host0 = time.time()
+    start.record()
+    for i in range(args.steps):
+        step(node_events[i])
+    stop.record()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    t_host1 = time.time()
+    elapsed_ms = start.elapsed_time(stop)
+    node_ms = [a.elapsed_time(b) for a, b in node_events]
+    if dist:
+        tt = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tt.item())
+    clocks = sampler.stop(t_host0, t_host1) if sampler else None
+    status_bits = int(ver.status.max().item()) if w.batch else 0
+
+    ms_per_step = elapsed_ms / args.steps
+    value = world * nodes_per_step / (ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel (the per-node kernel): algorithmic bytes per launch =
+    # every target row once + every draft row once (none at temperature 0) + 12 bytes of
+    # candidate token and uniforms per node
+    algo_bytes = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
+    node_ms_avg = sum(node_ms) / len(node_ms)
+    achieved = algo_bytes / (node_ms_avg * 1e-3) / 1e9
+    peak, peak_kind = measured_peaks()
+    roofline = {"bound": "hbm", "kernel": "node_kernel" if w.temperature > 0 else "argmax_kernel",
+                "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_avg": node_ms_avg,
+                "kernel_ms_min": min(node_ms), "step_share": node_ms_avg / ms_per_step,
+                "traffic": recorded_traffic(w.name, w.batch * st["n_nodes"])}
+
+    # end to end through the host-buffer entry point: pinned host inputs, copies inside
+    e2e = None
+    if rank == 0 or world > 1:
+        e2e = run_e2e(args, w, inp, dist, world, dev)
+
+    cpu_baseline = None
+    parity = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline, ref = oracle_sample(inp, args.oracle_seqs)
+        parity = parity_on_sample(inp, ver, ref, min(args.oracle_seqs, w.batch))
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": workload_config(w, st, parallelism=f"replicas x{world} (batch split, no collective)",
+                                          l2="inputs (%.2f GB per GPU) far larger than the 126 MB L2" %
+                                          (inp.logit_bytes() / 1e9) if inp.logit_bytes() > 4 * 126e6 else
+                                          "inputs smaller than 4x L2: latency/L2-bound point",
+                                          logit_gb_per_gpu=inp.logit_bytes() / 1e9),
+                "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+                "hbm_gbs_whole_step": algo_bytes / (ms_per_step * 1e-3) / 1e9,
+                "device_status_bits": status_bits, "parity_on_oracle_sample": parity}
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+def parity_on_sample(inp, ver, ref, n_seq):
+    from oracle import compare
+    w = inp.workload
+    t, d, c, u = inp.host_f32(0, n_seq)
+    rep = compare.compare(t, d, inp.parent, c, u, w.temperature, w.mode, w.dtype,
+                          accept_len=ver.accept_len[:n_seq].cpu().numpy(), tokens=ver.tokens[:n_seq].cpu().numpy(),
+                          residual=ver.residual[:n_seq].cpu().numpy(), status=ver.status[:n_seq].cpu().numpy(),
+                          oracle_result=ref)
+    out = rep.summary()
+    out["ok"] = rep.ok
+    out["accept_len_mean"] = float(ref.accept_len.mean())
+    return out
+
+
+def run_e2e(args, w, inp, dist, world, dev):
+    from paper_2401_06706_b200 import binding
+    from dataclasses import replace
+    nb = min(w.batch, args.e2e_batch)
+    st = inp.stats
+    pin = lambda t: None if t is None else t[:nb].cpu().pin_memory()
+    target, cand, unif = pin(inp.target), pin(inp.cand), pin(inp.unif)
+    draft = pin(inp.draft) if w.temperature > 0 else None
+    out = {"accept_len": torch.empty(nb, dtype=torch.int32).pin_memory(),
+           "tokens": torch.empty((nb, st["gamma"] + 1), dtype=torch.int32).pin_memory(),
+           "residual": torch.empty((nb, w.vocab), dtype=torch.float32).pin_memory(),
+           "status": torch.zeros(nb, dtype=torch.int32).pin_memory()}
+    h2d = sum(t.numel() * t.element_size() for t in (target, draft, cand, unif) if t is not None)
+    d2h = sum(t.numel() * t.element_size() for t in out.values())
+
+    def step():
+        binding.mcsd_verify_host(target, draft, inp.parent, cand, unif, w.temperature, w.mode, out=out)
+
+    step()
+    steps = max(1, min(args.steps, args.e2e_steps))
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()                      # synchronises internally before it returns
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    if dist:
+        tt = torch.tensor([dt], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dt = float(tt.item())
+    value = world * nb * st["n_draft"] * steps / dt
+    return {"value": value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": dt / steps * 1e3, "steps": steps, "batch": nb,
+            "note": "mcsd_verify_host on pinned host buffers; device allocation, copies in both directions and "
+                    "kernels inside the timed region; bound by the host link"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="cfg5_largest")
+    ap.add_argument("--oracle-seqs", type=int, default=256,
+                    help="sequences of the workload the CPU oracle is timed on")
+    ap.add_argument("--e2e-batch", type=int, default=128, help="sequences per end-to-end step")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
