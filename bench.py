@@ -117,14 +117,17 @@ def dist_env():
     return rank, world, local
 
 
-def pick_workload(name: str) -> synth.Workload:
+def pick_workload(name: str, batch: int = 0) -> synth.Workload:
+    from dataclasses import replace
     named = synth.named_workloads()
-    if name in named:
-        return named[name]
-    for w in synth.sweep_workloads():
-        if w.name == name:
-            return w
-    raise SystemExit(f"unknown workload {name!r}; named: {sorted(named)}")
+    found = named.get(name)
+    if found is None:
+        for w in synth.sweep_workloads():
+            if w.name == name:
+                found = w
+    if found is None:
+        raise SystemExit(f"unknown workload {name!r}; named: {sorted(named)}")
+    return replace(found, batch=batch) if batch > 0 else found
 
 
 def shard_for_rank(w: synth.Workload, rank: int, world: int) -> synth.Workload:
@@ -157,15 +160,24 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    w = pick_workload(args.workload)
-    n_seq = min(w.batch, args.oracle_seqs)
+    w = pick_workload(args.workload, args.batch)
     from dataclasses import replace
+    # size the per-step sample so that the whole run takes about a minute of wall time
+    probe = synth.make_inputs(replace(w, batch=min(w.batch, 8)), "cpu")
+    t, d, c, u = probe.host_f32()
+    dd = d if w.temperature > 0 else None
+    oracle.verify(t[:1], None if dd is None else dd[:1], probe.parent, c[:1], u[:1], w.temperature, w.mode)
+    t0 = time.perf_counter()
+    oracle.verify(t, dd, probe.parent, c, u, w.temperature, w.mode)
+    per_seq = (time.perf_counter() - t0) / t.shape[0]
+    budget = 60.0 / max(args.steps + max(args.warmup, 1), 1)
+    n_seq = int(max(1, min(w.batch, args.oracle_seqs, budget / max(per_seq, 1e-9))))
     sample = replace(w, batch=n_seq)
     inp = synth.make_inputs(sample, "cpu")
     t, d, c, u = inp.host_f32()
     dd = d if w.temperature > 0 else None
     for _ in range(max(args.warmup, 1)):
-        oracle.verify(t[:2], None if dd is None else dd[:2], inp.parent, c[:2], u[:2], w.temperature, w.mode)
+        oracle.verify(t, dd, inp.parent, c, u, w.temperature, w.mode)
     t0 = time.perf_counter()
     for _ in range(args.steps):
         oracle.verify(t, dd, inp.parent, c, u, w.temperature, w.mode)
@@ -208,7 +220,7 @@ def run_cuda(args):
     dev = torch.device("cuda", torch.cuda.current_device())
     binding.load_library()       # raises if the CUDA library is missing: no fallback
 
-    w = shard_for_rank(pick_workload(args.workload), rank, world)
+    w = shard_for_rank(pick_workload(args.workload, args.batch), rank, world)
     inp = synth.make_inputs(w, dev)
     st = inp.stats
     ver = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[w.dtype], dev)
@@ -284,7 +296,7 @@ def run_cuda(args):
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.no_e2e:
         e2e = run_e2e(args, w, inp, dist, world, dev)
 
     cpu_baseline = None
@@ -376,6 +388,8 @@ def main():
     ap.add_argument("--e2e-batch", type=int, default=128, help="sequences per end-to-end step")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch of the workload (profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
