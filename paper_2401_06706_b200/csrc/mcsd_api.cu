@@ -306,7 +306,8 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     p.slice = cfg.slice;
     p.n_items = static_cast<int32_t>(n_items);
     p.mode = mode;
-    p.scale = static_cast<float>(1.4426950408889634 / static_cast<double>(T));
+    p.scale_d = 1.4426950408889634 / static_cast<double>(T);
+    p.scale = static_cast<float>(p.scale_d);
     std::memcpy(p.child_first, c.plan.child_first, sizeof(p.child_first));
     std::memcpy(p.child_count, c.plan.child_count, sizeof(p.child_count));
 

@@ -43,8 +43,8 @@ constexpr int kMaxCluster = 8;
 constexpr uint32_t kWaitPolls = 1u << 22;
 
 struct __align__(16) NodeStats {
-    float m_t, m_d;  // row maxima of the raw target / draft logits
-    float z_t, z_d;  // sum_x exp((l - m)/T)
+    float r_t, r_d;  // references of the sums: fl(row maximum * scale), log2 units
+    float z_t, z_d;  // sum_x exp2(l * scale - r)
     float c, s;      // final c_n and S_n of the node (0 and 1 for a leaf)
     int32_t pad0, pad1;
 };
@@ -65,6 +65,7 @@ struct NodeParams {
     int32_t n_items; // B * n_nodes
     int32_t mode;
     float scale;     // log2(e) / T
+    double scale_d;  // the same in double, for the candidates' own probabilities
     uint16_t child_first[MCSD_MAX_NODES];
     uint8_t child_count[MCSD_MAX_NODES];
 };
@@ -208,10 +209,10 @@ __device__ __forceinline__ double shfl_d(double v, int src) {
     hi = __shfl_sync(0xffffffffu, hi, src);
     return __hiloint2double(hi, lo);
 }
-// exp2 of a difference with -inf handled: the factor that rescales a partial sum
-// taken relative to maximum m to the reference maximum M (>= m).
-__device__ __forceinline__ float rescale(float m, float M, float scale) {
-    return (m == -INFINITY) ? 0.f : ex2f((m - M) * scale);
+// Factor that moves a partial sum taken relative to reference r (log2 units) to the
+// reference R >= r; an empty partial sum has r = -inf and factor 0.
+__device__ __forceinline__ float rebase(float r, float R) {
+    return (r == -INFINITY) ? 0.f : ex2f(r - R);
 }
 
 // Shared state of the cluster-wide exchange: every CTA owns two slots of one float4
@@ -227,6 +228,42 @@ struct Exchange {
 };
 
 // ------------------------------------------------------------------ node kernel
+// Warp totals of N values per lane in N-1 + (5 - log2 N) shuffles instead of 5 N: each
+// halving step pairs lanes and splits the value indices between them.  On return
+// every lane holds in `out` the warp total of value index `idx` (the return value),
+// idx being fixed by lane bits 4, 3, 2 (N = 8), bits 4, 3 (N = 4) or bit 4 (N = 2).
+template <int HALF>
+__device__ __forceinline__ void halve_step(float *w, int lane, int off, int &idx)
+{
+    const bool hi = (lane & off) != 0;
+#pragma unroll
+    for (int j = 0; j < HALF; ++j) {
+        const float send = hi ? w[j] : w[j + HALF];
+        const float keep = hi ? w[j + HALF] : w[j];
+        w[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+    idx += hi ? HALF : 0;
+}
+template <int N>
+__device__ __forceinline__ int warp_multi_sum(const float (&v)[N], int lane, float &out)
+{
+    static_assert(N == 1 || N == 2 || N == 4 || N == 8, "unsupported count");
+    float w[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) w[j] = v[j];
+    int idx = 0;
+    if constexpr (N >= 2) halve_step<N / 2>(w, lane, 16, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 16);
+    if constexpr (N >= 4) halve_step<N / 4>(w, lane, 8, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 8);
+    if constexpr (N >= 8) halve_step<N / 8>(w, lane, 4, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 4);
+    w[0] += __shfl_xor_sync(0xffffffffu, w[0], 2);
+    w[0] += __shfl_xor_sync(0xffffffffu, w[0], 1);
+    out = w[0];
+    return idx;
+}
+
 // DT: element type; EPT: vocabulary elements per thread per row; DIRECT: read the
 // rows with plain scalar loads (any alignment) instead of bulk copies.
 template <int DT, int EPT, bool DIRECT>
@@ -244,12 +281,12 @@ node_kernel(const __grid_constant__ NodeParams P)
     __shared__ __align__(8) unsigned long long full_bar;
     __shared__ float4 red[kWarps];
     __shared__ float wsum[NVEC * kWarps];
+    __shared__ double s_px[MCSD_MAX_CHILDREN], s_qx[MCSD_MAX_CHILDREN];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t crank = cluster_ctarank(), csize = cluster_nctarank();
     const int cluster_id = blockIdx.x / csize, n_clusters = gridDim.x / csize;
     const float scale = P.scale;
-    const double scale_d = static_cast<double>(P.scale);
 
     const uint32_t full_addr = smem_u32(&full_bar);
     const uint32_t xbar_addr[2] = {smem_u32(&xch.bar[0]), smem_u32(&xch.bar[1])};
@@ -259,6 +296,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     const int v_begin = static_cast<int>(crank) * P.slice;
     int n_mine = P.V - v_begin;
     n_mine = n_mine < 0 ? 0 : (n_mine > P.slice ? P.slice : n_mine);
+    const int n_full_vec = n_mine / VEC;  // vectors that lie wholly inside the slice
     const uint32_t row_bytes = (static_cast<uint32_t>(n_mine) * E::kBytes + 15u) & ~15u;
 
     if (tid == 0) {
@@ -290,8 +328,8 @@ node_kernel(const __grid_constant__ NodeParams P)
         }
     };
 
-    // Cluster-wide exchange of one float4 per CTA.  `mine` must be valid in lanes
-    // 0..csize-1 of warp 0.  Returns false if the bounded wait expired.
+    // Cluster-wide exchange of one float4 per CTA; `mine` must be valid in lanes
+    // 0..csize-1 of warp 0.  Returns the slot holding all CTAs' values.
     auto exchange = [&](float4 mine) -> const float4 * {
         const uint32_t s = round & 1u;
         if (warp == 0 && lane < static_cast<int>(csize)) {
@@ -304,8 +342,38 @@ node_kernel(const __grid_constant__ NodeParams P)
         return xch.slot[s];
     };
 
+    // Candidate data is fetched ahead of use so that no DRAM latency sits on the
+    // per-node critical path: lane i of every warp holds candidate i of the node.
+    //   tokens (token id, acceptance uniform) two nodes ahead,
+    //   the candidate's own two logits one node ahead (they need the token id).
+    auto fetch_tokens = [&](int item, int &xt, float &u) {
+        xt = -1; u = 2.f;
+        if (item < P.n_items) {
+            const int b = item / P.n_nodes, n = item - b * P.n_nodes;
+            const int k = n < P.n_internal ? P.child_count[n] : 0;
+            if (lane < k) {
+                const long long ci = static_cast<long long>(b) * P.n_nodes + P.child_first[n] + lane;
+                xt = __ldg(P.cand + ci);
+                u = __ldg(P.unif + 2 * ci);
+            }
+        }
+    };
+    auto fetch_logits = [&](int item, int xt, float &tl, float &dl) {
+        tl = 0.f; dl = 0.f;
+        if (item < P.n_items && xt >= 0 && xt < P.V) {
+            const int b = item / P.n_nodes, n = item - b * P.n_nodes;
+            tl = E::load(P.target, static_cast<long long>(item) * P.ld_t + xt);
+            dl = E::load(P.draft, (static_cast<long long>(b) * P.n_internal + n) * P.ld_d + xt);
+        }
+    };
+
     int item = cluster_id;
     if (!DIRECT && tid == 0 && item < P.n_items) issue(item);
+    int xt, xt_n1, xt_n2;
+    float u_acc, u_n1, u_n2, tl, dl, tl_n1, dl_n1;
+    fetch_tokens(item, xt, u_acc);
+    fetch_tokens(item + n_clusters, xt_n1, u_n1);
+    fetch_logits(item, xt, tl, dl);
 
     for (; item < P.n_items; item += n_clusters) {
         const int b = item / P.n_nodes, n = item - b * P.n_nodes;
@@ -313,27 +381,10 @@ node_kernel(const __grid_constant__ NodeParams P)
         const int k = internal ? P.child_count[n] : 0;
         const int first = P.child_first[n];
         const long long node_idx = item;  // b * n_nodes + n
-        const unsigned char *t_row = reinterpret_cast<const unsigned char *>(P.target) +
-            node_idx * P.ld_t * E::kBytes;
-        const unsigned char *d_row = reinterpret_cast<const unsigned char *>(P.draft) +
-            (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes;
         int status_bits = 0;
 
-        // ---- candidate data of this node: lane i of every warp holds candidate i
-        int xt = -1;
-        float u_acc = 2.f;
-        double lt_x = 0.0, ld_x = 0.0;  // candidate's own logits, in log2 units
-        bool xt_valid = false;
-        if (lane < k) {
-            const long long ci = static_cast<long long>(b) * P.n_nodes + first + lane;
-            xt = __ldg(P.cand + ci);
-            u_acc = __ldg(P.unif + 2 * ci);
-            xt_valid = xt >= 0 && xt < P.V;
-            if (xt_valid) {
-                lt_x = static_cast<double>(E::load(t_row, xt)) * scale_d;
-                ld_x = static_cast<double>(E::load(d_row, xt)) * scale_d;
-            }
-        }
+        fetch_logits(item + n_clusters, xt_n1, tl_n1, dl_n1);
+        fetch_tokens(item + 2 * n_clusters, xt_n2, u_n2);
         const float u_end = __ldg(P.unif + 2 * node_idx + 1);
 
         // ---- bring the slice into registers: tv = target, dv = draft
@@ -344,21 +395,27 @@ node_kernel(const __grid_constant__ NodeParams P)
 #pragma unroll
             for (int j = 0; j < NVEC; ++j) {
                 const int vec = j * kThreads + tid;
-                const int rem = n_mine - vec * VEC;
                 uint4 raw = *reinterpret_cast<const uint4 *>(stage + vec * 16);
                 E::unpack(raw, &tv[j * VEC]);
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) tv[j * VEC + e] = (e < rem) ? tv[j * VEC + e] : -INFINITY;
                 if (internal) {
                     raw = *reinterpret_cast<const uint4 *>(stage + kRowBytes + vec * 16);
                     E::unpack(raw, &dv[j * VEC]);
+                }
+                if (vec >= n_full_vec) {  // ragged or empty vector: only at the slice end
+                    const int rem = n_mine - vec * VEC;
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) dv[j * VEC + e] = (e < rem) ? dv[j * VEC + e] : -INFINITY;
+                    for (int e = 0; e < VEC; ++e) {
+                        if (e >= rem) { tv[j * VEC + e] = -INFINITY; dv[j * VEC + e] = -INFINITY; }
+                    }
                 }
             }
             __syncthreads();  // stage fully consumed: refill it with the next node of this cluster
             if (tid == 0 && item + n_clusters < P.n_items) issue(item + n_clusters);
         } else {
+            const unsigned char *t_row = reinterpret_cast<const unsigned char *>(P.target) +
+                node_idx * P.ld_t * E::kBytes;
+            const unsigned char *d_row = reinterpret_cast<const unsigned char *>(P.draft) +
+                (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes;
 #pragma unroll
             for (int j = 0; j < NVEC; ++j) {
                 const int base = (j * kThreads + tid) * VEC;
@@ -370,86 +427,99 @@ node_kernel(const __grid_constant__ NodeParams P)
                 }
             }
         }
-        if (!internal) {
-#pragma unroll
-            for (int e = 0; e < EPT; ++e) dv[e] = 0.f;
-        }
 
-        // ---- softmax statistics, one cluster-wide round for both rows.
-        // Each thread exponentiates relative to its own maximum; the factor to the
-        // global maximum and normaliser is applied once afterwards.
+        // ---- softmax statistics, one cluster-wide round for both rows.  Each thread
+        // exponentiates relative to its own maximum (reference r = max * scale, in
+        // log2 units); the factor to the global reference and the normaliser are
+        // applied as per-thread scalars afterwards, never per element.
+        float vs[NVEC];  // per-vector weight sums of this thread, in the thread's own units
         float mt = -INFINITY, md = -INFINITY;
 #pragma unroll
         for (int e = 0; e < EPT; ++e) mt = fmaxf(mt, tv[e]);
-        const float mts = (mt == -INFINITY) ? 0.f : mt;
-        float zt = 0.f, zd = 0.f;
+        // rt / rd: this thread's references (-inf when it holds no finite element)
+        const float rt = (mt == -INFINITY) ? -INFINITY : mt * scale;
+        const float rt0 = (mt == -INFINITY) ? 0.f : rt;
+        float zt = 0.f, zd = 0.f, rd = -INFINITY;
 #pragma unroll
-        for (int e = 0; e < EPT; ++e) { tv[e] = ex2f((tv[e] - mts) * scale); zt += tv[e]; }
+        for (int j = 0; j < NVEC; ++j) {
+            float s = 0.f;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                const float x = ex2f(fmaf(tv[j * VEC + e], scale, -rt0));
+                tv[j * VEC + e] = x;
+                s += x;
+            }
+            vs[j] = s;
+            zt += s;
+        }
         if (internal) {
 #pragma unroll
             for (int e = 0; e < EPT; ++e) md = fmaxf(md, dv[e]);
-            const float mds = (md == -INFINITY) ? 0.f : md;
+            rd = (md == -INFINITY) ? -INFINITY : md * scale;
+            const float rd0 = (md == -INFINITY) ? 0.f : rd;
 #pragma unroll
-            for (int e = 0; e < EPT; ++e) { dv[e] = ex2f((dv[e] - mds) * scale); zd += dv[e]; }
+            for (int e = 0; e < EPT; ++e) {
+                const float x = ex2f(fmaf(dv[e], scale, -rd0));
+                dv[e] = x;
+                zd += x;
+            }
         }
         {
-            const float Mt = warp_max(mt), Md = warp_max(md);
-            const float st = warp_sum(zt * rescale(mt, Mt, scale));
-            const float sd = warp_sum(zd * rescale(md, Md, scale));
-            if (lane == 0) red[warp] = make_float4(Mt, st, Md, sd);
+            const float Rt = warp_max(rt), Rd = warp_max(rd);
+            const float st = warp_sum(zt * rebase(rt, Rt));
+            const float sd = warp_sum(zd * rebase(rd, Rd));
+            if (lane == 0) red[warp] = make_float4(Rt, st, Rd, sd);
         }
         __syncthreads();
         float4 cta = make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
         if (warp == 0) {
             if (lane < kWarps) cta = red[lane];
-            const float Mt = warp_max(cta.x), Md = warp_max(cta.z);
-            cta.y = warp_sum(cta.y * rescale(cta.x, Mt, scale));
-            cta.w = warp_sum(cta.w * rescale(cta.z, Md, scale));
-            cta.x = Mt; cta.z = Md;
+            const float Rt = warp_max(cta.x), Rd = warp_max(cta.z);
+            cta.y = warp_sum(cta.y * rebase(cta.x, Rt));
+            cta.w = warp_sum(cta.w * rebase(cta.z, Rd));
+            cta.x = Rt; cta.z = Rd;
         }
-        float M_t = -INFINITY, M_d = -INFINITY;
-        double Z_t = 0.0, Z_d = 0.0;
-        float cta_mass[kMaxCluster];  // each CTA's share of the current weight total
-        {
-            const float4 *all = exchange(cta);
-            for (uint32_t r = 0; r < csize; ++r) { M_t = fmaxf(M_t, all[r].x); M_d = fmaxf(M_d, all[r].z); }
+        const float4 *slot = exchange(cta);  // per CTA: (ref_t, z_t, ref_d, z_d)
+        float R_t = -INFINITY, R_d = -INFINITY;  // global references: fl(row maximum * scale)
 #pragma unroll
-            for (uint32_t r = 0; r < kMaxCluster; ++r) {
-                cta_mass[r] = 0.f;
-                if (r < csize) {
-                    const float zr = all[r].y * rescale(all[r].x, M_t, scale);
-                    cta_mass[r] = zr;
-                    Z_t += static_cast<double>(zr);
-                    Z_d += static_cast<double>(all[r].w * rescale(all[r].z, M_d, scale));
-                }
+        for (uint32_t r = 0; r < kMaxCluster; ++r)
+            if (r < csize) { R_t = fmaxf(R_t, slot[r].x); R_d = fmaxf(R_d, slot[r].z); }
+        float Z_t = 0.f, Z_d = 0.f;
+#pragma unroll
+        for (uint32_t r = 0; r < kMaxCluster; ++r)
+            if (r < csize) {
+                Z_t += slot[r].y * rebase(slot[r].x, R_t);
+                Z_d += slot[r].w * rebase(slot[r].z, R_d);
             }
-        }
-        const bool t_ok = Z_t > 0.0 && Z_t < INFINITY;           // false for an all -inf or NaN row
-        const bool d_ok = !internal || (Z_d > 0.0 && Z_d < INFINITY);
+        const bool t_ok = Z_t > 0.f && Z_t < INFINITY;            // false for an all -inf or NaN row
+        const bool d_ok = internal && Z_d > 0.f && Z_d < INFINITY;
         if (!t_ok) status_bits |= MCSD_STATUS_NO_MASS;
-        const float inv_zt = t_ok ? static_cast<float>(1.0 / Z_t) : 0.f;
-        const float inv_zd = (internal && d_ok) ? static_cast<float>(1.0 / Z_d) : 0.f;
-        {
-            const float a = rescale(mt, M_t, scale) * inv_zt;
-            const float bq = rescale(md, M_d, scale) * inv_zd;
-#pragma unroll
-            for (int e = 0; e < EPT; ++e) { tv[e] *= a; dv[e] *= bq; }   // tv = p, dv = q
-#pragma unroll
-            for (uint32_t r = 0; r < kMaxCluster; ++r) cta_mass[r] *= inv_zt;
+        // p(x) = tv * a, q(x) = dv * bq for this thread's elements
+        const float a = t_ok ? rebase(rt, R_t) / Z_t : 0.f;
+        const float bq = d_ok ? rebase(rd, R_d) / Z_d : 0.f;
+        const float b_over_a = a > 0.f ? bq / a : 0.f;
+        bool leaf_masses = true;  // slot holds softmax statistics (true) or residual partial sums
+
+        // ---- probabilities of the candidates themselves, once per CTA, in double
+        if (k > 0) {
+            if (warp == 0 && lane < k) {
+                const bool ok = xt >= 0 && xt < P.V;
+                s_px[lane] = (ok && t_ok) ? exp2(static_cast<double>(tl) * P.scale_d - static_cast<double>(R_t)) /
+                                                static_cast<double>(Z_t) : 0.0;
+                s_qx[lane] = (ok && d_ok) ? exp2(static_cast<double>(dl) * P.scale_d - static_cast<double>(R_d)) /
+                                                static_cast<double>(Z_d) : 0.0;
+            }
+            __syncthreads();
         }
 
         // ---- the rejection loop (Algorithm 1 / Algorithm 2), identical in every thread
-        double px = 0.0, qx = 0.0;  // lane i: p(x~_i), q(x~_i) of the original distributions
-        if (lane < k && xt_valid) {
-            px = t_ok ? exp2(lt_x - static_cast<double>(M_t) * scale_d) / Z_t : 0.0;
-            qx = d_ok ? exp2(ld_x - static_cast<double>(M_d) * scale_d) / Z_d : 0.0;
-        }
         double c = 0.0, S = 1.0, W = 1.0;
+        float kappa = 0.f;  // c * bq / a: the residual weight of an element is max(tv - kappa dv, 0) * a
         int accepted = -1;
         for (int i = 0; i < k; ++i) {
             const int xi = __shfl_sync(0xffffffffu, xt, i);
             const float ui = __shfl_sync(0xffffffffu, u_acc, i);
-            const double pxi = shfl_d(px, i), qxi = shfl_d(qx, i);
+            const double pxi = s_px[i], qxi = s_qx[i];
             const bool valid = xi >= 0 && xi < P.V;
             if (!valid) status_bits |= MCSD_STATUS_BAD_TOKEN;
             // Algorithm 2: a token rejected earlier at this node has draft probability 0 now
@@ -458,83 +528,93 @@ node_kernel(const __grid_constant__ NodeParams P)
             const bool zero_q = !valid || dup || !(qxi > 0.0) || !(W > 0.0);
             double Pn = pxi - c * qxi;
             Pn = Pn > 0.0 ? Pn : 0.0;
-            const double rho = zero_q ? -1.0 : (Pn / S) / (qxi / W);
+            // r <= [P_n(x~)/S_n] / [q(x~)/W_n], written without the divisions (all factors > 0)
+            const bool accept = !zero_q && static_cast<double>(ui) * S * qxi <= Pn * W;
             if (P.node_ratio && crank == 0 && tid == 0)
-                P.node_ratio[static_cast<long long>(b) * P.n_nodes + first + i] = static_cast<float>(rho);
-            if (!zero_q && static_cast<double>(ui) <= rho) { accepted = first + i; break; }
+                P.node_ratio[static_cast<long long>(b) * P.n_nodes + first + i] =
+                    zero_q ? -1.f : static_cast<float>((Pn / S) / (qxi / W));
+            if (accept) { accepted = first + i; break; }
             // rejected: p := norm(max(0, p - q)); Algorithm 2 also removes x~ from q
-            const double c_new = (W > 0.0) ? c + S / W : c;
+            double c_try = c;
+            if (W > 0.0) c_try = (P.mode == 1) ? c + S / W : c + S;
             if (P.mode == 1 && !zero_q) { W -= qxi; if (!(W > 0.0)) W = 0.0; }
-            const float cf = static_cast<float>(c_new);
-            float part = 0.f;
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                kappa = static_cast<float>(c_try) * b_over_a;
+                float part = 0.f;
 #pragma unroll
-            for (int e = 0; e < EPT; ++e) part += fmaxf(fmaf(-cf, dv[e], tv[e]), 0.f);
-            part = warp_sum(part);
-            if (lane == 0) red[warp].x = part;
-            __syncthreads();
-            float cta_part = 0.f;
-            if (warp == 0) cta_part = warp_sum(lane < kWarps ? red[lane].x : 0.f);
-            const float4 *all = exchange(make_float4(cta_part, 0.f, 0.f, 0.f));
-            double S_new = 0.0;
-            for (uint32_t r = 0; r < csize; ++r) S_new += static_cast<double>(all[r].x);
-            if (S_new > 0.0) {
-                c = c_new; S = S_new;
+                for (int j = 0; j < NVEC; ++j) {
+                    float s = 0.f;
 #pragma unroll
-                for (uint32_t r = 0; r < kMaxCluster; ++r) cta_mass[r] = (r < csize) ? all[r].x : 0.f;
-            } else {
-                status_bits |= MCSD_STATUS_DEGENERATE;  // residual kept as it was
+                    for (int e = 0; e < VEC; ++e) s += fmaxf(fmaf(-kappa, dv[j * VEC + e], tv[j * VEC + e]), 0.f);
+                    vs[j] = s;
+                    part += s;
+                }
+                part = warp_sum(part * a);
+                if (lane == 0) red[warp].x = part;
+                __syncthreads();
+                float cta_part = 0.f;
+                if (warp == 0) cta_part = warp_sum(lane < kWarps ? red[lane].x : 0.f);
+                slot = exchange(make_float4(cta_part, 0.f, 0.f, 0.f));
+                leaf_masses = false;
+                float S_new = 0.f;
+#pragma unroll
+                for (uint32_t r = 0; r < kMaxCluster; ++r)
+                    if (r < csize) S_new += slot[r].x;
+                if (S_new > 0.f) {
+                    if (attempt == 0) { c = c_try; S = static_cast<double>(S_new); }
+                    break;
+                }
+                // zero residual mass: keep the previous residual (recompute its sums once)
+                status_bits |= MCSD_STATUS_DEGENERATE;
+                c_try = c;
             }
         }
 
         // ---- endpoint token of a node that can end the walk: inverse CDF in token
         // order over w(x) = max(p - c q, 0); only the CTA whose slice holds the
-        // quantile searches, the others go on to their next node.
+        // quantile searches, the others go on to their next node.  vs[] holds this
+        // thread's per-vector sums of w / a.
         int bonus = -1;
         bool bonus_mine = false;
         if (accepted < 0) {
+            const float inv_zt = t_ok ? 1.f / Z_t : 0.f;
             float total = 0.f;
-            for (uint32_t r = 0; r < csize; ++r) total += cta_mass[r];
+#pragma unroll
+            for (uint32_t r = 0; r < kMaxCluster; ++r)
+                if (r < csize)
+                    total += leaf_masses ? slot[r].y * rebase(slot[r].x, R_t) * inv_zt : slot[r].x;
             const float target = u_end * total;
             int owner = -1, last_pos = -1;
-            float cum = 0.f, before = 0.f;
+            float cum = 0.f, before = 0.f, last_before = 0.f;
 #pragma unroll
             for (uint32_t r = 0; r < kMaxCluster; ++r) {
-                if (r < csize && owner < 0 && cta_mass[r] > 0.f) {
-                    last_pos = r;
-                    if (cum + cta_mass[r] > target) { owner = r; before = cum; }
+                if (r < csize) {
+                    const float m = leaf_masses ? slot[r].y * rebase(slot[r].x, R_t) * inv_zt : slot[r].x;
+                    if (m > 0.f) {
+                        last_pos = r; last_before = cum;
+                        if (owner < 0 && cum + m > target) { owner = r; before = cum; }
+                    }
+                    cum += m;
                 }
-                if (r < csize && owner < 0) cum += cta_mass[r];
             }
-            if (owner < 0 && last_pos >= 0) {  // rounding pushed the quantile past the end
-                owner = last_pos;
-                before = 0.f;
-                for (int r = 0; r < last_pos; ++r) before += cta_mass[r];
-            }
+            if (owner < 0) { owner = last_pos; before = last_before; }  // rounding pushed the quantile past the end
             if (owner < 0 || !(total > 0.f)) {
                 status_bits |= MCSD_STATUS_NO_MASS;
                 bonus_mine = crank == 0;
             } else if (owner == static_cast<int>(crank)) {
                 bonus_mine = true;
                 float tgt = target - before;  // quantile inside this CTA's slice
-                const float cf = static_cast<float>(c);
-                float vs[NVEC];
+                float wv[NVEC];
 #pragma unroll
-                for (int j = 0; j < NVEC; ++j) {
-                    float s = 0.f;
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) s += fmaxf(fmaf(-cf, dv[j * VEC + e], tv[j * VEC + e]), 0.f);
-                    vs[j] = s;
-                }
-#pragma unroll
-                for (int j = 0; j < NVEC; ++j) {
-                    const float w = warp_sum(vs[j]);
-                    if (lane == 0) wsum[j * kWarps + warp] = w;
-                }
+                for (int j = 0; j < NVEC; ++j) wv[j] = vs[j] * a;
+                float wtot;
+                const int wj = warp_multi_sum<NVEC>(wv, lane, wtot);
+                if ((lane & 3) == 0) wsum[wj * kWarps + warp] = wtot;  // lanes sharing an index write the same total
                 __syncthreads();
                 // level 1: (chunk j, warp) in token order
                 constexpr int kEntries = NVEC * kWarps;
                 int pick = -1, last_e = -1;
-                float run = 0.f, pick_before = 0.f, last_before = 0.f;
+                float run = 0.f, pick_before = 0.f, last_b = 0.f;
 #pragma unroll
                 for (int base = 0; base < kEntries; base += 32) {
                     const int idx = base + lane;
@@ -550,24 +630,24 @@ node_kernel(const __grid_constant__ NodeParams P)
                     if (pos) {
                         const int l = 31 - __clz(pos);
                         last_e = base + l;
-                        last_before = __shfl_sync(0xffffffffu, inc, l) - __shfl_sync(0xffffffffu, w, l);
+                        last_b = __shfl_sync(0xffffffffu, inc, l) - __shfl_sync(0xffffffffu, w, l);
                     }
                     run = __shfl_sync(0xffffffffu, inc, 31);
                 }
-                if (pick < 0) { pick = last_e; pick_before = last_before; }  // clamp to the last entry with mass
+                if (pick < 0) { pick = last_e; pick_before = last_b; }  // clamp to the last entry with mass
                 if (pick >= 0) {
                     const int pj = pick / kWarps, pw = pick - pj * kWarps;
                     if (warp == pw) {
                         tgt -= pick_before;
-                        float v = vs[0];
+                        float v = wv[0];
 #pragma unroll
-                        for (int j = 1; j < NVEC; ++j) v = (pj == j) ? vs[j] : v;
+                        for (int j = 1; j < NVEC; ++j) v = (pj == j) ? wv[j] : v;
                         const float inc = warp_scan_incl(v, lane);
-                        unsigned hit = __ballot_sync(0xffffffffu, v > 0.f && inc > tgt);
+                        const unsigned hit = __ballot_sync(0xffffffffu, v > 0.f && inc > tgt);
                         const unsigned pos = __ballot_sync(0xffffffffu, v > 0.f);
-                        int l = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
+                        const int l = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
                         if (l >= 0 && lane == l) {
-                            float rem = tgt - (inc - v);
+                            const float rem = tgt - (inc - v);
                             float acc = 0.f;
                             int pe = -1, last = -1;
 #pragma unroll
@@ -575,7 +655,8 @@ node_kernel(const __grid_constant__ NodeParams P)
                                 if (j == pj) {
 #pragma unroll
                                     for (int e = 0; e < VEC; ++e) {
-                                        const float w = fmaxf(fmaf(-cf, dv[j * VEC + e], tv[j * VEC + e]), 0.f);
+                                        const float w = (internal ? fmaxf(fmaf(-kappa, dv[j * VEC + e], tv[j * VEC + e]), 0.f)
+                                                                  : tv[j * VEC + e]) * a;
                                         if (w > 0.f) {
                                             acc += w;
                                             last = e;
@@ -602,8 +683,8 @@ node_kernel(const __grid_constant__ NodeParams P)
             if (accepted >= 0 || (bonus_mine && bonus < 0 && (status_bits & MCSD_STATUS_NO_MASS)))
                 P.node_bonus[node_idx] = -1;
             NodeStats st;
-            st.m_t = M_t; st.m_d = M_d;
-            st.z_t = static_cast<float>(Z_t); st.z_d = static_cast<float>(Z_d);
+            st.r_t = R_t; st.r_d = R_d;
+            st.z_t = Z_t; st.z_d = Z_d;
             st.c = static_cast<float>(c); st.s = static_cast<float>(S);
             st.pad0 = 0; st.pad1 = 0;
             P.stats[node_idx] = st;
@@ -611,6 +692,10 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
         status_bits = __reduce_or_sync(0xffffffffu, status_bits);
         if (status_bits && lane == 0) atomicOr(P.status + b, status_bits);
+
+        // rotate the candidate pipeline
+        xt = xt_n1; u_acc = u_n1; tl = tl_n1; dl = dl_n1;
+        xt_n1 = xt_n2; u_n1 = u_n2;
     }
 
     // no CTA may leave while a peer can still write into its shared memory
@@ -782,6 +867,8 @@ walk_kernel(const __grid_constant__ WalkParams P)
         (nb + n) * P.ld_t * E::kBytes;
     const unsigned char *d_row = reinterpret_cast<const unsigned char *>(P.draft) +
         (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes;
+    const float r_t = st.r_t == -INFINITY ? 0.f : st.r_t;
+    const float r_d = st.r_d == -INFINITY ? 0.f : st.r_d;
     const float inv_zt = st.z_t > 0.f ? 1.f / st.z_t : 0.f;
     const float cq = (internal && st.z_d > 0.f) ? st.c / st.z_d : 0.f;
     const float inv_s = st.s > 0.f ? 1.f / st.s : 0.f;
@@ -789,8 +876,8 @@ walk_kernel(const __grid_constant__ WalkParams P)
     for (int e = 0; e < 4; ++e) {
         const int x = x0 + e;
         if (x < P.V) {
-            float w = ex2f((E::load(t_row, x) - st.m_t) * P.scale) * inv_zt;
-            if (internal && cq > 0.f) w = fmaxf(fmaf(-cq, ex2f((E::load(d_row, x) - st.m_d) * P.scale), w), 0.f);
+            float w = ex2f(fmaf(E::load(t_row, x), P.scale, -r_t)) * inv_zt;
+            if (internal && cq > 0.f) w = fmaxf(fmaf(-cq, ex2f(fmaf(E::load(d_row, x), P.scale, -r_d)), w), 0.f);
             out[x] = w * inv_s;
         }
     }
