@@ -109,15 +109,15 @@ bool rows_aligned16(const void *base, long long ld, int dtype)
 
 // ---- node-kernel variants ---------------------------------------------------
 using NodeKernel = void (*)(const NodeParams);
-constexpr int kEptChoices[3] = {8, 16, 32};
+constexpr int kEptChoices[3] = {16, 32, 64};
 
 template <int DT, bool DIRECT>
 NodeKernel pick_ept(int ept)
 {
     switch (ept) {
-    case 8: return node_kernel<DT, 8, DIRECT>;
     case 16: return node_kernel<DT, 16, DIRECT>;
-    default: return node_kernel<DT, 32, DIRECT>;
+    case 32: return node_kernel<DT, 32, DIRECT>;
+    default: return node_kernel<DT, 64, DIRECT>;
     }
 }
 NodeKernel pick_node_kernel(int dtype, int ept, bool direct)
@@ -155,7 +155,7 @@ int choose_config(int vocab, int dtype, bool aligned, NodeConfig *cfg)
             const int e = kEptChoices[ei];
             if (force_e && e != force_e) continue;
             const long long slice = align_up((vocab + c - 1) / c, vec);
-            if (slice > static_cast<long long>(kThreads) * e) continue;
+            if (slice > static_cast<long long>(kNodeThreads) * e) continue;
             const long long cap = static_cast<long long>(c) * e;
             if (best_cap < 0 || cap < best_cap) { best_cap = cap; best_c = c; best_e = e; }
         }
@@ -184,14 +184,25 @@ int resident_clusters(NodeKernel fn, int cluster, size_t smem, cudaStream_t stre
     }
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return -1;
-    // ask for the largest shared-memory carveout so that as many CTAs as the register
-    // budget allows can hold their staging buffers at once
-    cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    int n_sm = 0;
+    // shared-memory carveout: what the CTAs the register budget admits need (dynamic +
+    // static + 1 KB the system reserves per CTA), the rest stays L1
+    int n_sm = 0, smem_sm = 0;
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+    cudaFuncAttributes fa = {};
+    if (cudaFuncGetAttributes(&fa, fn) == cudaSuccess && smem_sm > 0 && fa.numRegs > 0) {
+        int by_regs = 65536 / (fa.numRegs * kNodeThreads);
+        if (by_regs < 1) by_regs = 1;
+        const size_t per_cta = smem + fa.sharedSizeBytes + 1024;
+        size_t want = per_cta * static_cast<size_t>(by_regs);
+        if (want > static_cast<size_t>(smem_sm)) want = static_cast<size_t>(smem_sm);
+        int pct = static_cast<int>((want * 100 + smem_sm - 1) / smem_sm);
+        if (pct > 100) pct = 100;
+        cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, pct);
+    }
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(static_cast<unsigned>(cluster * n_sm * 4));
-    lc.blockDim = dim3(kThreads);
+    lc.gridDim = dim3(static_cast<unsigned>(cluster * n_sm * 8));
+    lc.blockDim = dim3(kNodeThreads);
     lc.dynamicSmemBytes = smem;
     lc.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -292,7 +303,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     int rc = choose_config(d->vocab, d->dtype, aligned, &cfg);
     if (rc != MCSD_OK) return rc;
     NodeKernel fn = pick_node_kernel(d->dtype, cfg.ept, cfg.direct);
-    const size_t smem = cfg.direct ? 0 : static_cast<size_t>(2) * kThreads * cfg.ept * elem_bytes(d->dtype);
+    const size_t smem = node_smem_bytes(elem_bytes(d->dtype), cfg.ept, cfg.direct);
     const int resident = resident_clusters(fn, cfg.cluster, smem, c.stream);
     if (resident < 1) return MCSD_ERR_CUDA;
     const long long n_clusters = n_items < resident ? n_items : resident;
@@ -313,7 +324,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
 
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(static_cast<unsigned>(n_clusters * cfg.cluster));
-    lc.blockDim = dim3(kThreads);
+    lc.blockDim = dim3(kNodeThreads);
     lc.dynamicSmemBytes = smem;
     lc.stream = c.stream;
     cudaLaunchAttribute attr[1];

@@ -1,14 +1,16 @@
 // Device code of the MCSD verification library (sm_100a).
 //
 // Three kernels:
-//   node_kernel      T > 0.  One thread-block cluster per tree node.  Each CTA of the
-//                    cluster owns a contiguous slice of the vocabulary, brings its
-//                    slice of the target row (and of the draft row for a node that
-//                    has children) into shared memory with one bulk async copy (TMA,
-//                    no multicast), moves it into registers, and from then on the two
-//                    distributions stay in registers while the k candidates of the
-//                    node are tested in order (Algorithm 1 / Algorithm 2).  Each logit
-//                    row is read from HBM exactly once.
+//   node_kernel      T > 0.  One thread-block cluster per tree node, persistent over the
+//                    (sequence, node) items.  Each CTA of the cluster owns a contiguous
+//                    slice of the vocabulary.  Its slice of the target row goes straight
+//                    into registers with coalesced 128-bit loads; its slice of the draft
+//                    row (nodes that have children) is brought into shared memory with
+//                    one bulk async copy (TMA, no multicast) and stays there.  Both are
+//                    exponentiated once and then stay on chip while the k candidates of
+//                    the node are tested in order (Algorithm 1 / Algorithm 2), so every
+//                    logit row is read from HBM exactly once.  The rows of the cluster's
+//                    next item are prefetched into L2 while the current one is computed.
 //   argmax_kernel    T == 0.  One CTA per target row; argmax with lowest index on ties
 //                    and the "candidate equals argmax" test (Section 4.4).
 //   walk_kernel      One row of CTAs per sequence: follows the accepted children from
@@ -22,8 +24,13 @@
 // Algorithm 2 (p and q are the ORIGINAL softmax outputs).  This follows from
 // p_{n+1} ~ max(p_n - q_n, 0) by induction and holds for every rejection that can
 // occur with r in (0,1).  The test of candidate n+1 is r <= [P_n(x~)/S_n]/[q(x~)/W_n].
-// So one rejection costs one scalar-parameter reduction over the register-resident
-// p and q, and nothing is written back.
+// So one rejection costs one scalar-parameter reduction over the on-chip p and q,
+// and nothing is written back.  c_1 = 1 whatever the candidates are, so the first
+// reduction is started before the first test has been decided.
+//
+// Softmax references are integers (ceil of the scaled row maximum, in log2 units), so
+// moving a partial sum from one reference to another is an exact multiplication by a
+// power of two and every thread can exponentiate against its own maximum.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -38,12 +45,12 @@ namespace mcsd {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxCluster = 8;
-// Polls of a bounded wait before it gives up (each poll can itself block for a
-// hardware-defined time slice, so this is seconds, far beyond any legitimate wait).
-constexpr uint32_t kWaitPolls = 1u << 22;
+// Polls of a bounded wait before it gives up; with the back-off between polls the
+// bound is about two seconds, far beyond any legitimate wait.
+constexpr uint32_t kWaitPolls = 1u << 21;
 
 struct __align__(16) NodeStats {
-    float r_t, r_d;  // references of the sums: fl(row maximum * scale), log2 units
+    float r_t, r_d;  // references of the sums: ceil(row maximum * scale), log2 units
     float z_t, z_d;  // sum_x exp2(l * scale - r)
     float c, s;      // final c_n and S_n of the node (0 and 1 for a leaf)
     int32_t pad0, pad1;
@@ -81,6 +88,8 @@ template <> struct Elem<MCSD_DTYPE_F32> {
     static __device__ __forceinline__ float load(const void *base, long long i) {
         return __ldg(reinterpret_cast<const float *>(base) + i);
     }
+    // value of element i given the aligned 32-bit word that contains it
+    static __device__ __forceinline__ float from_word(uint32_t w, long long) { return __uint_as_float(w); }
 };
 template <> struct Elem<MCSD_DTYPE_BF16> {
     static constexpr int kBytes = 2, kVec = 8;
@@ -93,6 +102,9 @@ template <> struct Elem<MCSD_DTYPE_BF16> {
     static __device__ __forceinline__ float load(const void *base, long long i) {
         unsigned short h = __ldg(reinterpret_cast<const unsigned short *>(base) + i);
         return __uint_as_float(static_cast<uint32_t>(h) << 16);
+    }
+    static __device__ __forceinline__ float from_word(uint32_t w, long long i) {
+        return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));
     }
 };
 template <> struct Elem<MCSD_DTYPE_F16> {
@@ -107,6 +119,10 @@ template <> struct Elem<MCSD_DTYPE_F16> {
     }
     static __device__ __forceinline__ float load(const void *base, long long i) {
         return __half2float(__ldg(reinterpret_cast<const __half *>(base) + i));
+    }
+    static __device__ __forceinline__ float from_word(uint32_t w, long long i) {
+        const unsigned short h = static_cast<unsigned short>((i & 1) ? (w >> 16) : (w & 0xffffu));
+        return __half2float(__ushort_as_half(h));
     }
 };
 
@@ -124,6 +140,12 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
 }
 __device__ __forceinline__ uint32_t cluster_nctarank() {
     uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void cluster_arrive_release() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -146,24 +168,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded waits: false when the poll budget ran out.
+// Bounded wait with back-off (a waiting thread must not eat the issue slots of the
+// working ones): false when the poll budget ran out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitPolls; ++i)
+    for (uint32_t i = 0; i < kWaitPolls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitPolls; ++i)
-        if (mbar_try_wait_cluster(bar, parity)) return true;
+        __nanosleep(i < 64 ? 64 : 1000);
+    }
     return false;
 }
 // One bulk async copy global -> this CTA's shared memory (TMA, no multicast);
@@ -171,6 +182,29 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Asks L2 to fetch a 16-byte-aligned range (size a multiple of 16); nothing waits on it.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+// 4-byte asynchronous copy global -> shared (no register holds the value in flight).
+// Orders this thread's earlier ordinary shared-memory accesses before later bulk
+// (async-proxy) copies into the same locations.
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void cp_async4(void *smem_dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+// 128-bit streaming load (read once, do not keep in L1).
+__device__ __forceinline__ uint4 ld_stream_v4(const void *p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
 }
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     uint32_t r;
@@ -180,9 +214,6 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void st_cluster_f4(uint32_t addr, float4 v) {
     asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
                  ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
 }
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -203,35 +234,53 @@ __device__ __forceinline__ float warp_scan_incl(float v, int lane) {
     }
     return v;
 }
-__device__ __forceinline__ double shfl_d(double v, int src) {
-    int lo = __double2loint(v), hi = __double2hiint(v);
-    lo = __shfl_sync(0xffffffffu, lo, src);
-    hi = __shfl_sync(0xffffffffu, hi, src);
-    return __hiloint2double(hi, lo);
+// 2^d for an integer-valued d (a difference of two references): exact; 0 when
+// d < -126 (also for d = -inf), clamped to 2^127 above.
+__device__ __forceinline__ float exp2i(float d) {
+    d = fminf(fmaxf(d, -127.f), 127.f);
+    return __int_as_float((static_cast<int>(d) + 127) << 23);
 }
-// Factor that moves a partial sum taken relative to reference r (log2 units) to the
-// reference R >= r; an empty partial sum has r = -inf and factor 0.
-__device__ __forceinline__ float rebase(float r, float R) {
-    return (r == -INFINITY) ? 0.f : ex2f(r - R);
+// The same in double for an integer e: 0 below 2^-1000.
+__device__ __forceinline__ double exp2i_d(int e) {
+    if (e < -1000) return 0.0;
+    e = e > 1000 ? 1000 : e;
+    return __hiloint2double((e + 1023) << 20, 0);
+}
+// Integer reference of a set whose largest scaled logit is m (log2 units); -inf for
+// an empty set.  NaN-free inputs give ceil(m), so that every exponent is <= 0.
+__device__ __forceinline__ float int_ref(float m_scaled) {
+    return (m_scaled == -INFINITY) ? -INFINITY : ceilf(m_scaled);
 }
 
-// Shared state of the cluster-wide exchange: every CTA owns two slots of one float4
-// per cluster rank and one mbarrier per slot.  In round r every CTA stores its value
-// into slot r&1 of every CTA (its own included) and arrives on that CTA's barrier;
-// a CTA that has seen `cluster size` arrivals holds all values of the round.  A slot
-// is rewritten two rounds later, which a peer can only reach after this CTA has
-// arrived for the round in between, i.e. after it finished reading (release/acquire
-// at cluster scope orders the accesses).
+// Shared state of the cluster-wide exchange: two buffers of one float4 per (cluster
+// rank, warp).  In round r every warp of every CTA stores its value into buffer r&1 of
+// every CTA of the cluster (its own included) and then all threads meet at the
+// hardware cluster barrier; after it every CTA holds all values of the round, in
+// vocabulary order (rank-major, then warp).  A buffer is rewritten two rounds later,
+// which a peer can only reach after this CTA's threads have arrived at the barrier in
+// between, i.e. after they finished reading (release/acquire at cluster scope).
 struct Exchange {
-    float4 slot[2][kMaxCluster];
-    unsigned long long bar[2];
+    float4 slot[2][kMaxCluster * 4];
+};
+
+// Candidate data of the next items, fetched ahead of use by warp 0 so that no DRAM
+// latency sits on the per-node critical path: lane i handles candidate i.
+//   token id and acceptance uniform   two items ahead  (ring of 3)
+//   the candidate's own two logits    one item ahead   (ring of 2; they need the token)
+//   the uniform of the endpoint draw  one item ahead   (ring of 2)
+struct CandRing {
+    int32_t tok[3][MCSD_MAX_CHILDREN];
+    float u[3][MCSD_MAX_CHILDREN];
+    uint32_t tl[2][MCSD_MAX_CHILDREN];  // aligned 32-bit word holding the target logit
+    uint32_t dl[2][MCSD_MAX_CHILDREN];  // same for the draft logit
+    float u_end[2];
 };
 
 // ------------------------------------------------------------------ node kernel
 // Warp totals of N values per lane in N-1 + (5 - log2 N) shuffles instead of 5 N: each
 // halving step pairs lanes and splits the value indices between them.  On return
 // every lane holds in `out` the warp total of value index `idx` (the return value),
-// idx being fixed by lane bits 4, 3, 2 (N = 8), bits 4, 3 (N = 4) or bit 4 (N = 2).
+// idx = lane / (32 / N).
 template <int HALF>
 __device__ __forceinline__ void halve_step(float *w, int lane, int off, int &idx)
 {
@@ -247,7 +296,7 @@ __device__ __forceinline__ void halve_step(float *w, int lane, int off, int &idx
 template <int N>
 __device__ __forceinline__ int warp_multi_sum(const float (&v)[N], int lane, float &out)
 {
-    static_assert(N == 1 || N == 2 || N == 4 || N == 8, "unsupported count");
+    static_assert(N == 1 || N == 2 || N == 4 || N == 8 || N == 16, "unsupported count");
     float w[N];
 #pragma unroll
     for (int j = 0; j < N; ++j) w[j] = v[j];
@@ -258,308 +307,397 @@ __device__ __forceinline__ int warp_multi_sum(const float (&v)[N], int lane, flo
     else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 8);
     if constexpr (N >= 8) halve_step<N / 8>(w, lane, 4, idx);
     else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 4);
-    w[0] += __shfl_xor_sync(0xffffffffu, w[0], 2);
+    if constexpr (N >= 16) halve_step<N / 16>(w, lane, 2, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 2);
     w[0] += __shfl_xor_sync(0xffffffffu, w[0], 1);
     out = w[0];
     return idx;
 }
 
+// Threads of one node-kernel CTA.  Few threads with many elements each: the per-thread
+// bookkeeping (about 60 registers) is paid once per 64 elements, so that four CTAs
+// with a 64-element target slice per thread fit the register file without spilling.
+constexpr int kNodeThreads = 128;
+constexpr int kNodeWarps = kNodeThreads / 32;
+// Resident CTAs per SM the register budget is held to (128 / 96 / 80 registers).
+constexpr int node_min_blocks(int ept) { return ept >= 64 ? 4 : (ept >= 32 ? 5 : 6); }
+// Dynamic shared memory of one CTA: the exponentiated draft slice (float) and, for
+// 2-byte logits on the bulk-copy path, the zone the raw draft slice lands in.
+constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
+    return static_cast<size_t>(kNodeThreads) * ept * 4 +
+           ((!direct && elem_bytes == 2) ? static_cast<size_t>(kNodeThreads) * ept * 2 : 0);
+}
+
 // DT: element type; EPT: vocabulary elements per thread per row; DIRECT: read the
-// rows with plain scalar loads (any alignment) instead of bulk copies.
+// rows with plain scalar loads (any alignment) instead of vector loads and bulk copies.
+//
+// Ownership inside a CTA: the slice is cut into 16-byte groups of GV elements; thread
+// (warp w, lane l) owns groups (w * NG + j) * 32 + l, j < NG, so that one warp-wide
+// access is contiguous and a warp's elements are one contiguous run of the vocabulary.
+//
+// Every decision of the rejection loop is taken by every warp of the cluster from
+// bit-identical inputs, so all CTAs of a cluster execute the same number of exchange
+// rounds (the cluster barrier counts on it).
 template <int DT, int EPT, bool DIRECT>
-__global__ void __launch_bounds__(kThreads, (EPT >= 32 ? 2 : (EPT >= 16 ? 3 : 4)))
+__global__ void __launch_bounds__(kNodeThreads, node_min_blocks(EPT))
 node_kernel(const __grid_constant__ NodeParams P)
 {
     using E = Elem<DT>;
-    constexpr int VEC = E::kVec;
-    constexpr int NVEC = EPT / VEC;
-    constexpr int kRowBytes = kThreads * EPT * E::kBytes;
-    static_assert(EPT % VEC == 0, "EPT must be a whole number of 16-byte vectors");
+    constexpr int NT = kNodeThreads, NW = kNodeWarps;
+    constexpr int GV = E::kVec;
+    constexpr int NG = EPT / GV;
+    constexpr int H = GV / 4;  // float4 per group once exponentiated
+    constexpr bool kRawZone = !DIRECT && E::kBytes == 2;
+    static_assert(EPT % GV == 0, "EPT must be a whole number of 16-byte groups");
+    static_assert(NW == 4, "the exchange buffers hold four warps per CTA");
 
-    extern __shared__ __align__(128) unsigned char stage[];  // [2][kRowBytes]: target slice, draft slice
+    extern __shared__ __align__(128) unsigned char dyn[];
+    float4 *qbuf = reinterpret_cast<float4 *>(dyn);  // exponentiated draft slice, thread-private slots
+    const uint4 *qraw = reinterpret_cast<const uint4 *>(dyn + static_cast<size_t>(NT) * EPT * 4);
     __shared__ Exchange xch;
     __shared__ __align__(8) unsigned long long full_bar;
-    __shared__ float4 red[kWarps];
-    __shared__ float wsum[NVEC * kWarps];
-    __shared__ double s_px[MCSD_MAX_CHILDREN], s_qx[MCSD_MAX_CHILDREN];
+    __shared__ double s_px[NW][MCSD_MAX_CHILDREN], s_qx[NW][MCSD_MAX_CHILDREN];
+    __shared__ CandRing ring;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t crank = cluster_ctarank(), csize = cluster_nctarank();
     const int cluster_id = blockIdx.x / csize, n_clusters = gridDim.x / csize;
+    const int n_entries = static_cast<int>(csize) * NW;  // values per exchange round (<= 32)
     const float scale = P.scale;
-
     const uint32_t full_addr = smem_u32(&full_bar);
-    const uint32_t xbar_addr[2] = {smem_u32(&xch.bar[0]), smem_u32(&xch.bar[1])};
-    const uint32_t stage_addr = smem_u32(stage);
 
     // this CTA's slice of the vocabulary
     const int v_begin = static_cast<int>(crank) * P.slice;
     int n_mine = P.V - v_begin;
     n_mine = n_mine < 0 ? 0 : (n_mine > P.slice ? P.slice : n_mine);
-    const int n_full_vec = n_mine / VEC;  // vectors that lie wholly inside the slice
-    const uint32_t row_bytes = (static_cast<uint32_t>(n_mine) * E::kBytes + 15u) & ~15u;
+    // bytes of the slice that are whole 16-byte groups: what one bulk copy / prefetch moves
+    const uint32_t bulk_bytes = DIRECT ? 0u : static_cast<uint32_t>(n_mine / GV) * 16u;
+
+    // slot of (group j, quarter h) in qbuf: for 4-byte logits it is the group's own place in
+    // the slice, so that the bulk copy lands the raw values where the exponentiated ones go
+    auto qslot = [&](int j, int h) -> int {
+        return E::kBytes == 4 ? (warp * NG + j) * 32 + lane : (j * H + h) * NT + tid;
+    };
+    auto group_of = [&](int j) -> int { return (warp * NG + j) * 32 + lane; };
 
     if (tid == 0) {
         mbar_init(full_addr, 1);
-        mbar_init(xbar_addr[0], csize);
-        mbar_init(xbar_addr[1], csize);
         fence_mbar_init();
     }
     __syncthreads();
-    cluster_sync_all();  // every CTA's barriers exist before anyone arrives remotely
+    cluster_sync_all();  // every CTA of the cluster is running before anyone stores into a peer
 
     uint32_t full_parity = 0, round = 0;
     int poisoned = 0;
 
-    auto issue = [&](int item) {
-        const int b = item / P.n_nodes, n = item - b * P.n_nodes;
-        const bool internal = n < P.n_internal;
-        const uint32_t total = row_bytes * (internal ? 2u : 1u);
-        mbar_arrive_expect_tx(full_addr, total);
-        if (row_bytes) {
-            const unsigned char *t = reinterpret_cast<const unsigned char *>(P.target) +
-                (static_cast<long long>(item) * P.ld_t + v_begin) * E::kBytes;
-            bulk_load(stage_addr, t, row_bytes, full_addr);
-            if (internal) {
-                const unsigned char *d = reinterpret_cast<const unsigned char *>(P.draft) +
-                    ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + v_begin) * E::kBytes;
-                bulk_load(stage_addr + kRowBytes, d, row_bytes, full_addr);
-            }
-        }
+    auto t_slice = [&](int item) -> const unsigned char * {
+        return reinterpret_cast<const unsigned char *>(P.target) +
+            (static_cast<long long>(item) * P.ld_t + v_begin) * E::kBytes;
+    };
+    auto d_slice = [&](int b, int n) -> const unsigned char * {
+        return reinterpret_cast<const unsigned char *>(P.draft) +
+            ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + v_begin) * E::kBytes;
     };
 
-    // Cluster-wide exchange of one float4 per CTA; `mine` must be valid in lanes
-    // 0..csize-1 of warp 0.  Returns the slot holding all CTAs' values.
-    auto exchange = [&](float4 mine) -> const float4 * {
-        const uint32_t s = round & 1u;
-        if (warp == 0 && lane < static_cast<int>(csize)) {
-            const uint32_t dst = map_to_rank(smem_u32(&xch.slot[s][crank]), lane);
+    // One exchange round.  send: `mine` is this warp's value (the same in all lanes); the
+    // threads then arrive at the cluster barrier, and whatever is placed between send and
+    // wait overlaps the barrier's latency.  wait: returns entry `lane` of the round
+    // (rank-major, then warp), the given identity for lanes beyond the entry count.
+    auto exchange_send = [&](float4 mine) {
+        if (lane < static_cast<int>(csize)) {
+            const uint32_t dst = map_to_rank(smem_u32(&xch.slot[round & 1u][crank * NW + warp]), lane);
             st_cluster_f4(dst, mine);
-            mbar_arrive_remote(map_to_rank(xbar_addr[s], lane));
         }
-        if (!mbar_wait_cluster(xbar_addr[s], (round >> 1) & 1u)) poisoned = 1;
+        cluster_arrive_release();
+    };
+    auto exchange_wait = [&](float4 identity) -> float4 {
+        cluster_wait_acquire();
+        const float4 e = lane < n_entries ? xch.slot[round & 1u][lane] : identity;
         ++round;
-        return xch.slot[s];
+        return e;
     };
 
-    // Candidate data is fetched ahead of use so that no DRAM latency sits on the
-    // per-node critical path: lane i of every warp holds candidate i of the node.
-    //   tokens (token id, acceptance uniform) two nodes ahead,
-    //   the candidate's own two logits one node ahead (they need the token id).
-    auto fetch_tokens = [&](int item, int &xt, float &u) {
-        xt = -1; u = 2.f;
+    // ---- candidate pipeline (warp 0 only) -------------------------------------------
+    auto fetch_tokens = [&](int item, int slot3) {
         if (item < P.n_items) {
             const int b = item / P.n_nodes, n = item - b * P.n_nodes;
             const int k = n < P.n_internal ? P.child_count[n] : 0;
             if (lane < k) {
                 const long long ci = static_cast<long long>(b) * P.n_nodes + P.child_first[n] + lane;
-                xt = __ldg(P.cand + ci);
-                u = __ldg(P.unif + 2 * ci);
+                cp_async4(&ring.tok[slot3][lane], P.cand + ci);
+                cp_async4(&ring.u[slot3][lane], P.unif + 2 * ci);
             }
         }
     };
-    auto fetch_logits = [&](int item, int xt, float &tl, float &dl) {
-        tl = 0.f; dl = 0.f;
-        if (item < P.n_items && xt >= 0 && xt < P.V) {
+    auto fetch_u_end = [&](int item, int slot2) {
+        if (item < P.n_items && lane == 0) cp_async4(&ring.u_end[slot2], P.unif + 2 * static_cast<long long>(item) + 1);
+    };
+    // needs the item's tokens to have arrived (cp_async_wait_all by this thread)
+    auto fetch_logits = [&](int item, int slot3, int slot2) {
+        if (item < P.n_items) {
             const int b = item / P.n_nodes, n = item - b * P.n_nodes;
-            tl = E::load(P.target, static_cast<long long>(item) * P.ld_t + xt);
-            dl = E::load(P.draft, (static_cast<long long>(b) * P.n_internal + n) * P.ld_d + xt);
+            const int k = n < P.n_internal ? P.child_count[n] : 0;
+            if (lane < k) {
+                const int xt = ring.tok[slot3][lane];
+                if (xt >= 0 && xt < P.V) {
+                    const unsigned char *t = reinterpret_cast<const unsigned char *>(P.target) +
+                        (static_cast<long long>(item) * P.ld_t + xt) * E::kBytes;
+                    const unsigned char *d = reinterpret_cast<const unsigned char *>(P.draft) +
+                        ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + xt) * E::kBytes;
+                    if (!DIRECT) {  // rows are 16-byte aligned: the enclosing word lies inside the row
+                        cp_async4(&ring.tl[slot2][lane], reinterpret_cast<const void *>(reinterpret_cast<uintptr_t>(t) & ~uintptr_t(3)));
+                        cp_async4(&ring.dl[slot2][lane], reinterpret_cast<const void *>(reinterpret_cast<uintptr_t>(d) & ~uintptr_t(3)));
+                    } else {        // any alignment: plain loads of exactly the element, kept as float
+                        ring.tl[slot2][lane] = __float_as_uint(E::load(t, 0));
+                        ring.dl[slot2][lane] = __float_as_uint(E::load(d, 0));
+                    }
+                }
+            }
         }
     };
 
     int item = cluster_id;
-    if (!DIRECT && tid == 0 && item < P.n_items) issue(item);
-    int xt, xt_n1, xt_n2;
-    float u_acc, u_n1, u_n2, tl, dl, tl_n1, dl_n1;
-    fetch_tokens(item, xt, u_acc);
-    fetch_tokens(item + n_clusters, xt_n1, u_n1);
-    fetch_logits(item, xt, tl, dl);
+    uint32_t it = 0;  // iteration count of this cluster
+    if (warp == 0) {
+        fetch_tokens(item, 0);
+        fetch_u_end(item, 0);
+        cp_async_wait_all();
+        __syncwarp();
+        fetch_logits(item, 0, 0);
+        fetch_tokens(item + n_clusters, 1);
+    }
+    if (!DIRECT && tid == 0 && item < P.n_items && bulk_bytes) {
+        const int b = item / P.n_nodes, n = item - b * P.n_nodes;
+        bulk_prefetch_l2(t_slice(item), bulk_bytes);
+        if (n < P.n_internal) bulk_prefetch_l2(d_slice(b, n), bulk_bytes);
+    }
 
-    for (; item < P.n_items; item += n_clusters) {
+    for (; item < P.n_items; item += n_clusters, ++it) {
         const int b = item / P.n_nodes, n = item - b * P.n_nodes;
         const bool internal = n < P.n_internal;
         const int k = internal ? P.child_count[n] : 0;
         const int first = P.child_first[n];
         const long long node_idx = item;  // b * n_nodes + n
+        const int s3 = it % 3u, s2 = it & 1u;
         int status_bits = 0;
 
-        fetch_logits(item + n_clusters, xt_n1, tl_n1, dl_n1);
-        fetch_tokens(item + 2 * n_clusters, xt_n2, u_n2);
-        const float u_end = __ldg(P.unif + 2 * node_idx + 1);
+        // this item's candidate data has landed (it was requested one item ago) ...
+        if (warp == 0) cp_async_wait_all();
+        // ... and every warp is done with the previous item: the draft buffer and the
+        // oldest ring entries may be overwritten
+        if (!DIRECT) fence_proxy_async();
+        __syncthreads();
 
-        // ---- bring the slice into registers: tv = target, dv = draft
-        float tv[EPT], dv[EPT];
-        if (!DIRECT) {
-            if (!mbar_wait(full_addr, full_parity)) poisoned = 1;
-            full_parity ^= 1u;
-#pragma unroll
-            for (int j = 0; j < NVEC; ++j) {
-                const int vec = j * kThreads + tid;
-                uint4 raw = *reinterpret_cast<const uint4 *>(stage + vec * 16);
-                E::unpack(raw, &tv[j * VEC]);
-                if (internal) {
-                    raw = *reinterpret_cast<const uint4 *>(stage + kRowBytes + vec * 16);
-                    E::unpack(raw, &dv[j * VEC]);
-                }
-                if (vec >= n_full_vec) {  // ragged or empty vector: only at the slice end
-                    const int rem = n_mine - vec * VEC;
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) {
-                        if (e >= rem) { tv[j * VEC + e] = -INFINITY; dv[j * VEC + e] = -INFINITY; }
-                    }
-                }
+        const unsigned char *t_row = t_slice(item);
+        const unsigned char *d_row = d_slice(b, n);
+        const bool q_bulk = internal && bulk_bytes != 0;
+        if (tid == 0) {
+            if (q_bulk && !poisoned) {  // (after an expired wait nothing more is copied)
+                mbar_arrive_expect_tx(full_addr, bulk_bytes);
+                bulk_load(smem_u32(kRawZone ? static_cast<const void *>(qraw) : static_cast<const void *>(qbuf)),
+                          d_row, bulk_bytes, full_addr);
             }
-            __syncthreads();  // stage fully consumed: refill it with the next node of this cluster
-            if (tid == 0 && item + n_clusters < P.n_items) issue(item + n_clusters);
-        } else {
-            const unsigned char *t_row = reinterpret_cast<const unsigned char *>(P.target) +
-                node_idx * P.ld_t * E::kBytes;
-            const unsigned char *d_row = reinterpret_cast<const unsigned char *>(P.draft) +
-                (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes;
-#pragma unroll
-            for (int j = 0; j < NVEC; ++j) {
-                const int base = (j * kThreads + tid) * VEC;
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) {
-                    const bool ok = base + e < n_mine;
-                    tv[j * VEC + e] = ok ? E::load(t_row, v_begin + base + e) : -INFINITY;
-                    if (internal) dv[j * VEC + e] = ok ? E::load(d_row, v_begin + base + e) : -INFINITY;
-                }
+            const int nx = item + n_clusters;
+            if (!DIRECT && nx < P.n_items && bulk_bytes) {
+                const int nb = nx / P.n_nodes, nn = nx - nb * P.n_nodes;
+                bulk_prefetch_l2(t_slice(nx), bulk_bytes);
+                if (nn < P.n_internal) bulk_prefetch_l2(d_slice(nb, nn), bulk_bytes);
             }
         }
+        if (warp == 0) {
+            fetch_logits(item + n_clusters, (it + 1) % 3u, s2 ^ 1);
+            fetch_tokens(item + 2 * n_clusters, (it + 2) % 3u);
+            fetch_u_end(item + n_clusters, s2 ^ 1);
+        }
 
-        // ---- softmax statistics, one cluster-wide round for both rows.  Each thread
-        // exponentiates relative to its own maximum (reference r = max * scale, in
-        // log2 units); the factor to the global reference and the normaliser are
-        // applied as per-thread scalars afterwards, never per element.
-        float vs[NVEC];  // per-vector weight sums of this thread, in the thread's own units
-        float mt = -INFINITY, md = -INFINITY;
+        // ---- target slice -> registers
+        float tv[EPT];
+#pragma unroll
+        for (int j = 0; j < NG; ++j) {
+            const int e0 = group_of(j) * GV;
+            if (!DIRECT && e0 + GV <= n_mine) {
+                E::unpack(ld_stream_v4(t_row + static_cast<size_t>(e0) * E::kBytes), &tv[j * GV]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < GV; ++e)
+                    tv[j * GV + e] = (e0 + e < n_mine) ? E::load(t_row, e0 + e) : -INFINITY;
+            }
+        }
+        // Each thread exponentiates relative to its own integer reference; the factor to
+        // the row's reference and the normaliser are applied as per-thread scalars later.
+        float mt = -INFINITY;
 #pragma unroll
         for (int e = 0; e < EPT; ++e) mt = fmaxf(mt, tv[e]);
-        // rt / rd: this thread's references (-inf when it holds no finite element)
-        const float rt = (mt == -INFINITY) ? -INFINITY : mt * scale;
-        const float rt0 = (mt == -INFINITY) ? 0.f : rt;
-        float zt = 0.f, zd = 0.f, rd = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < NVEC; ++j) {
-            float s = 0.f;
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                const float x = ex2f(fmaf(tv[j * VEC + e], scale, -rt0));
-                tv[j * VEC + e] = x;
-                s += x;
-            }
-            vs[j] = s;
-            zt += s;
-        }
-        if (internal) {
-#pragma unroll
-            for (int e = 0; e < EPT; ++e) md = fmaxf(md, dv[e]);
-            rd = (md == -INFINITY) ? -INFINITY : md * scale;
-            const float rd0 = (md == -INFINITY) ? 0.f : rd;
+        const float rt = int_ref(mt * scale);
+        float zt = 0.f;
+        {
+            const float rt0 = (rt == -INFINITY) ? 0.f : rt;
+            float z[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int e = 0; e < EPT; ++e) {
-                const float x = ex2f(fmaf(dv[e], scale, -rd0));
-                dv[e] = x;
-                zd += x;
+                const float x = ex2f(fmaf(tv[e], scale, -rt0));
+                tv[e] = x;
+                z[e & 3] += x;
             }
+            zt = (z[0] + z[1]) + (z[2] + z[3]);
         }
+
+        // ---- draft slice: exponentiated in shared memory
+        auto read_q_raw = [&](int j, float *r) {
+            const int e0 = group_of(j) * GV;
+            if (!DIRECT && e0 + GV <= n_mine) {
+                const uint4 raw = kRawZone ? qraw[group_of(j)]
+                                           : *reinterpret_cast<const uint4 *>(&qbuf[group_of(j)]);
+                E::unpack(raw, r);
+            } else {
+#pragma unroll
+                for (int e = 0; e < GV; ++e) r[e] = (e0 + e < n_mine) ? E::load(d_row, e0 + e) : -INFINITY;
+            }
+        };
+        float zd = 0.f, rd = -INFINITY;
+        if (internal) {
+            if (q_bulk && !poisoned) {
+                if (!mbar_wait(full_addr, full_parity)) poisoned = 1;
+                full_parity ^= 1u;
+            }
+            float md = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                float r[GV];
+                read_q_raw(j, r);
+#pragma unroll
+                for (int e = 0; e < GV; ++e) md = fmaxf(md, r[e]);
+            }
+            rd = int_ref(md * scale);
+            const float rd0 = (rd == -INFINITY) ? 0.f : rd;
+            float z[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                float r[GV];
+                read_q_raw(j, r);
+#pragma unroll
+                for (int e = 0; e < GV; ++e) {
+                    r[e] = ex2f(fmaf(r[e], scale, -rd0));
+                    z[e & 3] += r[e];
+                }
+#pragma unroll
+                for (int h = 0; h < H; ++h)
+                    qbuf[qslot(j, h)] = make_float4(r[4 * h], r[4 * h + 1], r[4 * h + 2], r[4 * h + 3]);
+            }
+            zd = (z[0] + z[1]) + (z[2] + z[3]);
+        }
+
+        // ---- softmax statistics of both rows: one exchange round
         {
             const float Rt = warp_max(rt), Rd = warp_max(rd);
-            const float st = warp_sum(zt * rebase(rt, Rt));
-            const float sd = warp_sum(zd * rebase(rd, Rd));
-            if (lane == 0) red[warp] = make_float4(Rt, st, Rd, sd);
+            const float st = warp_sum(zt * exp2i(rt - Rt));
+            const float sd = warp_sum(zd * exp2i(rd - Rd));
+            exchange_send(make_float4(Rt, st, Rd, sd));  // per warp: (ref_t, z_t, ref_d, z_d)
         }
-        __syncthreads();
-        float4 cta = make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
-        if (warp == 0) {
-            if (lane < kWarps) cta = red[lane];
-            const float Rt = warp_max(cta.x), Rd = warp_max(cta.z);
-            cta.y = warp_sum(cta.y * rebase(cta.x, Rt));
-            cta.w = warp_sum(cta.w * rebase(cta.z, Rd));
-            cta.x = Rt; cta.z = Rd;
-        }
-        const float4 *slot = exchange(cta);  // per CTA: (ref_t, z_t, ref_d, z_d)
-        float R_t = -INFINITY, R_d = -INFINITY;  // global references: fl(row maximum * scale)
-#pragma unroll
-        for (uint32_t r = 0; r < kMaxCluster; ++r)
-            if (r < csize) { R_t = fmaxf(R_t, slot[r].x); R_d = fmaxf(R_d, slot[r].z); }
-        float Z_t = 0.f, Z_d = 0.f;
-#pragma unroll
-        for (uint32_t r = 0; r < kMaxCluster; ++r)
-            if (r < csize) {
-                Z_t += slot[r].y * rebase(slot[r].x, R_t);
-                Z_d += slot[r].w * rebase(slot[r].z, R_d);
+        // While the round is in flight: the candidates' own logits as 2^int * frac in double
+        // (lane i = candidate i; every warp keeps its own copy so that no CTA barrier is needed).
+        double frac_t = 0.0, frac_d = 0.0;
+        int int_t = 0, int_d = 0;
+        bool cand_ok = false;
+        int my_tok = -1;
+        if (lane < k) {
+            my_tok = ring.tok[s3][lane];
+            cand_ok = my_tok >= 0 && my_tok < P.V;
+            if (cand_ok) {
+                const uint32_t wt = ring.tl[s2][lane], wd = ring.dl[s2][lane];
+                const double at = static_cast<double>(DIRECT ? __uint_as_float(wt) : E::from_word(wt, my_tok)) * P.scale_d;
+                const double ad = static_cast<double>(DIRECT ? __uint_as_float(wd) : E::from_word(wd, my_tok)) * P.scale_d;
+                const double it_ = rint(at), id_ = rint(ad);
+                // |scaled logit| beyond 2^30 cannot be told from +-inf here
+                int_t = static_cast<int>(fmin(fmax(it_, -1073741824.0), 1073741824.0));
+                int_d = static_cast<int>(fmin(fmax(id_, -1073741824.0), 1073741824.0));
+                frac_t = (at == at && fabs(at) < 1e300) ? exp2(at - it_) : (at > 0 ? INFINITY : 0.0);
+                frac_d = (ad == ad && fabs(ad) < 1e300) ? exp2(ad - id_) : (ad > 0 ? INFINITY : 0.0);
             }
+        }
+        float4 ent = exchange_wait(make_float4(-INFINITY, 0.f, -INFINITY, 0.f));
+        // row references ceil(row maximum * scale) and normalisers, the same bits in every thread
+        const float R_t = warp_max(ent.x), R_d = warp_max(ent.z);
+        const float Z_t = warp_sum(ent.y * exp2i(ent.x - R_t));
+        const float Z_d = warp_sum(ent.w * exp2i(ent.z - R_d));
         const bool t_ok = Z_t > 0.f && Z_t < INFINITY;            // false for an all -inf or NaN row
         const bool d_ok = internal && Z_d > 0.f && Z_d < INFINITY;
         if (!t_ok) status_bits |= MCSD_STATUS_NO_MASS;
         // p(x) = tv * a, q(x) = dv * bq for this thread's elements
-        const float a = t_ok ? rebase(rt, R_t) / Z_t : 0.f;
-        const float bq = d_ok ? rebase(rd, R_d) / Z_d : 0.f;
-        const float b_over_a = a > 0.f ? bq / a : 0.f;
-        bool leaf_masses = true;  // slot holds softmax statistics (true) or residual partial sums
+        const float a = t_ok ? exp2i(rt - R_t) / Z_t : 0.f;
+        float b_over_a = 0.f;  // bq / a
+        if (a > 0.f && d_ok && rd != -INFINITY)
+            b_over_a = exp2i((rd - R_d) - (rt - R_t)) * (Z_t / Z_d);
+        // mass of this lane's exchange entry under the distribution the endpoint is drawn
+        // from; starts as the target softmax, replaced by residual partial sums below
+        float ent_mass = t_ok ? ent.y * exp2i(ent.x - R_t) / Z_t : 0.f;
+        if (crank == 0 && tid == 0)
+            *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
 
-        // ---- probabilities of the candidates themselves, once per CTA, in double
-        if (k > 0) {
-            if (warp == 0 && lane < k) {
-                const bool ok = xt >= 0 && xt < P.V;
-                s_px[lane] = (ok && t_ok) ? exp2(static_cast<double>(tl) * P.scale_d - static_cast<double>(R_t)) /
-                                                static_cast<double>(Z_t) : 0.0;
-                s_qx[lane] = (ok && d_ok) ? exp2(static_cast<double>(dl) * P.scale_d - static_cast<double>(R_d)) /
-                                                static_cast<double>(Z_d) : 0.0;
+        // Candidates' probabilities, both multiplied by K = Z_t * Z_d so that no division is
+        // needed: px' = 2^(l_t*scale - R_t) * Z_d, qx' = 2^(l_d*scale - R_d) * Z_t.
+        const double K = static_cast<double>(Z_t) * static_cast<double>(Z_d);
+        if (lane < k) {
+            double px = 0.0, qx = 0.0;
+            if (cand_ok && t_ok && d_ok) {
+                px = frac_t * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
+                qx = frac_d * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
             }
-            __syncthreads();
+            s_px[warp][lane] = px;
+            s_qx[warp][lane] = qx;
         }
+        __syncwarp();
 
-        // ---- the rejection loop (Algorithm 1 / Algorithm 2), identical in every thread
-        double c = 0.0, S = 1.0, W = 1.0;
-        float kappa = 0.f;  // c * bq / a: the residual weight of an element is max(tv - kappa dv, 0) * a
+        // residual mass of this warp's run for a given c
+        auto residual_pass = [&](float c_f) -> float {
+            const float kappa = fminf(c_f * b_over_a, 3.0e38f);
+            float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    const float4 d = qbuf[qslot(j, h)];
+                    const int o = j * GV + 4 * h;
+                    s[0] += fmaxf(fmaf(-kappa, d.x, tv[o]), 0.f);
+                    s[1] += fmaxf(fmaf(-kappa, d.y, tv[o + 1]), 0.f);
+                    s[2] += fmaxf(fmaf(-kappa, d.z, tv[o + 2]), 0.f);
+                    s[3] += fmaxf(fmaf(-kappa, d.w, tv[o + 3]), 0.f);
+                }
+            }
+            return warp_sum(((s[0] + s[1]) + (s[2] + s[3])) * a);
+        };
+
+        // ---- the rejection loop (Algorithm 1 / Algorithm 2), identical in every thread;
+        // state in units where W' = W * K
+        double c = 0.0, S = 1.0, Wk = K;
         int accepted = -1;
         for (int i = 0; i < k; ++i) {
-            const int xi = __shfl_sync(0xffffffffu, xt, i);
-            const float ui = __shfl_sync(0xffffffffu, u_acc, i);
-            const double pxi = s_px[i], qxi = s_qx[i];
+            const int xi = __shfl_sync(0xffffffffu, my_tok, i);
+            const double ui = static_cast<double>(ring.u[s3][i]);
+            const double pxi = s_px[warp][i], qxi = s_qx[warp][i];
             const bool valid = xi >= 0 && xi < P.V;
             if (!valid) status_bits |= MCSD_STATUS_BAD_TOKEN;
             // Algorithm 2: a token rejected earlier at this node has draft probability 0 now
             const bool dup = P.mode == 1 &&
-                (__ballot_sync(0xffffffffu, lane < i && xt == xi) != 0u);
-            const bool zero_q = !valid || dup || !(qxi > 0.0) || !(W > 0.0);
+                (__ballot_sync(0xffffffffu, lane < i && my_tok == xi) != 0u);
+            const bool zero_q = !valid || dup || !(qxi > 0.0) || !(Wk > 0.0);
             double Pn = pxi - c * qxi;
             Pn = Pn > 0.0 ? Pn : 0.0;
-            // r <= [P_n(x~)/S_n] / [q(x~)/W_n], written without the divisions (all factors > 0)
-            const bool accept = !zero_q && static_cast<double>(ui) * S * qxi <= Pn * W;
+            // r <= [P_n(x~)/S_n] / [q(x~)/W_n] without divisions (all factors > 0)
+            const bool accept = !zero_q && ui * S * qxi * K <= Pn * Wk;
             if (P.node_ratio && crank == 0 && tid == 0)
                 P.node_ratio[static_cast<long long>(b) * P.n_nodes + first + i] =
-                    zero_q ? -1.f : static_cast<float>((Pn / S) / (qxi / W));
+                    zero_q ? -1.f : static_cast<float>((Pn / S) / (qxi * K / Wk));
             if (accept) { accepted = first + i; break; }
             // rejected: p := norm(max(0, p - q)); Algorithm 2 also removes x~ from q
             double c_try = c;
-            if (W > 0.0) c_try = (P.mode == 1) ? c + S / W : c + S;
-            if (P.mode == 1 && !zero_q) { W -= qxi; if (!(W > 0.0)) W = 0.0; }
+            if (Wk > 0.0) c_try = (P.mode == 1) ? c + S * K / Wk : c + S;
+            if (P.mode == 1 && !zero_q) { Wk -= qxi; if (!(Wk > 0.0)) Wk = 0.0; }
             for (int attempt = 0; attempt < 2; ++attempt) {
-                kappa = static_cast<float>(c_try) * b_over_a;
-                float part = 0.f;
-#pragma unroll
-                for (int j = 0; j < NVEC; ++j) {
-                    float s = 0.f;
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) s += fmaxf(fmaf(-kappa, dv[j * VEC + e], tv[j * VEC + e]), 0.f);
-                    vs[j] = s;
-                    part += s;
-                }
-                part = warp_sum(part * a);
-                if (lane == 0) red[warp].x = part;
-                __syncthreads();
-                float cta_part = 0.f;
-                if (warp == 0) cta_part = warp_sum(lane < kWarps ? red[lane].x : 0.f);
-                slot = exchange(make_float4(cta_part, 0.f, 0.f, 0.f));
-                leaf_masses = false;
-                float S_new = 0.f;
-#pragma unroll
-                for (uint32_t r = 0; r < kMaxCluster; ++r)
-                    if (r < csize) S_new += slot[r].x;
+                exchange_send(make_float4(residual_pass(static_cast<float>(c_try)), 0.f, 0.f, 0.f));
+                ent = exchange_wait(make_float4(0.f, 0.f, 0.f, 0.f));
+                ent_mass = ent.x;
+                const float S_new = warp_sum(ent.x);
                 if (S_new > 0.f) {
                     if (attempt == 0) { c = c_try; S = static_cast<double>(S_new); }
                     break;
@@ -571,107 +709,98 @@ node_kernel(const __grid_constant__ NodeParams P)
         }
 
         // ---- endpoint token of a node that can end the walk: inverse CDF in token
-        // order over w(x) = max(p - c q, 0); only the CTA whose slice holds the
-        // quantile searches, the others go on to their next node.  vs[] holds this
-        // thread's per-vector sums of w / a.
+        // order over w(x) = max(p - c q, 0).  The exchange entries are the masses of all
+        // warps' runs in vocabulary order, so every warp can tell which one holds the
+        // quantile; only that warp searches, everyone else moves on.
         int bonus = -1;
-        bool bonus_mine = false;
+        bool no_mass = false;
         if (accepted < 0) {
-            const float inv_zt = t_ok ? 1.f / Z_t : 0.f;
-            float total = 0.f;
-#pragma unroll
-            for (uint32_t r = 0; r < kMaxCluster; ++r)
-                if (r < csize)
-                    total += leaf_masses ? slot[r].y * rebase(slot[r].x, R_t) * inv_zt : slot[r].x;
+            const float u_end = ring.u_end[s2];
+            const float total = warp_sum(ent_mass);
             const float target = u_end * total;
-            int owner = -1, last_pos = -1;
-            float cum = 0.f, before = 0.f, last_before = 0.f;
-#pragma unroll
-            for (uint32_t r = 0; r < kMaxCluster; ++r) {
-                if (r < csize) {
-                    const float m = leaf_masses ? slot[r].y * rebase(slot[r].x, R_t) * inv_zt : slot[r].x;
-                    if (m > 0.f) {
-                        last_pos = r; last_before = cum;
-                        if (owner < 0 && cum + m > target) { owner = r; before = cum; }
-                    }
-                    cum += m;
-                }
-            }
-            if (owner < 0) { owner = last_pos; before = last_before; }  // rounding pushed the quantile past the end
-            if (owner < 0 || !(total > 0.f)) {
+            const float inc = warp_scan_incl(ent_mass, lane);
+            const unsigned hit = __ballot_sync(0xffffffffu, ent_mass > 0.f && inc > target);
+            const unsigned pos = __ballot_sync(0xffffffffu, ent_mass > 0.f);
+            // (rounding may push the quantile past the end: clamp to the last entry with mass)
+            const int pick = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
+            if (pick < 0 || !(total > 0.f)) {
+                no_mass = true;
                 status_bits |= MCSD_STATUS_NO_MASS;
-                bonus_mine = crank == 0;
-            } else if (owner == static_cast<int>(crank)) {
-                bonus_mine = true;
-                float tgt = target - before;  // quantile inside this CTA's slice
-                float wv[NVEC];
+            } else if (pick == static_cast<int>(crank) * NW + warp) {
+                float tgt = target - __shfl_sync(0xffffffffu, inc - ent_mass, pick);  // quantile inside this run
+                const float kappa = internal ? fminf(static_cast<float>(c) * b_over_a, 3.0e38f) : 0.f;
+                auto weight = [&](int j, int h, int q4, const float4 &d) -> float {
+                    const float dq = q4 == 0 ? d.x : (q4 == 1 ? d.y : (q4 == 2 ? d.z : d.w));
+                    const float t = tv[j * GV + 4 * h + q4];
+                    return (internal ? fmaxf(fmaf(-kappa, dq, t), 0.f) : t) * a;
+                };
+                // level 2: group index j (32 consecutive groups each), warp totals per j
+                float wg[NG];
 #pragma unroll
-                for (int j = 0; j < NVEC; ++j) wv[j] = vs[j] * a;
-                float wtot;
-                const int wj = warp_multi_sum<NVEC>(wv, lane, wtot);
-                if ((lane & 3) == 0) wsum[wj * kWarps + warp] = wtot;  // lanes sharing an index write the same total
-                __syncthreads();
-                // level 1: (chunk j, warp) in token order
-                constexpr int kEntries = NVEC * kWarps;
-                int pick = -1, last_e = -1;
-                float run = 0.f, pick_before = 0.f, last_b = 0.f;
+                for (int j = 0; j < NG; ++j) {
+                    float sum = 0.f;
 #pragma unroll
-                for (int base = 0; base < kEntries; base += 32) {
-                    const int idx = base + lane;
-                    const float w = idx < kEntries ? wsum[idx] : 0.f;
-                    const float inc = warp_scan_incl(w, lane) + run;
-                    const unsigned hit = __ballot_sync(0xffffffffu, w > 0.f && inc > tgt);
-                    const unsigned pos = __ballot_sync(0xffffffffu, w > 0.f);
-                    if (pick < 0 && hit) {
-                        const int l = __ffs(hit) - 1;
-                        pick = base + l;
-                        pick_before = __shfl_sync(0xffffffffu, inc, l) - __shfl_sync(0xffffffffu, w, l);
+                    for (int h = 0; h < H; ++h) {
+                        const float4 d = internal ? qbuf[qslot(j, h)] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) sum += weight(j, h, q4, d);
                     }
-                    if (pos) {
-                        const int l = 31 - __clz(pos);
-                        last_e = base + l;
-                        last_b = __shfl_sync(0xffffffffu, inc, l) - __shfl_sync(0xffffffffu, w, l);
-                    }
-                    run = __shfl_sync(0xffffffffu, inc, 31);
+                    wg[j] = sum;
                 }
-                if (pick < 0) { pick = last_e; pick_before = last_b; }  // clamp to the last entry with mass
-                if (pick >= 0) {
-                    const int pj = pick / kWarps, pw = pick - pj * kWarps;
-                    if (warp == pw) {
-                        tgt -= pick_before;
-                        float v = wv[0];
+                float tj;
+                warp_multi_sum<NG>(wg, lane, tj);  // lane j * (32 / NG) holds the total of index j
+                int pj = -1, last_j = -1;
+                float runj = 0.f, pj_before = 0.f, last_jb = 0.f;
 #pragma unroll
-                        for (int j = 1; j < NVEC; ++j) v = (pj == j) ? wv[j] : v;
-                        const float inc = warp_scan_incl(v, lane);
-                        const unsigned hit = __ballot_sync(0xffffffffu, v > 0.f && inc > tgt);
-                        const unsigned pos = __ballot_sync(0xffffffffu, v > 0.f);
-                        const int l = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
-                        if (l >= 0 && lane == l) {
-                            const float rem = tgt - (inc - v);
-                            float acc = 0.f;
-                            int pe = -1, last = -1;
+                for (int j = 0; j < NG; ++j) {
+                    const float m = __shfl_sync(0xffffffffu, tj, j * (32 / NG));
+                    if (m > 0.f) {
+                        last_j = j; last_jb = runj;
+                        if (pj < 0 && runj + m > tgt) { pj = j; pj_before = runj; }
+                    }
+                    runj += m;
+                }
+                if (pj < 0) { pj = last_j; pj_before = last_jb; }
+                if (pj >= 0) {
+                    tgt -= pj_before;
+                    // level 3: the lane inside index pj
+                    float v = wg[0];
 #pragma unroll
-                            for (int j = 0; j < NVEC; ++j) {
-                                if (j == pj) {
+                    for (int j = 1; j < NG; ++j) v = (pj == j) ? wg[j] : v;
+                    const float incl = warp_scan_incl(v, lane);
+                    const unsigned hit3 = __ballot_sync(0xffffffffu, v > 0.f && incl > tgt);
+                    const unsigned pos3 = __ballot_sync(0xffffffffu, v > 0.f);
+                    const int l = hit3 ? __ffs(hit3) - 1 : (pos3 ? 31 - __clz(pos3) : -1);
+                    if (l >= 0 && lane == l) {
+                        // level 4: the element inside the group
+                        const float rem = tgt - (incl - v);
+                        float acc = 0.f;
+                        int pe = -1, last = -1;
 #pragma unroll
-                                    for (int e = 0; e < VEC; ++e) {
-                                        const float w = (internal ? fmaxf(fmaf(-kappa, dv[j * VEC + e], tv[j * VEC + e]), 0.f)
-                                                                  : tv[j * VEC + e]) * a;
+                        for (int j = 0; j < NG; ++j) {
+                            if (j == pj) {
+#pragma unroll
+                                for (int h = 0; h < H; ++h) {
+                                    const float4 d = internal ? qbuf[qslot(j, h)] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                                    for (int q4 = 0; q4 < 4; ++q4) {
+                                        const float w = weight(j, h, q4, d);
                                         if (w > 0.f) {
                                             acc += w;
-                                            last = e;
-                                            if (pe < 0 && acc > rem) pe = e;
+                                            last = 4 * h + q4;
+                                            if (pe < 0 && acc > rem) pe = 4 * h + q4;
                                         }
                                     }
                                 }
                             }
-                            if (pe < 0) pe = last;
-                            bonus = v_begin + (pj * kThreads + warp * 32 + lane) * VEC + pe;
-                            P.node_bonus[node_idx] = bonus;
                         }
+                        if (pe < 0) pe = last;
+                        bonus = v_begin + group_of(pj) * GV + pe;
+                        P.node_bonus[node_idx] = bonus;
                     }
-                } else if (tid == 0) {
-                    P.node_bonus[node_idx] = -1;
+                } else {
+                    // the run's exchanged mass was positive but its elements sum to nothing
+                    if (lane == 0) P.node_bonus[node_idx] = -1;
                     status_bits |= MCSD_STATUS_NO_MASS;
                 }
             }
@@ -680,24 +809,16 @@ node_kernel(const __grid_constant__ NodeParams P)
         // ---- per-node results
         if (crank == 0 && tid == 0) {
             P.node_accept[node_idx] = accepted;
-            if (accepted >= 0 || (bonus_mine && bonus < 0 && (status_bits & MCSD_STATUS_NO_MASS)))
-                P.node_bonus[node_idx] = -1;
-            NodeStats st;
-            st.r_t = R_t; st.r_d = R_d;
-            st.z_t = Z_t; st.z_d = Z_d;
-            st.c = static_cast<float>(c); st.s = static_cast<float>(S);
-            st.pad0 = 0; st.pad1 = 0;
-            P.stats[node_idx] = st;
+            if (accepted >= 0 || no_mass) P.node_bonus[node_idx] = -1;
+            reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
+                make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
         }
         if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
         status_bits = __reduce_or_sync(0xffffffffu, status_bits);
         if (status_bits && lane == 0) atomicOr(P.status + b, status_bits);
-
-        // rotate the candidate pipeline
-        xt = xt_n1; u_acc = u_n1; tl = tl_n1; dl = dl_n1;
-        xt_n1 = xt_n2; u_n1 = u_n2;
     }
 
+    if (warp == 0) cp_async_wait_all();
     // no CTA may leave while a peer can still write into its shared memory
     cluster_sync_all();
 }

@@ -74,13 +74,14 @@ def test_padded_row_stride():
     assert_parity(inp, out)
 
 
-@pytest.mark.parametrize("cluster,ept", [(1, 32), (2, 16), (4, 8), (8, 8), (8, 32), (2, 32)])
-def test_forced_cluster_shapes(cluster, ept, monkeypatch):
-    """Every cluster size / per-thread share computes the same thing."""
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("cluster,ept", [(1, 64), (2, 16), (4, 16), (8, 16), (8, 32), (2, 64), (4, 32)])
+def test_forced_cluster_shapes(cluster, ept, dtype, monkeypatch):
+    """Every cluster size / per-thread share computes the same thing (128 threads per CTA)."""
     monkeypatch.setenv("MCSD_CLUSTER", str(cluster))
     monkeypatch.setenv("MCSD_EPT", str(ept))
-    vocab = min(cluster * ept * 256 - 24, 9000)
-    w = synth.Workload("forced", 6, vocab, "4x2x1", "fp32", "normal", 2.5, 1.0, 1.0, 1.0, 1, 31 + cluster + ept)
+    vocab = min(cluster * ept * 128 - 24, 9000)
+    w = synth.Workload("forced", 6, vocab, "4x2x1", dtype, "normal", 2.5, 1.0, 1.0, 1.0, 1, 31 + cluster + ept)
     inp = synth.make_inputs(w, "cuda")
     _, out = run_library(inp)
     assert_parity(inp, out)
