@@ -316,6 +316,8 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     p.B = d->batch; p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
     p.slice = cfg.slice;
     p.n_items = static_cast<int32_t>(n_items);
+    p.step_b = static_cast<int32_t>(n_clusters / d->n_nodes);
+    p.step_n = static_cast<int32_t>(n_clusters % d->n_nodes);
     p.mode = mode;
     p.scale_d = 1.4426950408889634 / static_cast<double>(T);
     p.scale = static_cast<float>(p.scale_d);

@@ -70,6 +70,7 @@ struct NodeParams {
     int32_t B, n_nodes, n_internal, V;
     int32_t slice;   // vocabulary elements owned by one CTA of the cluster
     int32_t n_items; // B * n_nodes
+    int32_t step_b, step_n;  // quotient and remainder of (clusters in the grid) / n_nodes
     int32_t mode;
     float scale;     // log2(e) / T
     double scale_d;  // the same in double, for the candidates' own probabilities
@@ -106,6 +107,8 @@ template <> struct Elem<MCSD_DTYPE_BF16> {
     static __device__ __forceinline__ float from_word(uint32_t w, long long i) {
         return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));
     }
+    // 16-bit pattern of a value that this type represents exactly
+    static __device__ __forceinline__ uint32_t to_bits(float f) { return __float_as_uint(f) >> 16; }
 };
 template <> struct Elem<MCSD_DTYPE_F16> {
     static constexpr int kBytes = 2, kVec = 8;
@@ -124,6 +127,7 @@ template <> struct Elem<MCSD_DTYPE_F16> {
         const unsigned short h = static_cast<unsigned short>((i & 1) ? (w >> 16) : (w & 0xffffu));
         return __half2float(__ushort_as_half(h));
     }
+    static __device__ __forceinline__ uint32_t to_bits(float f) { return __half_as_ushort(__float2half_rn(f)); }
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -216,10 +220,19 @@ __device__ __forceinline__ void st_cluster_f4(uint32_t addr, float4 v) {
                  ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
+// Packed pairs of floats: sm_100 executes fma and add on both halves of an aligned
+// register pair with one instruction (each half rounds exactly like the scalar operation).
+typedef float2 f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { return __fadd2_rn(a, b); }
+// Three-input maximum (a NaN operand is ignored, as with fmaxf).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d;
+}
+// Warp-wide maximum in one instruction (NaN inputs are ignored).
 __device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
+    float d; asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(d) : "f"(v)); return d;
 }
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -334,6 +347,7 @@ constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
 // Ownership inside a CTA: the slice is cut into 16-byte groups of GV elements; thread
 // (warp w, lane l) owns groups (w * NG + j) * 32 + l, j < NG, so that one warp-wide
 // access is contiguous and a warp's elements are one contiguous run of the vocabulary.
+// Groups past the end of the slice hold -inf (probability 0).
 //
 // Every decision of the rejection loop is taken by every warp of the cluster from
 // bit-identical inputs, so all CTAs of a cluster execute the same number of exchange
@@ -353,7 +367,7 @@ node_kernel(const __grid_constant__ NodeParams P)
 
     extern __shared__ __align__(128) unsigned char dyn[];
     float4 *qbuf = reinterpret_cast<float4 *>(dyn);  // exponentiated draft slice, thread-private slots
-    const uint4 *qraw = reinterpret_cast<const uint4 *>(dyn + static_cast<size_t>(NT) * EPT * 4);
+    uint4 *qraw = reinterpret_cast<uint4 *>(dyn + static_cast<size_t>(NT) * EPT * 4);
     __shared__ Exchange xch;
     __shared__ __align__(8) unsigned long long full_bar;
     __shared__ double s_px[NW][MCSD_MAX_CHILDREN], s_qx[NW][MCSD_MAX_CHILDREN];
@@ -361,24 +375,27 @@ node_kernel(const __grid_constant__ NodeParams P)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t crank = cluster_ctarank(), csize = cluster_nctarank();
-    const int cluster_id = blockIdx.x / csize, n_clusters = gridDim.x / csize;
+    const int cluster_id = blockIdx.x / csize;
     const int n_entries = static_cast<int>(csize) * NW;  // values per exchange round (<= 32)
     const float scale = P.scale;
     const uint32_t full_addr = smem_u32(&full_bar);
 
-    // this CTA's slice of the vocabulary
+    // this CTA's slice of the vocabulary and this warp's run of it
     const int v_begin = static_cast<int>(crank) * P.slice;
     int n_mine = P.V - v_begin;
     n_mine = n_mine < 0 ? 0 : (n_mine > P.slice ? P.slice : n_mine);
-    // bytes of the slice that are whole 16-byte groups: what one bulk copy / prefetch moves
-    const uint32_t bulk_bytes = DIRECT ? 0u : static_cast<uint32_t>(n_mine / GV) * 16u;
+    const int n_full_groups = n_mine / GV;            // whole 16-byte groups
+    const int g0 = warp * (NG * 32) + lane;           // this thread's group of chunk 0
+    // every group of this warp is a whole group: the common case takes unpredicated loads
+    const bool warp_full = !DIRECT && (warp + 1) * (NG * 32) <= n_full_groups;
+    // bytes of the slice that are whole groups: what one bulk copy / prefetch moves
+    const uint32_t bulk_bytes = DIRECT ? 0u : static_cast<uint32_t>(n_full_groups) * 16u;
 
-    // slot of (group j, quarter h) in qbuf: for 4-byte logits it is the group's own place in
+    // slot of (chunk j, quarter h) in qbuf: for 4-byte logits it is the group's own place in
     // the slice, so that the bulk copy lands the raw values where the exponentiated ones go
     auto qslot = [&](int j, int h) -> int {
-        return E::kBytes == 4 ? (warp * NG + j) * 32 + lane : (j * H + h) * NT + tid;
+        return E::kBytes == 4 ? g0 + j * 32 : (j * H + h) * NT + tid;
     };
-    auto group_of = [&](int j) -> int { return (warp * NG + j) * 32 + lane; };
 
     if (tid == 0) {
         mbar_init(full_addr, 1);
@@ -390,9 +407,8 @@ node_kernel(const __grid_constant__ NodeParams P)
     uint32_t full_parity = 0, round = 0;
     int poisoned = 0;
 
-    auto t_slice = [&](int item) -> const unsigned char * {
-        return reinterpret_cast<const unsigned char *>(P.target) +
-            (static_cast<long long>(item) * P.ld_t + v_begin) * E::kBytes;
+    auto t_slice = [&](long long item) -> const unsigned char * {
+        return reinterpret_cast<const unsigned char *>(P.target) + (item * P.ld_t + v_begin) * E::kBytes;
     };
     auto d_slice = [&](int b, int n) -> const unsigned char * {
         return reinterpret_cast<const unsigned char *>(P.draft) +
@@ -417,10 +433,17 @@ node_kernel(const __grid_constant__ NodeParams P)
         return e;
     };
 
+    // (sequence, node) of the items this cluster visits: the current one and the two after
+    // it, advanced by the precomputed quotient and remainder of the stride
+    auto advance = [&](int &b, int &n) {
+        b += P.step_b;
+        n += P.step_n;
+        if (n >= P.n_nodes) { n -= P.n_nodes; ++b; }
+    };
+
     // ---- candidate pipeline (warp 0 only) -------------------------------------------
-    auto fetch_tokens = [&](int item, int slot3) {
-        if (item < P.n_items) {
-            const int b = item / P.n_nodes, n = item - b * P.n_nodes;
+    auto fetch_tokens = [&](int b, int n, int slot3) {
+        if (b < P.B) {
             const int k = n < P.n_internal ? P.child_count[n] : 0;
             if (lane < k) {
                 const long long ci = static_cast<long long>(b) * P.n_nodes + P.child_first[n] + lane;
@@ -429,19 +452,19 @@ node_kernel(const __grid_constant__ NodeParams P)
             }
         }
     };
-    auto fetch_u_end = [&](int item, int slot2) {
-        if (item < P.n_items && lane == 0) cp_async4(&ring.u_end[slot2], P.unif + 2 * static_cast<long long>(item) + 1);
+    auto fetch_u_end = [&](int b, int n, int slot2) {
+        if (b < P.B && lane == 0)
+            cp_async4(&ring.u_end[slot2], P.unif + 2 * (static_cast<long long>(b) * P.n_nodes + n) + 1);
     };
     // needs the item's tokens to have arrived (cp_async_wait_all by this thread)
-    auto fetch_logits = [&](int item, int slot3, int slot2) {
-        if (item < P.n_items) {
-            const int b = item / P.n_nodes, n = item - b * P.n_nodes;
+    auto fetch_logits = [&](int b, int n, int slot3, int slot2) {
+        if (b < P.B) {
             const int k = n < P.n_internal ? P.child_count[n] : 0;
             if (lane < k) {
                 const int xt = ring.tok[slot3][lane];
                 if (xt >= 0 && xt < P.V) {
                     const unsigned char *t = reinterpret_cast<const unsigned char *>(P.target) +
-                        (static_cast<long long>(item) * P.ld_t + xt) * E::kBytes;
+                        ((static_cast<long long>(b) * P.n_nodes + n) * P.ld_t + xt) * E::kBytes;
                     const unsigned char *d = reinterpret_cast<const unsigned char *>(P.draft) +
                         ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + xt) * E::kBytes;
                     if (!DIRECT) {  // rows are 16-byte aligned: the enclosing word lies inside the row
@@ -456,28 +479,30 @@ node_kernel(const __grid_constant__ NodeParams P)
         }
     };
 
-    int item = cluster_id;
+    int b = cluster_id / P.n_nodes, n = cluster_id - b * P.n_nodes;  // current item
+    int b1 = b, n1 = n;                                              // the next one
+    advance(b1, n1);
+    int b2 = b1, n2 = n1;                                            // the one after
+    advance(b2, n2);
     uint32_t it = 0;  // iteration count of this cluster
     if (warp == 0) {
-        fetch_tokens(item, 0);
-        fetch_u_end(item, 0);
+        fetch_tokens(b, n, 0);
+        fetch_u_end(b, n, 0);
         cp_async_wait_all();
         __syncwarp();
-        fetch_logits(item, 0, 0);
-        fetch_tokens(item + n_clusters, 1);
+        fetch_logits(b, n, 0, 0);
+        fetch_tokens(b1, n1, 1);
     }
-    if (!DIRECT && tid == 0 && item < P.n_items && bulk_bytes) {
-        const int b = item / P.n_nodes, n = item - b * P.n_nodes;
-        bulk_prefetch_l2(t_slice(item), bulk_bytes);
+    if (!DIRECT && tid == 0 && b < P.B && bulk_bytes) {
+        bulk_prefetch_l2(t_slice(static_cast<long long>(b) * P.n_nodes + n), bulk_bytes);
         if (n < P.n_internal) bulk_prefetch_l2(d_slice(b, n), bulk_bytes);
     }
 
-    for (; item < P.n_items; item += n_clusters, ++it) {
-        const int b = item / P.n_nodes, n = item - b * P.n_nodes;
+    for (; b < P.B; ++it) {
         const bool internal = n < P.n_internal;
         const int k = internal ? P.child_count[n] : 0;
         const int first = P.child_first[n];
-        const long long node_idx = item;  // b * n_nodes + n
+        const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
         const int s3 = it % 3u, s2 = it & 1u;
         int status_bits = 0;
 
@@ -488,7 +513,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (!DIRECT) fence_proxy_async();
         __syncthreads();
 
-        const unsigned char *t_row = t_slice(item);
+        const unsigned char *t_row = t_slice(node_idx);
         const unsigned char *d_row = d_slice(b, n);
         const bool q_bulk = internal && bulk_bytes != 0;
         if (tid == 0) {
@@ -497,94 +522,155 @@ node_kernel(const __grid_constant__ NodeParams P)
                 bulk_load(smem_u32(kRawZone ? static_cast<const void *>(qraw) : static_cast<const void *>(qbuf)),
                           d_row, bulk_bytes, full_addr);
             }
-            const int nx = item + n_clusters;
-            if (!DIRECT && nx < P.n_items && bulk_bytes) {
-                const int nb = nx / P.n_nodes, nn = nx - nb * P.n_nodes;
-                bulk_prefetch_l2(t_slice(nx), bulk_bytes);
-                if (nn < P.n_internal) bulk_prefetch_l2(d_slice(nb, nn), bulk_bytes);
+            if (!DIRECT && b1 < P.B && bulk_bytes) {
+                bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
+                if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
             }
         }
         if (warp == 0) {
-            fetch_logits(item + n_clusters, (it + 1) % 3u, s2 ^ 1);
-            fetch_tokens(item + 2 * n_clusters, (it + 2) % 3u);
-            fetch_u_end(item + n_clusters, s2 ^ 1);
+            fetch_logits(b1, n1, (it + 1) % 3u, s2 ^ 1);
+            fetch_tokens(b2, n2, (it + 2) % 3u);
+            fetch_u_end(b1, n1, s2 ^ 1);
         }
 
-        // ---- target slice -> registers
-        float tv[EPT];
+        // ---- target slice -> registers, as packed pairs
+        f32x2 tv[EPT / 2];
+        if (warp_full) {
+            // every group of this warp is a whole group inside the slice
 #pragma unroll
-        for (int j = 0; j < NG; ++j) {
-            const int e0 = group_of(j) * GV;
-            if (!DIRECT && e0 + GV <= n_mine) {
-                E::unpack(ld_stream_v4(t_row + static_cast<size_t>(e0) * E::kBytes), &tv[j * GV]);
-            } else {
+            for (int j = 0; j < NG; ++j) {
+                float f[GV];
+                E::unpack(ld_stream_v4(t_row + static_cast<size_t>(g0 + j * 32) * 16), f);
 #pragma unroll
-                for (int e = 0; e < GV; ++e)
-                    tv[j * GV + e] = (e0 + e < n_mine) ? E::load(t_row, e0 + e) : -INFINITY;
+                for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                const int g = g0 + j * 32;
+                float f[GV];
+                if (!DIRECT && g < n_full_groups) {
+                    E::unpack(ld_stream_v4(t_row + static_cast<size_t>(g) * 16), f);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(t_row, g * GV + e) : -INFINITY;
+                }
+#pragma unroll
+                for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
             }
         }
         // Each thread exponentiates relative to its own integer reference; the factor to
         // the row's reference and the normaliser are applied as per-thread scalars later.
-        float mt = -INFINITY;
-#pragma unroll
-        for (int e = 0; e < EPT; ++e) mt = fmaxf(mt, tv[e]);
-        const float rt = int_ref(mt * scale);
-        float zt = 0.f;
+        float rt, zt;
         {
-            const float rt0 = (rt == -INFINITY) ? 0.f : rt;
-            float z[4] = {0.f, 0.f, 0.f, 0.f};
+            float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-            for (int e = 0; e < EPT; ++e) {
-                const float x = ex2f(fmaf(tv[e], scale, -rt0));
-                tv[e] = x;
-                z[e & 3] += x;
+            for (int p = 0; p < EPT / 2; p += 2) {
+                m0 = max3(m0, tv[p].x, tv[p].y);
+                m1 = max3(m1, tv[p + 1].x, tv[p + 1].y);
             }
-            zt = (z[0] + z[1]) + (z[2] + z[3]);
+            rt = int_ref(fmaxf(m0, m1) * scale);
+            const float rt0 = (rt == -INFINITY) ? 0.f : rt;
+            const f32x2 scale2 = pack2(scale, scale), nref2 = pack2(-rt0, -rt0);
+            f32x2 z0 = pack2(0.f, 0.f), z1 = z0;
+#pragma unroll
+            for (int p = 0; p < EPT / 2; p += 2) {
+                const f32x2 x01 = fma2(tv[p], scale2, nref2), x23 = fma2(tv[p + 1], scale2, nref2);
+                tv[p] = pack2(ex2f(x01.x), ex2f(x01.y));
+                tv[p + 1] = pack2(ex2f(x23.x), ex2f(x23.y));
+                z0 = add2(z0, tv[p]);
+                z1 = add2(z1, tv[p + 1]);
+            }
+            const f32x2 z = add2(z0, z1);
+            zt = z.x + z.y;
         }
 
-        // ---- draft slice: exponentiated in shared memory
-        auto read_q_raw = [&](int j, float *r) {
-            const int e0 = group_of(j) * GV;
-            if (!DIRECT && e0 + GV <= n_mine) {
-                const uint4 raw = kRawZone ? qraw[group_of(j)]
-                                           : *reinterpret_cast<const uint4 *>(&qbuf[group_of(j)]);
-                E::unpack(raw, r);
-            } else {
-#pragma unroll
-                for (int e = 0; e < GV; ++e) r[e] = (e0 + e < n_mine) ? E::load(d_row, e0 + e) : -INFINITY;
-            }
-        };
+        // ---- draft slice: exponentiated in shared memory, in the slots of its owner
         float zd = 0.f, rd = -INFINITY;
         if (internal) {
-            if (q_bulk && !poisoned) {
-                if (!mbar_wait(full_addr, full_parity)) poisoned = 1;
-                full_parity ^= 1u;
-            }
-            float md = -INFINITY;
+            if (DIRECT) {
+                // the owner copies its raw elements into its slots, as float
 #pragma unroll
-            for (int j = 0; j < NG; ++j) {
-                float r[GV];
-                read_q_raw(j, r);
+                for (int j = 0; j < NG; ++j) {
+                    const int g = g0 + j * 32;
+                    float f[GV];
 #pragma unroll
-                for (int e = 0; e < GV; ++e) md = fmaxf(md, r[e]);
-            }
-            rd = int_ref(md * scale);
-            const float rd0 = (rd == -INFINITY) ? 0.f : rd;
-            float z[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(d_row, g * GV + e) : -INFINITY;
 #pragma unroll
-            for (int j = 0; j < NG; ++j) {
-                float r[GV];
-                read_q_raw(j, r);
-#pragma unroll
-                for (int e = 0; e < GV; ++e) {
-                    r[e] = ex2f(fmaf(r[e], scale, -rd0));
-                    z[e & 3] += r[e];
+                    for (int h = 0; h < H; ++h)
+                        qbuf[qslot(j, h)] = make_float4(f[4 * h], f[4 * h + 1], f[4 * h + 2], f[4 * h + 3]);
                 }
+            } else {
+                if (q_bulk && !poisoned) {
+                    if (!mbar_wait(full_addr, full_parity)) poisoned = 1;
+                    full_parity ^= 1u;
+                }
+                if (!warp_full) {
+                    // groups the bulk copy did not bring: -inf past the data, and the ragged
+                    // last group of the slice element by element (the slots are this thread's own)
 #pragma unroll
-                for (int h = 0; h < H; ++h)
-                    qbuf[qslot(j, h)] = make_float4(r[4 * h], r[4 * h + 1], r[4 * h + 2], r[4 * h + 3]);
+                    for (int j = 0; j < NG; ++j) {
+                        const int g = g0 + j * 32;
+                        if (g >= n_full_groups) {
+                            float f[GV];
+#pragma unroll
+                            for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(d_row, g * GV + e) : -INFINITY;
+                            if constexpr (kRawZone) {
+                                uint4 r;
+                                r.x = E::to_bits(f[0]) | (E::to_bits(f[1]) << 16);
+                                r.y = E::to_bits(f[2]) | (E::to_bits(f[3]) << 16);
+                                r.z = E::to_bits(f[4]) | (E::to_bits(f[5]) << 16);
+                                r.w = E::to_bits(f[6]) | (E::to_bits(f[7]) << 16);
+                                qraw[g] = r;
+                            } else {
+                                qbuf[g] = make_float4(f[0], f[1], f[2], f[3]);
+                            }
+                        }
+                    }
+                }
             }
-            zd = (z[0] + z[1]) + (z[2] + z[3]);
+            auto read_q_raw = [&](int j, float *r) {
+                if constexpr (kRawZone) {
+                    E::unpack(qraw[g0 + j * 32], r);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < H; ++h) {
+                        const float4 v = qbuf[qslot(j, h)];
+                        r[4 * h] = v.x; r[4 * h + 1] = v.y; r[4 * h + 2] = v.z; r[4 * h + 3] = v.w;
+                    }
+                }
+            };
+            float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                float r[GV];
+                read_q_raw(j, r);
+#pragma unroll
+                for (int e = 0; e < GV; e += 4) {
+                    m0 = max3(m0, r[e], r[e + 1]);
+                    m1 = max3(m1, r[e + 2], r[e + 3]);
+                }
+            }
+            rd = int_ref(fmaxf(m0, m1) * scale);
+            const float rd0 = (rd == -INFINITY) ? 0.f : rd;
+            const f32x2 scale2 = pack2(scale, scale), nref2 = pack2(-rd0, -rd0);
+            f32x2 z0 = pack2(0.f, 0.f), z1 = z0;
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                float r[GV];
+                read_q_raw(j, r);
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    const f32x2 x01 = fma2(pack2(r[4 * h], r[4 * h + 1]), scale2, nref2);
+                    const f32x2 x23 = fma2(pack2(r[4 * h + 2], r[4 * h + 3]), scale2, nref2);
+                    const float4 ev = make_float4(ex2f(x01.x), ex2f(x01.y), ex2f(x23.x), ex2f(x23.y));
+                    qbuf[qslot(j, h)] = ev;
+                    z0 = add2(z0, pack2(ev.x, ev.y));
+                    z1 = add2(z1, pack2(ev.z, ev.w));
+                }
+            }
+            const f32x2 z = add2(z0, z1);
+            zd = z.x + z.y;
         }
 
         // ---- softmax statistics of both rows: one exchange round
@@ -624,13 +710,14 @@ node_kernel(const __grid_constant__ NodeParams P)
         const bool d_ok = internal && Z_d > 0.f && Z_d < INFINITY;
         if (!t_ok) status_bits |= MCSD_STATUS_NO_MASS;
         // p(x) = tv * a, q(x) = dv * bq for this thread's elements
-        const float a = t_ok ? exp2i(rt - R_t) / Z_t : 0.f;
+        const float inv_zt = t_ok ? 1.f / Z_t : 0.f;
+        const float a = exp2i(rt - R_t) * inv_zt;
         float b_over_a = 0.f;  // bq / a
         if (a > 0.f && d_ok && rd != -INFINITY)
             b_over_a = exp2i((rd - R_d) - (rt - R_t)) * (Z_t / Z_d);
         // mass of this lane's exchange entry under the distribution the endpoint is drawn
         // from; starts as the target softmax, replaced by residual partial sums below
-        float ent_mass = t_ok ? ent.y * exp2i(ent.x - R_t) / Z_t : 0.f;
+        float ent_mass = ent.y * exp2i(ent.x - R_t) * inv_zt;
         if (crank == 0 && tid == 0)
             *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
 
@@ -651,20 +738,22 @@ node_kernel(const __grid_constant__ NodeParams P)
         // residual mass of this warp's run for a given c
         auto residual_pass = [&](float c_f) -> float {
             const float kappa = fminf(c_f * b_over_a, 3.0e38f);
-            float s[4] = {0.f, 0.f, 0.f, 0.f};
+            const f32x2 nk2 = pack2(-kappa, -kappa);
+            f32x2 s0 = pack2(0.f, 0.f), s1 = s0;
 #pragma unroll
             for (int j = 0; j < NG; ++j) {
 #pragma unroll
                 for (int h = 0; h < H; ++h) {
                     const float4 d = qbuf[qslot(j, h)];
-                    const int o = j * GV + 4 * h;
-                    s[0] += fmaxf(fmaf(-kappa, d.x, tv[o]), 0.f);
-                    s[1] += fmaxf(fmaf(-kappa, d.y, tv[o + 1]), 0.f);
-                    s[2] += fmaxf(fmaf(-kappa, d.z, tv[o + 2]), 0.f);
-                    s[3] += fmaxf(fmaf(-kappa, d.w, tv[o + 3]), 0.f);
+                    const int o = (j * GV + 4 * h) / 2;
+                    const f32x2 x01 = fma2(pack2(d.x, d.y), nk2, tv[o]);
+                    const f32x2 x23 = fma2(pack2(d.z, d.w), nk2, tv[o + 1]);
+                    s0 = add2(s0, pack2(fmaxf(x01.x, 0.f), fmaxf(x01.y, 0.f)));
+                    s1 = add2(s1, pack2(fmaxf(x23.x, 0.f), fmaxf(x23.y, 0.f)));
                 }
             }
-            return warp_sum(((s[0] + s[1]) + (s[2] + s[3])) * a);
+            const f32x2 t = add2(s0, s1);
+            return warp_sum((t.x + t.y) * a);
         };
 
         // ---- the rejection loop (Algorithm 1 / Algorithm 2), identical in every thread;
@@ -712,7 +801,6 @@ node_kernel(const __grid_constant__ NodeParams P)
         // order over w(x) = max(p - c q, 0).  The exchange entries are the masses of all
         // warps' runs in vocabulary order, so every warp can tell which one holds the
         // quantile; only that warp searches, everyone else moves on.
-        int bonus = -1;
         bool no_mass = false;
         if (accepted < 0) {
             const float u_end = ring.u_end[s2];
@@ -729,21 +817,29 @@ node_kernel(const __grid_constant__ NodeParams P)
             } else if (pick == static_cast<int>(crank) * NW + warp) {
                 float tgt = target - __shfl_sync(0xffffffffu, inc - ent_mass, pick);  // quantile inside this run
                 const float kappa = internal ? fminf(static_cast<float>(c) * b_over_a, 3.0e38f) : 0.f;
-                auto weight = [&](int j, int h, int q4, const float4 &d) -> float {
-                    const float dq = q4 == 0 ? d.x : (q4 == 1 ? d.y : (q4 == 2 ? d.z : d.w));
-                    const float t = tv[j * GV + 4 * h + q4];
-                    return (internal ? fmaxf(fmaf(-kappa, dq, t), 0.f) : t) * a;
+                // weights of the four elements of quarter h of chunk j
+                auto weights = [&](int j, int h, float *w) {
+                    float t0 = tv[(j * GV + 4 * h) / 2].x, t1 = tv[(j * GV + 4 * h) / 2].y;
+                    float t2 = tv[(j * GV + 4 * h) / 2 + 1].x, t3 = tv[(j * GV + 4 * h) / 2 + 1].y;
+                    if (internal) {
+                        const float4 d = qbuf[qslot(j, h)];
+                        t0 = fmaxf(fmaf(-kappa, d.x, t0), 0.f);
+                        t1 = fmaxf(fmaf(-kappa, d.y, t1), 0.f);
+                        t2 = fmaxf(fmaf(-kappa, d.z, t2), 0.f);
+                        t3 = fmaxf(fmaf(-kappa, d.w, t3), 0.f);
+                    }
+                    w[0] = t0 * a; w[1] = t1 * a; w[2] = t2 * a; w[3] = t3 * a;
                 };
-                // level 2: group index j (32 consecutive groups each), warp totals per j
+                // level 2: chunk index j (32 consecutive groups each), warp totals per j
                 float wg[NG];
 #pragma unroll
                 for (int j = 0; j < NG; ++j) {
                     float sum = 0.f;
 #pragma unroll
                     for (int h = 0; h < H; ++h) {
-                        const float4 d = internal ? qbuf[qslot(j, h)] : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) sum += weight(j, h, q4, d);
+                        float w[4];
+                        weights(j, h, w);
+                        sum += (w[0] + w[1]) + (w[2] + w[3]);
                     }
                     wg[j] = sum;
                 }
@@ -763,7 +859,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                 if (pj < 0) { pj = last_j; pj_before = last_jb; }
                 if (pj >= 0) {
                     tgt -= pj_before;
-                    // level 3: the lane inside index pj
+                    // level 3: the lane inside chunk pj
                     float v = wg[0];
 #pragma unroll
                     for (int j = 1; j < NG; ++j) v = (pj == j) ? wg[j] : v;
@@ -781,12 +877,12 @@ node_kernel(const __grid_constant__ NodeParams P)
                             if (j == pj) {
 #pragma unroll
                                 for (int h = 0; h < H; ++h) {
-                                    const float4 d = internal ? qbuf[qslot(j, h)] : make_float4(0.f, 0.f, 0.f, 0.f);
+                                    float w[4];
+                                    weights(j, h, w);
 #pragma unroll
                                     for (int q4 = 0; q4 < 4; ++q4) {
-                                        const float w = weight(j, h, q4, d);
-                                        if (w > 0.f) {
-                                            acc += w;
+                                        if (w[q4] > 0.f) {
+                                            acc += w[q4];
                                             last = 4 * h + q4;
                                             if (pe < 0 && acc > rem) pe = 4 * h + q4;
                                         }
@@ -795,8 +891,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                             }
                         }
                         if (pe < 0) pe = last;
-                        bonus = v_begin + group_of(pj) * GV + pe;
-                        P.node_bonus[node_idx] = bonus;
+                        P.node_bonus[node_idx] = v_begin + (g0 + pj * 32) * GV + pe;
                     }
                 } else {
                     // the run's exchanged mass was positive but its elements sum to nothing
@@ -816,6 +911,10 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
         status_bits = __reduce_or_sync(0xffffffffu, status_bits);
         if (status_bits && lane == 0) atomicOr(P.status + b, status_bits);
+
+        b = b1; n = n1;
+        b1 = b2; n1 = n2;
+        advance(b2, n2);
     }
 
     if (warp == 0) cp_async_wait_all();
