@@ -235,7 +235,7 @@ def run_cuda(args):
         e0.record()
         ver.mcsd_verify_nodes(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
         e1.record()
-        ver.mcsd_verify_walk(inp.target, draft, inp.cand, w.temperature)
+        ver.mcsd_verify_walk(inp.target, draft, inp.cand, inp.unif, w.temperature)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -243,7 +243,7 @@ def run_cuda(args):
     launches_per_step = 0
     ver.mcsd_verify_nodes(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
     launches_per_step += binding.mcsd_last_launch_count()
-    ver.mcsd_verify_walk(inp.target, draft, inp.cand, w.temperature)
+    ver.mcsd_verify_walk(inp.target, draft, inp.cand, inp.unif, w.temperature)
     launches_per_step += binding.mcsd_last_launch_count()
     torch.cuda.synchronize()
 

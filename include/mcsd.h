@@ -99,7 +99,8 @@ typedef struct mcsd_desc {
      * the first two in the workspace:                                              */
     int32_t *node_accept; /* [B][n_nodes] accepted child of each node, or -1          */
     int32_t *node_bonus;  /* [B][n_nodes] endpoint token of each node that can end a
-                             walk (leaf, or all candidates rejected), else -1       */
+                             walk (leaf, or all candidates rejected), else -1;
+                             asking for it adds a pass over every such node       */
     float *node_ratio;    /* [B][n_nodes] p/q seen by the test of each draft node; -1
                              for a forced rejection; untouched if never tested      */
     int32_t *out_status;  /* [B] MCSD_STATUS_* bits (device), NULL to skip            */
@@ -136,11 +137,11 @@ int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *dr
                 int32_t *out_tokens, float *out_residual);
 
 /*
- * Stage 1: the per-node part (softmax statistics of both models, the rejection
- * loop of Algorithm 1 / 2, the endpoint token of every node that can end a
- * walk).  Fills node_accept / node_bonus (in the workspace when the descriptor
- * leaves them NULL) and the per-node statistics kept in the workspace.
- * Arguments as in mcsd_verify.
+ * Stage 1: the per-node part (softmax statistics of both models at every node,
+ * the rejection loop of Algorithm 1 / 2 at every node that has children).  Fills
+ * node_accept (in the workspace when the descriptor leaves it NULL) and the
+ * per-node statistics kept in the workspace; at temperature 0 also node_bonus
+ * (the target argmax of every node).  Arguments as in mcsd_verify.
  */
 int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                       const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
@@ -148,13 +149,19 @@ int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const vo
 
 /*
  * Stage 2: the walk of Section 3 from the root along accepted children, using
- * what stage 1 left in the workspace of the same descriptor, and the residual
- * distribution of the node where each walk stops (recomputed from that node's
- * two logit rows and stored statistics).  Arguments as in mcsd_verify.
+ * what stage 1 left in the workspace of the same descriptor; then, for the node
+ * where each walk stops, the distribution its endpoint token is drawn from (the
+ * final residual of Algorithm 1 / 2, rebuilt from that node's two logit rows and
+ * the stored statistics) and the endpoint token itself ("x_end ~ p", last line
+ * of both algorithms).  An endpoint token is only ever used at the node where a
+ * walk stops, so it is drawn there and nowhere else; when the descriptor asks
+ * for node_bonus, the same draw is also made at every node that accepted no
+ * candidate, one CTA per node (a checking aid, not part of the timed path).
+ * Arguments as in mcsd_verify.
  */
 int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
-                     const int32_t *tree_parent, const int32_t *cand_tokens, float temperature,
-                     int32_t *out_accept_len, int32_t *out_tokens, float *out_residual);
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual);
 
 /*
  * The same step for callers whose data lives in HOST memory: every pointer below

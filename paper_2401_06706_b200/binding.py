@@ -62,7 +62,7 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_verify.restype = ctypes.c_int
     lib.mcsd_verify_nodes.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int]
     lib.mcsd_verify_nodes.restype = ctypes.c_int
-    lib.mcsd_verify_walk.argtypes = [dp, vp, vp, vp, vp, f32, vp, vp, vp]
+    lib.mcsd_verify_walk.argtypes = [dp, vp, vp, vp, vp, vp, f32, vp, vp, vp]
     lib.mcsd_verify_walk.restype = ctypes.c_int
     lib.mcsd_verify_host.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp, vp]
     lib.mcsd_verify_host.restype = ctypes.c_int
@@ -214,10 +214,10 @@ class Verifier:
                                           self.parent.ctypes.data, _ptr(cand), _ptr(unif), float(temperature),
                                           int(mode)))
 
-    def mcsd_verify_walk(self, target, draft, cand, temperature: float) -> VerifyOutput:
+    def mcsd_verify_walk(self, target, draft, cand, unif, temperature: float) -> VerifyOutput:
         self._bind(target, draft)
         _check(self.lib.mcsd_verify_walk(ctypes.byref(self.desc), _ptr(target), _ptr(draft),
-                                         self.parent.ctypes.data, _ptr(cand), float(temperature),
+                                         self.parent.ctypes.data, _ptr(cand), _ptr(unif), float(temperature),
                                          _ptr(self.accept_len), _ptr(self.tokens), _ptr(self.residual)))
         return self._out()
 

@@ -56,11 +56,12 @@ struct Workspace {
     int32_t *node_accept;
     int32_t *node_bonus;
     NodeStats *stats;
+    float2 *leaf_part;
     int32_t *status;
     size_t bytes;
 };
 
-Workspace carve(void *base, long long n_items, int batch)
+Workspace carve(void *base, long long n_items, long long n_leaf_items, int batch)
 {
     Workspace w;
     size_t off = 0;
@@ -72,6 +73,7 @@ Workspace carve(void *base, long long n_items, int batch)
     w.node_accept = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
     w.node_bonus = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
     w.stats = reinterpret_cast<NodeStats *>(take(sizeof(NodeStats) * n_items));
+    w.leaf_part = reinterpret_cast<float2 *>(take(sizeof(float2) * 32 * n_leaf_items));
     w.status = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
     w.bytes = off;
     return w;
@@ -93,7 +95,8 @@ int check_desc(const mcsd_desc *d)
 
 int check_workspace(const mcsd_desc *d)
 {
-    const Workspace need = carve(nullptr, static_cast<long long>(d->batch) * d->n_nodes, d->batch);
+    const Workspace need = carve(nullptr, static_cast<long long>(d->batch) * d->n_nodes,
+                                 static_cast<long long>(d->batch) * (d->n_nodes - d->n_internal), d->batch);
     if (!d->workspace) return MCSD_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(d->workspace) % 256 != 0) return MCSD_ERR_WORKSPACE;
     if (d->workspace_bytes < need.bytes) return MCSD_ERR_WORKSPACE;
@@ -239,7 +242,8 @@ int prepare(const mcsd_desc *d, const int32_t *parent, Call *c)
     rc = check_workspace(d);
     if (rc != MCSD_OK) return rc;
     c->d = d;
-    c->ws = carve(d->workspace, static_cast<long long>(d->batch) * d->n_nodes, d->batch);
+    c->ws = carve(d->workspace, static_cast<long long>(d->batch) * d->n_nodes,
+                  static_cast<long long>(d->batch) * (d->n_nodes - d->n_internal), d->batch);
     c->node_accept = d->node_accept ? d->node_accept : c->ws.node_accept;
     c->node_bonus = d->node_bonus ? d->node_bonus : c->ws.node_bonus;
     c->status = d->out_status ? d->out_status : c->ws.status;
@@ -310,8 +314,8 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
 
     NodeParams p = {};
     p.target = target; p.draft = draft; p.cand = cand; p.unif = unif;
-    p.node_accept = c.node_accept; p.node_bonus = c.node_bonus; p.node_ratio = d->node_ratio;
-    p.stats = c.ws.stats; p.status = c.status;
+    p.node_accept = c.node_accept; p.node_ratio = d->node_ratio;
+    p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part; p.status = c.status;
     p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
     p.B = d->batch; p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
     p.slice = cfg.slice;
@@ -344,27 +348,43 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     return MCSD_OK;
 }
 
-int launch_walk(const Call &c, const void *target, const void *draft, const int32_t *cand, float T,
-                int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
+int launch_walk(const Call &c, const void *target, const void *draft, const int32_t *cand,
+                const float *unif, float T, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
 {
     const mcsd_desc *d = c.d;
     if (d->batch == 0) return MCSD_OK;
     WalkParams p = {};
-    p.target = target; p.draft = draft; p.cand = cand;
-    p.node_accept = c.node_accept; p.node_bonus = c.node_bonus; p.stats = c.ws.stats;
+    p.target = target; p.draft = draft; p.cand = cand; p.unif = unif;
+    p.node_accept = c.node_accept; p.node_bonus = c.node_bonus;
+    p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part; p.status = c.status;
     p.out_accept_len = out_accept_len; p.out_tokens = out_tokens; p.out_residual = out_residual;
     p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
     p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab; p.gamma = c.plan.gamma;
     p.scale = T > 0.f ? static_cast<float>(1.4426950408889634 / static_cast<double>(T)) : 0.f;
-    const unsigned gx = out_residual ? static_cast<unsigned>((d->vocab + kThreads * 4 - 1) / (kThreads * 4)) : 1u;
-    const dim3 grid(gx, static_cast<unsigned>(d->batch));
-    switch (d->dtype) {
-    case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32><<<grid, kThreads, 0, c.stream>>>(p); break;
-    case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16><<<grid, kThreads, 0, c.stream>>>(p); break;
-    default: walk_kernel<MCSD_DTYPE_F16><<<grid, kThreads, 0, c.stream>>>(p); break;
+    const bool aligned = rows_aligned16(target, d->ld_target, d->dtype) &&
+        (T == 0.f || d->n_internal == 0 || rows_aligned16(draft, d->ld_draft, d->dtype));
+    p.vector_ok = aligned ? 1 : 0;
+    if (T > 0.f) {
+        // the leaf statistics were left one entry per warp of the node kernel's cluster
+        const bool node_aligned = rows_aligned16(target, d->ld_target, d->dtype) &&
+            (d->n_internal == 0 || rows_aligned16(draft, d->ld_draft, d->dtype));
+        NodeConfig cfg;
+        const int rc = choose_config(d->vocab, d->dtype, node_aligned, &cfg);
+        if (rc != MCSD_OK) return rc;
+        p.n_entries = cfg.cluster * kNodeWarps;
     }
-    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
-    g_last_launches += 1;
+    // all-nodes pass first (only when per-node endpoint tokens were asked for), then the walks
+    for (int all = (T > 0.f && d->node_bonus) ? 1 : 0; all >= 0; --all) {
+        p.all_nodes = all;
+        const unsigned grid = static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch);
+        switch (d->dtype) {
+        case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
+        case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
+        default: walk_kernel<MCSD_DTYPE_F16><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
+        }
+        if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+        g_last_launches += 1;
+    }
     return MCSD_OK;
 }
 
@@ -398,7 +418,8 @@ const char *mcsd_status_string(int code)
 size_t mcsd_workspace_bytes(const mcsd_desc *desc)
 {
     if (check_desc(desc) != MCSD_OK) return 0;
-    return carve(nullptr, static_cast<long long>(desc->batch) * desc->n_nodes, desc->batch).bytes;
+    return carve(nullptr, static_cast<long long>(desc->batch) * desc->n_nodes,
+                 static_cast<long long>(desc->batch) * (desc->n_nodes - desc->n_internal), desc->batch).bytes;
 }
 
 int mcsd_tree_depth(const int32_t *tree_parent, int32_t n_nodes)
@@ -426,19 +447,19 @@ int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const vo
 }
 
 int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
-                     const int32_t *tree_parent, const int32_t *cand_tokens, float temperature,
-                     int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
 {
     Call c;
     int rc = prepare(desc, tree_parent, &c);
     if (rc != MCSD_OK) return rc;
     g_last_launches = 0;
     if (desc->batch == 0) return MCSD_OK;
-    rc = check_common(desc, target_logits, draft_logits, cand_tokens, nullptr, temperature,
-                      MCSD_MODE_WITH_REPLACEMENT, false);
+    rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
+                      MCSD_MODE_WITH_REPLACEMENT, true);
     if (rc != MCSD_OK) return rc;
     if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
-    return launch_walk(c, target_logits, draft_logits, cand_tokens, temperature, out_accept_len,
+    return launch_walk(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, out_accept_len,
                        out_tokens, out_residual);
 }
 
@@ -458,7 +479,7 @@ int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *dr
     if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
     rc = launch_nodes(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, replacement_mode);
     if (rc != MCSD_OK) return rc;
-    return launch_walk(c, target_logits, draft_logits, cand_tokens, temperature, out_accept_len,
+    return launch_walk(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, out_accept_len,
                        out_tokens, out_residual);
 }
 

@@ -62,9 +62,9 @@ struct NodeParams {
     const int32_t *cand;
     const float *unif;
     int32_t *node_accept;
-    int32_t *node_bonus;
     float *node_ratio;  // may be null
-    NodeStats *stats;
+    NodeStats *stats;   // [B][n_nodes], written for nodes with children
+    float2 *leaf_part;  // [B][n_nodes - n_internal][32] per-warp (reference, sum) of every leaf row
     int32_t *status;  // [B]
     long long ld_t, ld_d;
     int32_t B, n_nodes, n_internal, V;
@@ -280,13 +280,11 @@ struct Exchange {
 // latency sits on the per-node critical path: lane i handles candidate i.
 //   token id and acceptance uniform   two items ahead  (ring of 3)
 //   the candidate's own two logits    one item ahead   (ring of 2; they need the token)
-//   the uniform of the endpoint draw  one item ahead   (ring of 2)
 struct CandRing {
     int32_t tok[3][MCSD_MAX_CHILDREN];
     float u[3][MCSD_MAX_CHILDREN];
     uint32_t tl[2][MCSD_MAX_CHILDREN];  // aligned 32-bit word holding the target logit
     uint32_t dl[2][MCSD_MAX_CHILDREN];  // same for the draft logit
-    float u_end[2];
 };
 
 // ------------------------------------------------------------------ node kernel
@@ -452,10 +450,6 @@ node_kernel(const __grid_constant__ NodeParams P)
             }
         }
     };
-    auto fetch_u_end = [&](int b, int n, int slot2) {
-        if (b < P.B && lane == 0)
-            cp_async4(&ring.u_end[slot2], P.unif + 2 * (static_cast<long long>(b) * P.n_nodes + n) + 1);
-    };
     // needs the item's tokens to have arrived (cp_async_wait_all by this thread)
     auto fetch_logits = [&](int b, int n, int slot3, int slot2) {
         if (b < P.B) {
@@ -485,9 +479,9 @@ node_kernel(const __grid_constant__ NodeParams P)
     int b2 = b1, n2 = n1;                                            // the one after
     advance(b2, n2);
     uint32_t it = 0;  // iteration count of this cluster
+    bool prev_internal = false;
     if (warp == 0) {
         fetch_tokens(b, n, 0);
-        fetch_u_end(b, n, 0);
         cp_async_wait_all();
         __syncwarp();
         fetch_logits(b, n, 0, 0);
@@ -508,30 +502,40 @@ node_kernel(const __grid_constant__ NodeParams P)
 
         // this item's candidate data has landed (it was requested one item ago) ...
         if (warp == 0) cp_async_wait_all();
-        // ... and every warp is done with the previous item: the draft buffer and the
-        // oldest ring entries may be overwritten
-        if (!DIRECT) fence_proxy_async();
-        __syncthreads();
+        // ... and, around an item with children, all warps meet: they are done with the
+        // previous item (its draft buffer and ring entries may be overwritten) and they
+        // see this item's ring entries.  A run of leaves needs no meeting at all.
+        if (internal || prev_internal) {
+            if (!DIRECT) fence_proxy_async();
+            __syncthreads();
+        }
+        prev_internal = internal;
 
         const unsigned char *t_row = t_slice(node_idx);
         const unsigned char *d_row = d_slice(b, n);
         const bool q_bulk = internal && bulk_bytes != 0;
-        if (tid == 0) {
-            if (q_bulk && !poisoned) {  // (after an expired wait nothing more is copied)
-                mbar_arrive_expect_tx(full_addr, bulk_bytes);
-                bulk_load(smem_u32(kRawZone ? static_cast<const void *>(qraw) : static_cast<const void *>(qbuf)),
-                          d_row, bulk_bytes, full_addr);
-            }
-            if (!DIRECT && b1 < P.B && bulk_bytes) {
-                bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
-                if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
-            }
+        if (tid == 0 && q_bulk && !poisoned) {  // (after an expired wait nothing more is copied)
+            mbar_arrive_expect_tx(full_addr, bulk_bytes);
+            bulk_load(smem_u32(kRawZone ? static_cast<const void *>(qraw) : static_cast<const void *>(qbuf)),
+                      d_row, bulk_bytes, full_addr);
         }
-        if (warp == 0) {
-            fetch_logits(b1, n1, (it + 1) % 3u, s2 ^ 1);
-            fetch_tokens(b2, n2, (it + 2) % 3u);
-            fetch_u_end(b1, n1, s2 ^ 1);
-        }
+        // look-ahead duties of warp 0: L2 prefetch of the next item's slices, candidate
+        // data of the next two items
+        auto look_ahead = [&]() {
+            if (warp == 0) {
+                if (!DIRECT && lane == 0 && b1 < P.B && bulk_bytes) {
+                    bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
+                    if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
+                }
+                fetch_logits(b1, n1, (it + 1) % 3u, s2 ^ 1);
+                fetch_tokens(b2, n2, (it + 2) % 3u);
+            }
+        };
+        auto next_item = [&]() {
+            b = b1; n = n1;
+            b1 = b2; n1 = n2;
+            advance(b2, n2);
+        };
 
         // ---- target slice -> registers, as packed pairs
         f32x2 tv[EPT / 2];
@@ -585,9 +589,24 @@ node_kernel(const __grid_constant__ NodeParams P)
             zt = z.x + z.y;
         }
 
+        if (!internal) {
+            // A leaf decides nothing.  Its softmax statistics are only needed if a walk ends
+            // here, so each warp leaves the partial statistics of its run in global memory
+            // (the walk kernel combines them) and goes on: no exchange, no barrier.
+            const float Rt = warp_max(rt);
+            const float st = warp_sum(zt * exp2i(rt - Rt));
+            if (lane == 0)
+                P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * 32 +
+                            crank * NW + warp] = make_float2(Rt, st);
+            if (crank == 0 && tid == 0) P.node_accept[node_idx] = -1;
+            look_ahead();
+            next_item();
+            continue;
+        }
+
         // ---- draft slice: exponentiated in shared memory, in the slots of its owner
         float zd = 0.f, rd = -INFINITY;
-        if (internal) {
+        {
             if (DIRECT) {
                 // the owner copies its raw elements into its slots, as float
 #pragma unroll
@@ -680,6 +699,7 @@ node_kernel(const __grid_constant__ NodeParams P)
             const float sd = warp_sum(zd * exp2i(rd - Rd));
             exchange_send(make_float4(Rt, st, Rd, sd));  // per warp: (ref_t, z_t, ref_d, z_d)
         }
+        look_ahead();  // in the shadow of the exchange
         // While the round is in flight: the candidates' own logits as 2^int * frac in double
         // (lane i = candidate i; every warp keeps its own copy so that no CTA barrier is needed).
         double frac_t = 0.0, frac_d = 0.0;
@@ -715,9 +735,6 @@ node_kernel(const __grid_constant__ NodeParams P)
         float b_over_a = 0.f;  // bq / a
         if (a > 0.f && d_ok && rd != -INFINITY)
             b_over_a = exp2i((rd - R_d) - (rt - R_t)) * (Z_t / Z_d);
-        // mass of this lane's exchange entry under the distribution the endpoint is drawn
-        // from; starts as the target softmax, replaced by residual partial sums below
-        float ent_mass = ent.y * exp2i(ent.x - R_t) * inv_zt;
         if (crank == 0 && tid == 0)
             *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
 
@@ -785,7 +802,6 @@ node_kernel(const __grid_constant__ NodeParams P)
             for (int attempt = 0; attempt < 2; ++attempt) {
                 exchange_send(make_float4(residual_pass(static_cast<float>(c_try)), 0.f, 0.f, 0.f));
                 ent = exchange_wait(make_float4(0.f, 0.f, 0.f, 0.f));
-                ent_mass = ent.x;
                 const float S_new = warp_sum(ent.x);
                 if (S_new > 0.f) {
                     if (attempt == 0) { c = c_try; S = static_cast<double>(S_new); }
@@ -797,124 +813,17 @@ node_kernel(const __grid_constant__ NodeParams P)
             }
         }
 
-        // ---- endpoint token of a node that can end the walk: inverse CDF in token
-        // order over w(x) = max(p - c q, 0).  The exchange entries are the masses of all
-        // warps' runs in vocabulary order, so every warp can tell which one holds the
-        // quantile; only that warp searches, everyone else moves on.
-        bool no_mass = false;
-        if (accepted < 0) {
-            const float u_end = ring.u_end[s2];
-            const float total = warp_sum(ent_mass);
-            const float target = u_end * total;
-            const float inc = warp_scan_incl(ent_mass, lane);
-            const unsigned hit = __ballot_sync(0xffffffffu, ent_mass > 0.f && inc > target);
-            const unsigned pos = __ballot_sync(0xffffffffu, ent_mass > 0.f);
-            // (rounding may push the quantile past the end: clamp to the last entry with mass)
-            const int pick = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
-            if (pick < 0 || !(total > 0.f)) {
-                no_mass = true;
-                status_bits |= MCSD_STATUS_NO_MASS;
-            } else if (pick == static_cast<int>(crank) * NW + warp) {
-                float tgt = target - __shfl_sync(0xffffffffu, inc - ent_mass, pick);  // quantile inside this run
-                const float kappa = internal ? fminf(static_cast<float>(c) * b_over_a, 3.0e38f) : 0.f;
-                // weights of the four elements of quarter h of chunk j
-                auto weights = [&](int j, int h, float *w) {
-                    float t0 = tv[(j * GV + 4 * h) / 2].x, t1 = tv[(j * GV + 4 * h) / 2].y;
-                    float t2 = tv[(j * GV + 4 * h) / 2 + 1].x, t3 = tv[(j * GV + 4 * h) / 2 + 1].y;
-                    if (internal) {
-                        const float4 d = qbuf[qslot(j, h)];
-                        t0 = fmaxf(fmaf(-kappa, d.x, t0), 0.f);
-                        t1 = fmaxf(fmaf(-kappa, d.y, t1), 0.f);
-                        t2 = fmaxf(fmaf(-kappa, d.z, t2), 0.f);
-                        t3 = fmaxf(fmaf(-kappa, d.w, t3), 0.f);
-                    }
-                    w[0] = t0 * a; w[1] = t1 * a; w[2] = t2 * a; w[3] = t3 * a;
-                };
-                // level 2: chunk index j (32 consecutive groups each), warp totals per j
-                float wg[NG];
-#pragma unroll
-                for (int j = 0; j < NG; ++j) {
-                    float sum = 0.f;
-#pragma unroll
-                    for (int h = 0; h < H; ++h) {
-                        float w[4];
-                        weights(j, h, w);
-                        sum += (w[0] + w[1]) + (w[2] + w[3]);
-                    }
-                    wg[j] = sum;
-                }
-                float tj;
-                warp_multi_sum<NG>(wg, lane, tj);  // lane j * (32 / NG) holds the total of index j
-                int pj = -1, last_j = -1;
-                float runj = 0.f, pj_before = 0.f, last_jb = 0.f;
-#pragma unroll
-                for (int j = 0; j < NG; ++j) {
-                    const float m = __shfl_sync(0xffffffffu, tj, j * (32 / NG));
-                    if (m > 0.f) {
-                        last_j = j; last_jb = runj;
-                        if (pj < 0 && runj + m > tgt) { pj = j; pj_before = runj; }
-                    }
-                    runj += m;
-                }
-                if (pj < 0) { pj = last_j; pj_before = last_jb; }
-                if (pj >= 0) {
-                    tgt -= pj_before;
-                    // level 3: the lane inside chunk pj
-                    float v = wg[0];
-#pragma unroll
-                    for (int j = 1; j < NG; ++j) v = (pj == j) ? wg[j] : v;
-                    const float incl = warp_scan_incl(v, lane);
-                    const unsigned hit3 = __ballot_sync(0xffffffffu, v > 0.f && incl > tgt);
-                    const unsigned pos3 = __ballot_sync(0xffffffffu, v > 0.f);
-                    const int l = hit3 ? __ffs(hit3) - 1 : (pos3 ? 31 - __clz(pos3) : -1);
-                    if (l >= 0 && lane == l) {
-                        // level 4: the element inside the group
-                        const float rem = tgt - (incl - v);
-                        float acc = 0.f;
-                        int pe = -1, last = -1;
-#pragma unroll
-                        for (int j = 0; j < NG; ++j) {
-                            if (j == pj) {
-#pragma unroll
-                                for (int h = 0; h < H; ++h) {
-                                    float w[4];
-                                    weights(j, h, w);
-#pragma unroll
-                                    for (int q4 = 0; q4 < 4; ++q4) {
-                                        if (w[q4] > 0.f) {
-                                            acc += w[q4];
-                                            last = 4 * h + q4;
-                                            if (pe < 0 && acc > rem) pe = 4 * h + q4;
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                        if (pe < 0) pe = last;
-                        P.node_bonus[node_idx] = v_begin + (g0 + pj * 32) * GV + pe;
-                    }
-                } else {
-                    // the run's exchanged mass was positive but its elements sum to nothing
-                    if (lane == 0) P.node_bonus[node_idx] = -1;
-                    status_bits |= MCSD_STATUS_NO_MASS;
-                }
-            }
-        }
-
-        // ---- per-node results
+        // ---- per-node results (the endpoint token is drawn by the walk kernel, and only
+        // for the node where a walk stops)
         if (crank == 0 && tid == 0) {
             P.node_accept[node_idx] = accepted;
-            if (accepted >= 0 || no_mass) P.node_bonus[node_idx] = -1;
             reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
                 make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
         }
         if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
         status_bits = __reduce_or_sync(0xffffffffu, status_bits);
         if (status_bits && lane == 0) atomicOr(P.status + b, status_bits);
-
-        b = b1; n = n1;
-        b1 = b2; n1 = n2;
-        advance(b2, n2);
+        next_item();
     }
 
     if (warp == 0) cp_async_wait_all();
@@ -1023,83 +932,238 @@ argmax_kernel(const __grid_constant__ ArgmaxParams P)
     }
 }
 
-// ------------------------------------------------------------------ walk + terminal residual
+// ------------------------------------------------------------------ walk + endpoint + residual
 struct WalkParams {
     const void *target;
     const void *draft;
     const int32_t *cand;
+    const float *unif;           // may be null at temperature 0
     const int32_t *node_accept;
-    const int32_t *node_bonus;
+    int32_t *node_bonus;         // T == 0: read (argmax of every node); T > 0: written in all-nodes mode
     const NodeStats *stats;
+    const float2 *leaf_part;
     int32_t *out_accept_len;
     int32_t *out_tokens;
     float *out_residual;  // may be null
+    int32_t *status;      // [B]
     long long ld_t, ld_d;
     int32_t n_nodes, n_internal, V, gamma;
-    float scale;  // log2(e)/T, or 0 for the argmax rule
+    int32_t n_entries;    // per-warp statistics entries a leaf row has (cluster size * warps per CTA)
+    int32_t all_nodes;    // 0: one CTA per sequence, walk then endpoint of the stopping node;
+                          // 1: one CTA per (sequence, node), endpoint of every node into node_bonus
+    int32_t vector_ok;    // logit rows are 16-byte aligned
+    float scale;          // log2(e)/T, or 0 for the argmax rule
 };
 
-// grid = (ceil(V / (kThreads*4)), B).  Every CTA of a row repeats the (at most gamma
-// hop) walk; the first one writes the tokens.
+constexpr int kWalkThreads = 1024;
+constexpr int kWalkWarps = kWalkThreads / 32;
+
+// One CTA per sequence.  Thread 0 follows the accepted children from the root (Section 3)
+// and writes the accepted tokens.  Then the whole CTA forms the distribution the endpoint
+// token of the stopping node is drawn from, w(x) = max(p(x) - c q(x), 0) / S with the
+// statistics the node kernel left (p alone for a leaf), writes it to out_residual, and
+// draws the token by inverse CDF in token order with that node's second uniform:
+// warp totals of contiguous runs -> the run holding the quantile -> that warp walks its
+// run again, 128 elements at a time.
 template <int DT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kWalkThreads)
 walk_kernel(const __grid_constant__ WalkParams P)
 {
     using E = Elem<DT>;
-    __shared__ int s_term;
-    const int b = blockIdx.y;
+    constexpr int GV = E::kVec;
+    __shared__ int s_term, s_len;
+    __shared__ float s_wtot[kWalkWarps];
+    __shared__ float s_leaf[2];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int b, n;
+    if (P.all_nodes) {
+        b = blockIdx.x / P.n_nodes;
+        n = blockIdx.x - b * P.n_nodes;
+    } else {
+        b = blockIdx.x;
+        n = 0;
+    }
     const long long nb = static_cast<long long>(b) * P.n_nodes;
-    if (threadIdx.x == 0) {
-        int n = 0, len = 0;
-        int32_t *tok = P.out_tokens + static_cast<long long>(b) * (P.gamma + 1);
-        const bool writer = blockIdx.x == 0;
-        // bounded by the depth of the tree even if node_accept were corrupt
-        for (int hop = 0; hop < P.gamma; ++hop) {
-            const int nx = P.node_accept[nb + n];
-            if (nx <= n || nx >= P.n_nodes) break;
-            n = nx;
-            if (writer) tok[len] = P.cand[nb + n];
-            ++len;
-        }
-        if (writer) {
-            tok[len] = P.node_bonus[nb + n];
+    int32_t *tok = P.out_tokens + static_cast<long long>(b) * (P.gamma + 1);
+    int len = 0;
+    if (!P.all_nodes) {
+        if (tid == 0) {
+            // bounded by the depth of the tree even if node_accept were corrupt
+            for (int hop = 0; hop < P.gamma; ++hop) {
+                const int nx = P.node_accept[nb + n];
+                if (nx <= n || nx >= P.n_nodes) break;
+                n = nx;
+                tok[len] = P.cand[nb + n];
+                ++len;
+            }
             for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
             P.out_accept_len[b] = len;
+            s_term = n;
+            s_len = len;
         }
-        s_term = n;
-    }
-    __syncthreads();
-    if (!P.out_residual) return;
-    const int n = s_term;
-    float *out = P.out_residual + static_cast<long long>(b) * P.V;
-    const int x0 = (blockIdx.x * kThreads + threadIdx.x) * 4;
-    if (x0 >= P.V) return;
-    if (P.scale == 0.f) {
-        const int a = P.node_bonus[nb + n];
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if (x0 + e < P.V) out[x0 + e] = (x0 + e == a) ? 1.f : 0.f;
+        __syncthreads();
+        n = s_term;
+        len = s_len;
+    } else if (P.node_accept[nb + n] >= 0) {
+        if (tid == 0) P.node_bonus[nb + n] = -1;  // a walk never stops here
         return;
     }
-    const NodeStats st = P.stats[nb + n];
+    float *out = P.out_residual ? P.out_residual + static_cast<long long>(b) * P.V : nullptr;
+
+    if (P.scale == 0.f) {
+        // argmax rule: the endpoint is the target argmax of the stopping node, the
+        // distribution is one-hot (all-nodes mode has nothing to add here)
+        const int a = P.node_bonus[nb + n];
+        if (tid == 0 && !P.all_nodes) tok[len] = a;
+        if (out)
+            for (int x = tid; x < P.V; x += kWalkThreads) out[x] = (x == a) ? 1.f : 0.f;
+        return;
+    }
+
+    // ---- statistics of the stopping node
     const bool internal = n < P.n_internal;
-    const unsigned char *t_row = reinterpret_cast<const unsigned char *>(P.target) +
-        (nb + n) * P.ld_t * E::kBytes;
+    float r_t, z_t, r_d = 0.f, z_d = 0.f, c = 0.f, S = 1.f;
+    if (internal) {
+        const NodeStats st = P.stats[nb + n];
+        r_t = st.r_t; r_d = st.r_d; z_t = st.z_t; z_d = st.z_d; c = st.c; S = st.s;
+    } else {
+        if (warp == 0) {
+            float2 e = make_float2(-INFINITY, 0.f);
+            if (lane < P.n_entries)
+                e = P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * 32 + lane];
+            const float R = warp_max(e.x);
+            const float Z = warp_sum(e.y * exp2i(e.x - R));
+            if (lane == 0) { s_leaf[0] = R; s_leaf[1] = Z; }
+        }
+        __syncthreads();
+        r_t = s_leaf[0]; z_t = s_leaf[1];
+    }
+    const bool t_ok = z_t > 0.f && z_t < INFINITY;
+    const float r_t0 = r_t == -INFINITY ? 0.f : r_t, r_d0 = r_d == -INFINITY ? 0.f : r_d;
+    const float inv_zt = t_ok ? 1.f / z_t : 0.f;
+    const float cq = (internal && z_d > 0.f && z_d < INFINITY) ? c / z_d : 0.f;
+    const float inv_s = S > 0.f ? 1.f / S : 0.f;
+    const unsigned char *t_row = reinterpret_cast<const unsigned char *>(P.target) + (nb + n) * P.ld_t * E::kBytes;
     const unsigned char *d_row = reinterpret_cast<const unsigned char *>(P.draft) +
         (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes;
-    const float r_t = st.r_t == -INFINITY ? 0.f : st.r_t;
-    const float r_d = st.r_d == -INFINITY ? 0.f : st.r_d;
-    const float inv_zt = st.z_t > 0.f ? 1.f / st.z_t : 0.f;
-    const float cq = (internal && st.z_d > 0.f) ? st.c / st.z_d : 0.f;
-    const float inv_s = st.s > 0.f ? 1.f / st.s : 0.f;
+
+    // weights of the GV elements starting at x0 (0 past the end of the vocabulary)
+    auto weights = [&](int x0, float *w) {
+        float t[GV], d[GV];
+        if (P.vector_ok && x0 + GV <= P.V) {
+            E::unpack(__ldg(reinterpret_cast<const uint4 *>(t_row + static_cast<size_t>(x0) * E::kBytes)), t);
+            if (cq > 0.f) E::unpack(__ldg(reinterpret_cast<const uint4 *>(d_row + static_cast<size_t>(x0) * E::kBytes)), d);
+        } else {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int x = x0 + e;
-        if (x < P.V) {
-            float w = ex2f(fmaf(E::load(t_row, x), P.scale, -r_t)) * inv_zt;
-            if (internal && cq > 0.f) w = fmaxf(fmaf(-cq, ex2f(fmaf(E::load(d_row, x), P.scale, -r_d)), w), 0.f);
-            out[x] = w * inv_s;
+            for (int e = 0; e < GV; ++e) {
+                t[e] = x0 + e < P.V ? E::load(t_row, x0 + e) : -INFINITY;
+                d[e] = (cq > 0.f && x0 + e < P.V) ? E::load(d_row, x0 + e) : -INFINITY;
+            }
         }
+#pragma unroll
+        for (int e = 0; e < GV; ++e) {
+            float v = ex2f(fmaf(t[e], P.scale, -r_t0)) * inv_zt;
+            if (cq > 0.f) v = fmaxf(fmaf(-cq, ex2f(fmaf(d[e], P.scale, -r_d0)), v), 0.f);
+            w[e] = v;
+        }
+    };
+
+    // contiguous runs: warp w owns [w * run, (w + 1) * run), walked 32 * GV elements at a time
+    constexpr int kStep = 32 * GV;
+    const int run = ((P.V + kWalkWarps - 1) / kWalkWarps + kStep - 1) / kStep * kStep;
+    const int x_lo = warp * run;
+    int x_hi = x_lo + run;
+    x_hi = x_hi > P.V ? P.V : x_hi;
+
+    // pass 1: the distribution itself and the mass of every run
+    float mass = 0.f;
+    for (int x0 = x_lo + lane * GV; x0 < x_hi; x0 += kStep) {
+        float w[GV];
+        weights(x0, w);
+#pragma unroll
+        for (int e = 0; e < GV; ++e) {
+            mass += w[e];
+            if (out && x0 + e < P.V) out[x0 + e] = w[e] * inv_s;
+        }
+    }
+    mass = warp_sum(mass);
+    if (lane == 0) s_wtot[warp] = mass;
+    __syncthreads();
+
+    // the run that holds the quantile (every warp finds the same one)
+    const float u_end = P.unif[2 * (nb + n) + 1];
+    const float m = s_wtot[lane];
+    const float total = warp_sum(m);
+    const float target = u_end * total;
+    const float inc = warp_scan_incl(m, lane);
+    const unsigned hit = __ballot_sync(0xffffffffu, m > 0.f && inc > target);
+    const unsigned pos = __ballot_sync(0xffffffffu, m > 0.f);
+    // (rounding may push the quantile past the end: clamp to the last run with mass)
+    const int pick = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
+    int32_t *dst = P.all_nodes ? P.node_bonus + nb + n : tok + len;
+    if (pick < 0 || !(total > 0.f)) {
+        if (tid == 0) {
+            *dst = -1;
+            atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
+        }
+        return;
+    }
+    if (warp != pick) return;
+
+    // pass 2 (one warp): 32 * GV elements at a time until the quantile is passed
+    float tgt = target - __shfl_sync(0xffffffffu, inc - m, pick);
+    int found = -1, last_x0 = -1;     // element index; start of the last step that had mass
+    float runsum = 0.f;
+    for (int x0 = x_lo; x0 < x_hi && found < 0; x0 += kStep) {
+        float w[GV];
+        weights(x0 + lane * GV, w);
+        float g = 0.f;
+#pragma unroll
+        for (int e = 0; e < GV; ++e) g += w[e];
+        const float gi = warp_scan_incl(g, lane);
+        const float step_total = __shfl_sync(0xffffffffu, gi, 31);
+        if (step_total > 0.f) {
+            last_x0 = x0;
+            if (runsum + step_total > tgt) {
+                const float t2 = tgt - runsum;
+                const unsigned h2 = __ballot_sync(0xffffffffu, g > 0.f && gi > t2);
+                const unsigned p2 = __ballot_sync(0xffffffffu, g > 0.f);
+                const int l = h2 ? __ffs(h2) - 1 : 31 - __clz(p2);
+                int pe = -1, last = -1;
+                if (lane == l) {
+                    const float rem = t2 - (gi - g);
+                    float acc = 0.f;
+#pragma unroll
+                    for (int e = 0; e < GV; ++e) {
+                        if (w[e] > 0.f) {
+                            acc += w[e];
+                            last = e;
+                            if (pe < 0 && acc > rem) pe = e;
+                        }
+                    }
+                    if (pe < 0) pe = last;
+                }
+                found = __shfl_sync(0xffffffffu, x0 + lane * GV + pe, l);
+            }
+        }
+        runsum += step_total;
+    }
+    if (found < 0 && last_x0 >= 0) {
+        // rounding: the quantile lies past the run's own sum; take its last element with mass
+        float w[GV];
+        weights(last_x0 + lane * GV, w);
+        int last = -1;
+#pragma unroll
+        for (int e = 0; e < GV; ++e) if (w[e] > 0.f) last = e;
+        const unsigned p2 = __ballot_sync(0xffffffffu, last >= 0);
+        if (p2) {
+            const int l = 31 - __clz(p2);
+            found = __shfl_sync(0xffffffffu, last_x0 + lane * GV + last, l);
+        }
+    }
+    if (lane == 0) {
+        *dst = found;
+        if (found < 0) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
     }
 }
 

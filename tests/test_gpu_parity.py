@@ -168,7 +168,7 @@ def test_staged_entry_points_equal_the_fused_call():
     ref = (to_np(out.accept_len).copy(), to_np(out.tokens).copy(), to_np(out.residual).copy())
     v2 = binding.Verifier(w.batch, inp.parent, w.vocab, torch.bfloat16, "cuda")
     v2.mcsd_verify_nodes(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
-    o2 = v2.mcsd_verify_walk(inp.target, inp.draft, inp.cand, w.temperature)
+    o2 = v2.mcsd_verify_walk(inp.target, inp.draft, inp.cand, inp.unif, w.temperature)
     torch.cuda.synchronize()
     assert np.array_equal(ref[0], to_np(o2.accept_len)) and np.array_equal(ref[1], to_np(o2.tokens))
     assert np.array_equal(ref[2], to_np(o2.residual))
