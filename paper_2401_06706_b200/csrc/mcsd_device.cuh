@@ -371,8 +371,10 @@ node_kernel(const __grid_constant__ NodeParams P)
     __shared__ double s_px[NW][MCSD_MAX_CHILDREN], s_qx[NW][MCSD_MAX_CHILDREN];
     __shared__ CandRing ring;
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t crank = cluster_ctarank(), csize = cluster_nctarank();
+    const int tid = threadIdx.x, lane = tid & 31;
+    // (broadcast from lane 0 so that the compiler knows the warp index is warp-uniform)
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+    const uint32_t crank = __clusterRelativeBlockRank(), csize = __clusterSizeInBlocks();
     const int cluster_id = blockIdx.x / csize;
     const int n_entries = static_cast<int>(csize) * NW;  // values per exchange round (<= 32)
     const float scale = P.scale;
@@ -702,11 +704,11 @@ node_kernel(const __grid_constant__ NodeParams P)
         look_ahead();  // in the shadow of the exchange
         // While the round is in flight: the candidates' own logits as 2^int * frac in double
         // (lane i = candidate i; every warp keeps its own copy so that no CTA barrier is needed).
-        double frac_t = 0.0, frac_d = 0.0;
         int int_t = 0, int_d = 0;
         bool cand_ok = false;
         int my_tok = -1;
         if (lane < k) {
+            double frac_t = 0.0, frac_d = 0.0;
             my_tok = ring.tok[s3][lane];
             cand_ok = my_tok >= 0 && my_tok < P.V;
             if (cand_ok) {
@@ -720,6 +722,8 @@ node_kernel(const __grid_constant__ NodeParams P)
                 frac_t = (at == at && fabs(at) < 1e300) ? exp2(at - it_) : (at > 0 ? INFINITY : 0.0);
                 frac_d = (ad == ad && fabs(ad) < 1e300) ? exp2(ad - id_) : (ad > 0 ? INFINITY : 0.0);
             }
+            s_px[warp][lane] = frac_t;  // parked here until the exchange has completed
+            s_qx[warp][lane] = frac_d;
         }
         float4 ent = exchange_wait(make_float4(-INFINITY, 0.f, -INFINITY, 0.f));
         // row references ceil(row maximum * scale) and normalisers, the same bits in every thread
@@ -744,8 +748,8 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (lane < k) {
             double px = 0.0, qx = 0.0;
             if (cand_ok && t_ok && d_ok) {
-                px = frac_t * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
-                qx = frac_d * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
+                px = s_px[warp][lane] * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
+                qx = s_qx[warp][lane] * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
             }
             s_px[warp][lane] = px;
             s_qx[warp][lane] = qx;
