@@ -76,6 +76,10 @@ extern "C" {
 #define MCSD_ERR_WORKSPACE (-8)   /* workspace missing, misaligned or too small       */
 #define MCSD_ERR_CUDA (-9)        /* a CUDA runtime call or kernel launch failed      */
 #define MCSD_ERR_UNSUPPORTED (-10)/* beyond MCSD_MAX_*                                */
+#define MCSD_ERR_STATIC_LIMIT (-11) /* mcsd_verify_static: scratch need > built-in array */
+
+/* Bytes of the scratch array built into the library for mcsd_verify_static. */
+#define MCSD_STATIC_WORKSPACE_BYTES (4u << 20)
 
 /* bits of out_status[b] */
 #define MCSD_STATUS_DEGENERATE 1 /* residual mass was 0 after a rejection; residual kept */
@@ -177,6 +181,40 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                      float temperature, int replacement_mode, int32_t *out_accept_len,
                      int32_t *out_tokens, float *out_residual, int32_t *out_status);
+
+/*
+ * mcsd_verify for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of mcsd_verify, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a serving
+ * loop that promised its memory pool a fixed footprint, in a plugin whose host
+ * owns every allocation, or late in a process whose device memory is already
+ * fully handed out - and that therefore has no buffer to put into
+ * desc->workspace.  Here the scratch memory (per-node accept decisions, softmax
+ * statistics, per-sequence status words) lives in an array of
+ * MCSD_STATIC_WORKSPACE_BYTES bytes compiled into the library; every GPU that
+ * loads the library carries that array until the process exits.  Inputs and
+ * outputs are still the caller's buffers; desc->workspace and
+ * desc->workspace_bytes are ignored.  Everything else is as in mcsd_verify.
+ *
+ * Limits and rules
+ *   - If mcsd_workspace_bytes(desc) exceeds MCSD_STATIC_WORKSPACE_BYTES the call
+ *     returns MCSD_ERR_STATIC_LIMIT and enqueues nothing (roughly: batch * nodes
+ *     per tree up to some tens of thousands; use mcsd_verify beyond that).
+ *   - The first call on each device looks up the array's device address (once,
+ *     with that device current).  Make that first call before any stream capture
+ *     begins.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called.
+ *   - All calls on one device share the one array, and it still holds what the
+ *     previous call left; the call clears the part that has to start at zero (the
+ *     status words) itself.  Two calls whose kernels can overlap on the GPU
+ *     (different streams, no dependency between them) race on the array: order
+ *     them.
+ */
+int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                       const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                       float temperature, int replacement_mode, int32_t *out_accept_len,
+                       int32_t *out_tokens, float *out_residual);
 
 /* Bytes of device workspace mcsd_verify needs for this descriptor (batch and
  * n_nodes are read); 0 if the descriptor is NULL or its shape is invalid. */

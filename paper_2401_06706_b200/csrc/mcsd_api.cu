@@ -411,6 +411,7 @@ const char *mcsd_status_string(int code)
     case MCSD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case MCSD_ERR_CUDA: return "a CUDA runtime call or kernel launch failed";
     case MCSD_ERR_UNSUPPORTED: return "size beyond the library limits";
+    case MCSD_ERR_STATIC_LIMIT: return "scratch need exceeds the built-in array of mcsd_verify_static; use mcsd_verify";
     default: return "unknown code";
     }
 }
@@ -481,6 +482,53 @@ int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *dr
     if (rc != MCSD_OK) return rc;
     return launch_walk(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, out_accept_len,
                        out_tokens, out_residual);
+}
+
+// ---- mcsd_verify_static: the scratch memory is an array built into the library --------
+// In host code the name below is only a handle for the runtime; the address kernels can
+// use comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_static_workspace[MCSD_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices] = {};
+
+// Device address of the built-in array on the current device, or nullptr on failure.
+void *static_workspace()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        g_static_ptr[dev] = ptr;
+    }
+    return g_static_ptr[dev];
+}
+}  // namespace
+
+int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                       const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                       float temperature, int replacement_mode, int32_t *out_accept_len,
+                       int32_t *out_tokens, float *out_residual)
+{
+    const int rc = check_desc(desc);
+    if (rc != MCSD_OK) return rc;
+    if (mcsd_workspace_bytes(desc) > MCSD_STATIC_WORKSPACE_BYTES) return MCSD_ERR_STATIC_LIMIT;
+    void *ws = static_workspace();
+    if (!ws) return MCSD_ERR_CUDA;
+    mcsd_desc with_scratch = *desc;
+    with_scratch.workspace = ws;
+    with_scratch.workspace_bytes = MCSD_STATIC_WORKSPACE_BYTES;
+    // the status words are cleared by the node stage itself; everything else in the
+    // array is written before it is read
+    return mcsd_verify(&with_scratch, target_logits, draft_logits, tree_parent, cand_tokens, uniforms,
+                       temperature, replacement_mode, out_accept_len, out_tokens, out_residual);
 }
 
 int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
