@@ -152,21 +152,22 @@ int choose_config(int vocab, int dtype, bool aligned, NodeConfig *cfg)
     int best_c = 0, best_e = 0;
     long long best_cap = -1;
     const int force_c = env_int("MCSD_CLUSTER", 0), force_e = env_int("MCSD_EPT", 0);
-    for (int c = 1; c <= kMaxCluster; c *= 2) {
+    for (int c = 1; c <= kMaxCluster; ++c) {
         if (force_c && c != force_c) continue;
         for (int ei = 2; ei >= 0; --ei) {
             const int e = kEptChoices[ei];
             if (force_e && e != force_e) continue;
-            const long long slice = align_up((vocab + c - 1) / c, vec);
-            if (slice > static_cast<long long>(kNodeThreads) * e) continue;
-            const long long cap = static_cast<long long>(c) * e;
+            const long long cap = static_cast<long long>(c) * kNodeThreads * e;
+            if (cap < vocab) continue;
             if (best_cap < 0 || cap < best_cap) { best_cap = cap; best_c = c; best_e = e; }
         }
     }
     if (best_cap < 0) return MCSD_ERR_UNSUPPORTED;
     cfg->cluster = best_c;
     cfg->ept = best_e;
-    cfg->slice = static_cast<int>(align_up((vocab + best_c - 1) / best_c, vec));
+    // every CTA but the last owns a full slice, so that only the last one has ragged warps
+    cfg->slice = kNodeThreads * best_e;
+    (void)vec;
     cfg->direct = !aligned || env_int("MCSD_DIRECT", 0) != 0;
     return MCSD_OK;
 }
@@ -323,8 +324,9 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     p.step_b = static_cast<int32_t>(n_clusters / d->n_nodes);
     p.step_n = static_cast<int32_t>(n_clusters % d->n_nodes);
     p.mode = mode;
-    p.scale_d = 1.4426950408889634 / static_cast<double>(T);
-    p.scale = static_cast<float>(p.scale_d);
+    const double scale_d = 1.4426950408889634 / static_cast<double>(T);
+    p.scale = static_cast<float>(scale_d);
+    p.scale_lo = static_cast<float>(scale_d - static_cast<double>(p.scale));
     std::memcpy(p.child_first, c.plan.child_first, sizeof(p.child_first));
     std::memcpy(p.child_count, c.plan.child_count, sizeof(p.child_count));
 

@@ -72,13 +72,21 @@ struct NodeParams {
     int32_t n_items; // B * n_nodes
     int32_t step_b, step_n;  // quotient and remainder of (clusters in the grid) / n_nodes
     int32_t mode;
-    float scale;     // log2(e) / T
-    double scale_d;  // the same in double, for the candidates' own probabilities
+    float scale;     // log2(e) / T rounded to float ...
+    float scale_lo;  // ... and what the rounding dropped (for the candidates' own probabilities)
     uint16_t child_first[MCSD_MAX_NODES];
     uint8_t child_count[MCSD_MAX_NODES];
 };
 
 // ------------------------------------------------------------------ element types
+// Three-input maximum (a NaN operand is ignored, as with fmaxf).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d;
+}
+
+// Per element type: unpacking of one 16-byte vector, scalar access, and a running maximum
+// over whole vectors that stays in the packed format for 2-byte types (two elements per
+// instruction) and is turned into a float once at the end.
 template <int DT> struct Elem;
 template <> struct Elem<MCSD_DTYPE_F32> {
     static constexpr int kBytes = 4, kVec = 4;
@@ -91,6 +99,13 @@ template <> struct Elem<MCSD_DTYPE_F32> {
     }
     // value of element i given the aligned 32-bit word that contains it
     static __device__ __forceinline__ float from_word(uint32_t w, long long) { return __uint_as_float(w); }
+    typedef float2 MaxAcc;
+    static __device__ __forceinline__ MaxAcc max_init() { return make_float2(-INFINITY, -INFINITY); }
+    static __device__ __forceinline__ void max_step(MaxAcc &a, const uint4 &r) {
+        a.x = max3(a.x, __uint_as_float(r.x), __uint_as_float(r.y));
+        a.y = max3(a.y, __uint_as_float(r.z), __uint_as_float(r.w));
+    }
+    static __device__ __forceinline__ float max_final(const MaxAcc &a) { return fmaxf(a.x, a.y); }
 };
 template <> struct Elem<MCSD_DTYPE_BF16> {
     static constexpr int kBytes = 2, kVec = 8;
@@ -109,6 +124,17 @@ template <> struct Elem<MCSD_DTYPE_BF16> {
     }
     // 16-bit pattern of a value that this type represents exactly
     static __device__ __forceinline__ uint32_t to_bits(float f) { return __float_as_uint(f) >> 16; }
+    typedef uint32_t MaxAcc;
+    static __device__ __forceinline__ uint32_t mx(uint32_t a, uint32_t b) {
+        const __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&a),
+                                         *reinterpret_cast<const __nv_bfloat162 *>(&b));
+        return *reinterpret_cast<const uint32_t *>(&r);
+    }
+    static __device__ __forceinline__ MaxAcc max_init() { return 0xff80ff80u; }  // (-inf, -inf)
+    static __device__ __forceinline__ void max_step(MaxAcc &a, const uint4 &r) {
+        a = mx(a, mx(mx(r.x, r.y), mx(r.z, r.w)));
+    }
+    static __device__ __forceinline__ float max_final(const MaxAcc &a) { return fmaxf(from_word(a, 0), from_word(a, 1)); }
 };
 template <> struct Elem<MCSD_DTYPE_F16> {
     static constexpr int kBytes = 2, kVec = 8;
@@ -128,6 +154,16 @@ template <> struct Elem<MCSD_DTYPE_F16> {
         return __half2float(__ushort_as_half(h));
     }
     static __device__ __forceinline__ uint32_t to_bits(float f) { return __half_as_ushort(__float2half_rn(f)); }
+    typedef uint32_t MaxAcc;
+    static __device__ __forceinline__ uint32_t mx(uint32_t a, uint32_t b) {
+        const __half2 r = __hmax2(*reinterpret_cast<const __half2 *>(&a), *reinterpret_cast<const __half2 *>(&b));
+        return *reinterpret_cast<const uint32_t *>(&r);
+    }
+    static __device__ __forceinline__ MaxAcc max_init() { return 0xfc00fc00u; }  // (-inf, -inf)
+    static __device__ __forceinline__ void max_step(MaxAcc &a, const uint4 &r) {
+        a = mx(a, mx(mx(r.x, r.y), mx(r.z, r.w)));
+    }
+    static __device__ __forceinline__ float max_final(const MaxAcc &a) { return fmaxf(from_word(a, 0), from_word(a, 1)); }
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -226,10 +262,6 @@ typedef float2 f32x2;
 __device__ __forceinline__ f32x2 pack2(float lo, float hi) { return make_float2(lo, hi); }
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { return __ffma2_rn(a, b, c); }
 __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { return __fadd2_rn(a, b); }
-// Three-input maximum (a NaN operand is ignored, as with fmaxf).
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d;
-}
 // Warp-wide maximum in one instruction (NaN inputs are ignored).
 __device__ __forceinline__ float warp_max(float v) {
     float d; asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(d) : "f"(v)); return d;
@@ -251,13 +283,38 @@ __device__ __forceinline__ float warp_scan_incl(float v, int lane) {
 // d < -126 (also for d = -inf), clamped to 2^127 above.
 __device__ __forceinline__ float exp2i(float d) {
     d = fminf(fmaxf(d, -127.f), 127.f);
-    return __int_as_float((static_cast<int>(d) + 127) << 23);
+    // adding 1.5 * 2^23 leaves the integer in the low mantissa bits (no conversion instruction)
+    const int i = __float_as_int(d + 12582912.f) - 0x4b400000;
+    return __int_as_float((i + 127) << 23);
 }
 // The same in double for an integer e: 0 below 2^-1000.
 __device__ __forceinline__ double exp2i_d(int e) {
     if (e < -1000) return 0.0;
     e = e > 1000 ? 1000 : e;
     return __hiloint2double((e + 1023) << 20, 0);
+}
+// 2^(l * (scale + scale_lo)) as 2^ip * (return value), ip an integer and the return value
+// in [2^-0.51, 2^0.51], to about 1e-7 relative however large the exponent is: the
+// product is formed exactly as a sum of two floats, its integer part goes to ip and only
+// the fraction is exponentiated.  Infinite or NaN products give 0 (or +inf) with ip = 0.
+__device__ __forceinline__ float split_exp2(float l, float scale, float scale_lo, int &ip) {
+    const float ph = l * scale;
+    ip = 0;
+    if (!(fabsf(ph) < 1.0e9f)) return ph > 0.f ? INFINITY : 0.f;
+    const float pe = fmaf(l, scale, -ph);      // exact error of the rounded product
+    const float pl = fmaf(l, scale_lo, pe);    // plus the part of the scale that float drops
+    const float ipf = rintf(ph);
+    const float f = (ph - ipf) + pl;           // |f| <= 0.5 + tiny; the subtraction is exact
+    ip = static_cast<int>(ipf);
+    // Taylor series of exp(f ln 2), |f ln 2| <= 0.36: the degree-7 remainder is below 6e-9
+    float y = 1.5252733804059841e-05f;
+    y = fmaf(y, f, 1.5403530393381608e-04f);
+    y = fmaf(y, f, 1.3333558146428443e-03f);
+    y = fmaf(y, f, 9.6181291076284772e-03f);
+    y = fmaf(y, f, 5.5504108664821580e-02f);
+    y = fmaf(y, f, 2.4022650695910071e-01f);
+    y = fmaf(y, f, 6.9314718055994531e-01f);
+    return fmaf(y, f, 1.f);
 }
 // Integer reference of a set whose largest scaled logit is m (log2 units); -inf for
 // an empty set.  NaN-free inputs give ceil(m), so that every exponent is <= 0.
@@ -661,18 +718,29 @@ node_kernel(const __grid_constant__ NodeParams P)
                     }
                 }
             };
-            float m0 = -INFINITY, m1 = -INFINITY;
+            float md;
+            if constexpr (kRawZone || E::kBytes == 4) {
+                // maximum over the raw vectors as they lie in shared memory (packed for 2-byte types)
+                typename E::MaxAcc acc = E::max_init();
 #pragma unroll
-            for (int j = 0; j < NG; ++j) {
-                float r[GV];
-                read_q_raw(j, r);
+                for (int j = 0; j < NG; ++j)
+                    E::max_step(acc, kRawZone ? qraw[g0 + j * 32] : *reinterpret_cast<const uint4 *>(&qbuf[qslot(j, 0)]));
+                md = E::max_final(acc);
+            } else {
+                float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-                for (int e = 0; e < GV; e += 4) {
-                    m0 = max3(m0, r[e], r[e + 1]);
-                    m1 = max3(m1, r[e + 2], r[e + 3]);
+                for (int j = 0; j < NG; ++j) {
+                    float r[GV];
+                    read_q_raw(j, r);
+#pragma unroll
+                    for (int e = 0; e < GV; e += 4) {
+                        m0 = max3(m0, r[e], r[e + 1]);
+                        m1 = max3(m1, r[e + 2], r[e + 3]);
+                    }
                 }
+                md = fmaxf(m0, m1);
             }
-            rd = int_ref(fmaxf(m0, m1) * scale);
+            rd = int_ref(md * scale);
             const float rd0 = (rd == -INFINITY) ? 0.f : rd;
             const f32x2 scale2 = pack2(scale, scale), nref2 = pack2(-rd0, -rd0);
             f32x2 z0 = pack2(0.f, 0.f), z1 = z0;
@@ -702,28 +770,23 @@ node_kernel(const __grid_constant__ NodeParams P)
             exchange_send(make_float4(Rt, st, Rd, sd));  // per warp: (ref_t, z_t, ref_d, z_d)
         }
         look_ahead();  // in the shadow of the exchange
-        // While the round is in flight: the candidates' own logits as 2^int * frac in double
-        // (lane i = candidate i; every warp keeps its own copy so that no CTA barrier is needed).
+        // While the round is in flight: 2^(scaled logit) of the candidates' own logits as
+        // 2^int * frac (lane i = candidate i; every warp keeps its own copy so that no CTA
+        // barrier is needed).
         int int_t = 0, int_d = 0;
         bool cand_ok = false;
         int my_tok = -1;
         if (lane < k) {
-            double frac_t = 0.0, frac_d = 0.0;
+            float frac_t = 0.f, frac_d = 0.f;
             my_tok = ring.tok[s3][lane];
             cand_ok = my_tok >= 0 && my_tok < P.V;
             if (cand_ok) {
                 const uint32_t wt = ring.tl[s2][lane], wd = ring.dl[s2][lane];
-                const double at = static_cast<double>(DIRECT ? __uint_as_float(wt) : E::from_word(wt, my_tok)) * P.scale_d;
-                const double ad = static_cast<double>(DIRECT ? __uint_as_float(wd) : E::from_word(wd, my_tok)) * P.scale_d;
-                const double it_ = rint(at), id_ = rint(ad);
-                // |scaled logit| beyond 2^30 cannot be told from +-inf here
-                int_t = static_cast<int>(fmin(fmax(it_, -1073741824.0), 1073741824.0));
-                int_d = static_cast<int>(fmin(fmax(id_, -1073741824.0), 1073741824.0));
-                frac_t = (at == at && fabs(at) < 1e300) ? exp2(at - it_) : (at > 0 ? INFINITY : 0.0);
-                frac_d = (ad == ad && fabs(ad) < 1e300) ? exp2(ad - id_) : (ad > 0 ? INFINITY : 0.0);
+                frac_t = split_exp2(DIRECT ? __uint_as_float(wt) : E::from_word(wt, my_tok), scale, P.scale_lo, int_t);
+                frac_d = split_exp2(DIRECT ? __uint_as_float(wd) : E::from_word(wd, my_tok), scale, P.scale_lo, int_d);
             }
-            s_px[warp][lane] = frac_t;  // parked here until the exchange has completed
-            s_qx[warp][lane] = frac_d;
+            s_px[warp][lane] = static_cast<double>(frac_t);  // parked here until the exchange has completed
+            s_qx[warp][lane] = static_cast<double>(frac_d);
         }
         float4 ent = exchange_wait(make_float4(-INFINITY, 0.f, -INFINITY, 0.f));
         // row references ceil(row maximum * scale) and normalisers, the same bits in every thread
