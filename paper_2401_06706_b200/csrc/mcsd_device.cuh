@@ -181,12 +181,6 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
 __device__ __forceinline__ uint32_t cluster_nctarank() {
     uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r;
 }
-__device__ __forceinline__ void cluster_arrive_release() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void cluster_wait_acquire() {
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -251,9 +245,12 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_f4(uint32_t addr, float4 v) {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
-                 ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+// Asynchronous 16-byte store into a CTA of the cluster that reports its bytes to an
+// mbarrier of that CTA: the data is visible to whoever sees the barrier's phase complete,
+// no fence on either side.
+__device__ __forceinline__ void st_async_f4(uint32_t addr, float4 v, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar) : "memory");
 }
 
 // Packed pairs of floats: sm_100 executes fma and add on both halves of an aligned
@@ -323,14 +320,18 @@ __device__ __forceinline__ float int_ref(float m_scaled) {
 }
 
 // Shared state of the cluster-wide exchange: two buffers of one float4 per (cluster
-// rank, warp).  In round r every warp of every CTA stores its value into buffer r&1 of
-// every CTA of the cluster (its own included) and then all threads meet at the
-// hardware cluster barrier; after it every CTA holds all values of the round, in
-// vocabulary order (rank-major, then warp).  A buffer is rewritten two rounds later,
-// which a peer can only reach after this CTA's threads have arrived at the barrier in
-// between, i.e. after they finished reading (release/acquire at cluster scope).
+// rank, warp) and one mbarrier per buffer.  In round r every warp of every CTA sends its
+// value into buffer r&1 of every CTA of the cluster (its own included) with asynchronous
+// stores that report their bytes to that CTA's barrier; the CTA armed the barrier with
+// the byte count of a whole round, so when its phase completes all values of the round
+// are there, in vocabulary order (rank-major, then warp).  One warp per CTA watches the
+// barrier (bounded, with back-off), the others wait for it at a CTA barrier, so nobody
+// spins on the issue slots the working CTAs need.  A buffer is rewritten two rounds
+// later, which a peer can only reach after all warps of this CTA have sent the round in
+// between, i.e. after they finished reading.
 struct Exchange {
     float4 slot[2][kMaxCluster * 4];
+    unsigned long long bar[2];
 };
 
 // Candidate data of the next items, fetched ahead of use by warp 0 so that no DRAM
@@ -406,7 +407,7 @@ constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
 //
 // Every decision of the rejection loop is taken by every warp of the cluster from
 // bit-identical inputs, so all CTAs of a cluster execute the same number of exchange
-// rounds (the cluster barrier counts on it).
+// rounds (the byte counts the exchange barriers are armed with rely on it).
 template <int DT, int EPT, bool DIRECT>
 __global__ void __launch_bounds__(kNodeThreads, node_min_blocks(EPT))
 node_kernel(const __grid_constant__ NodeParams P)
@@ -436,6 +437,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     const int n_entries = static_cast<int>(csize) * NW;  // values per exchange round (<= 32)
     const float scale = P.scale;
     const uint32_t full_addr = smem_u32(&full_bar);
+    const uint32_t xbar_addr[2] = {smem_u32(&xch.bar[0]), smem_u32(&xch.bar[1])};
 
     // this CTA's slice of the vocabulary and this warp's run of it
     const int v_begin = static_cast<int>(crank) * P.slice;
@@ -456,10 +458,12 @@ node_kernel(const __grid_constant__ NodeParams P)
 
     if (tid == 0) {
         mbar_init(full_addr, 1);
+        mbar_init(xbar_addr[0], 1);
+        mbar_init(xbar_addr[1], 1);
         fence_mbar_init();
     }
     __syncthreads();
-    cluster_sync_all();  // every CTA of the cluster is running before anyone stores into a peer
+    cluster_sync_all();  // every CTA's barriers exist before anyone stores into a peer
 
     uint32_t full_parity = 0, round = 0;
     int poisoned = 0;
@@ -472,20 +476,24 @@ node_kernel(const __grid_constant__ NodeParams P)
             ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + v_begin) * E::kBytes;
     };
 
-    // One exchange round.  send: `mine` is this warp's value (the same in all lanes); the
-    // threads then arrive at the cluster barrier, and whatever is placed between send and
-    // wait overlaps the barrier's latency.  wait: returns entry `lane` of the round
-    // (rank-major, then warp), the given identity for lanes beyond the entry count.
+    // One exchange round.  send: `mine` is this warp's value (the same in all lanes);
+    // whatever is placed between send and wait overlaps the round's latency.  wait:
+    // returns entry `lane` of the round (rank-major, then warp), the given identity for
+    // lanes beyond the entry count.
     auto exchange_send = [&](float4 mine) {
+        const uint32_t s = round & 1u;
+        if (tid == 0) mbar_arrive_expect_tx(xbar_addr[s], static_cast<uint32_t>(n_entries) * 16u);
         if (lane < static_cast<int>(csize)) {
-            const uint32_t dst = map_to_rank(smem_u32(&xch.slot[round & 1u][crank * NW + warp]), lane);
-            st_cluster_f4(dst, mine);
+            const uint32_t dst = map_to_rank(smem_u32(&xch.slot[s][crank * NW + warp]), lane);
+            st_async_f4(dst, mine, map_to_rank(xbar_addr[s], lane));
         }
-        cluster_arrive_release();
     };
     auto exchange_wait = [&](float4 identity) -> float4 {
-        cluster_wait_acquire();
-        const float4 e = lane < n_entries ? xch.slot[round & 1u][lane] : identity;
+        const uint32_t s = round & 1u;
+        // once a wait has expired the results are void and later rounds do not wait again
+        if (warp == 0 && !poisoned && !mbar_wait(xbar_addr[s], (round >> 1) & 1u)) poisoned = 1;
+        __syncthreads();
+        const float4 e = lane < n_entries ? xch.slot[s][lane] : identity;
         ++round;
         return e;
     };
