@@ -139,6 +139,20 @@ def shard_for_rank(w: synth.Workload, rank: int, world: int) -> synth.Workload:
     return replace(w, seed=w.seed + 7919 * rank) if world > 1 else w
 
 
+def max_over_ranks(dist, value: float, device) -> float:
+    """Largest value any rank holds (elapsed times are reported as the slowest rank's)."""
+    if dist is None:
+        return float(value)
+    tt = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_value(world: int, nodes_per_rank_step: int, ms_per_step: float) -> float:
+    """Verified tree nodes per second of the whole job: every rank verifies its own batch."""
+    return world * nodes_per_rank_step / (ms_per_step * 1e-3)
+
+
 def oracle_sample(inp: synth.Inputs, n_seq: int):
     """Times the CPU oracle, as it stands, on the first n_seq sequences."""
     import oracle
@@ -272,15 +286,12 @@ def run_cuda(args):
     t_host1 = time.time()
     elapsed_ms = start.elapsed_time(stop)
     node_ms = [a.elapsed_time(b) for a, b in node_events]
-    if dist:
-        tt = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt.item())
+    elapsed_ms = max_over_ranks(dist, elapsed_ms, dev)
     clocks = sampler.stop(t_host0, t_host1) if sampler else None
     status_bits = int(ver.status.max().item()) if w.batch else 0
 
     ms_per_step = elapsed_ms / args.steps
-    value = world * nodes_per_step / (ms_per_step * 1e-3)
+    value = whole_job_value(world, nodes_per_step, ms_per_step)
 
     # roofline of the dominant kernel (the per-node kernel): algorithmic bytes per launch =
     # every target row once + every draft row once (none at temperature 0) + 12 bytes of
@@ -367,10 +378,7 @@ def run_e2e(args, w, inp, dist, world, dev):
         step()                      # synchronises internally before it returns
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
-    if dist:
-        tt = torch.tensor([dt], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        dt = float(tt.item())
+    dt = max_over_ranks(dist, dt, dev)
     value = world * nb * st["n_draft"] * steps / dt
     return {"value": value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
             "ms_per_step": dt / steps * 1e3, "steps": steps, "batch": nb,
