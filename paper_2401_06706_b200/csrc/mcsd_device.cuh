@@ -334,6 +334,13 @@ struct Exchange {
     unsigned long long bar[2];
 };
 
+// What the leader warp of a CTA tells the other warps at the end of an exchange round.
+struct Action {
+    float4 stats;  // (row reference of p, of q, 1 / Z_t, Z_t / Z_d); written in the statistics round only
+    float c_try;   // c of the residual sum to form next
+    int more;      // 1: form that sum and run another round; 0: the node is decided
+};
+
 // Candidate data of the next items, fetched ahead of use by warp 0 so that no DRAM
 // latency sits on the per-node critical path: lane i handles candidate i.
 //   token id and acceptance uniform   two items ahead  (ring of 3)
@@ -426,8 +433,8 @@ node_kernel(const __grid_constant__ NodeParams P)
     uint4 *qraw = reinterpret_cast<uint4 *>(dyn + static_cast<size_t>(NT) * EPT * 4);
     __shared__ Exchange xch;
     __shared__ __align__(8) unsigned long long full_bar;
-    __shared__ double s_px[NW][MCSD_MAX_CHILDREN], s_qx[NW][MCSD_MAX_CHILDREN];
     __shared__ CandRing ring;
+    __shared__ Action act[2];
 
     const int tid = threadIdx.x, lane = tid & 31;
     // (broadcast from lane 0 so that the compiler knows the warp index is warp-uniform)
@@ -488,14 +495,17 @@ node_kernel(const __grid_constant__ NodeParams P)
             st_async_f4(dst, mine, map_to_rank(xbar_addr[s], lane));
         }
     };
-    auto exchange_wait = [&](float4 identity) -> float4 {
+    // leader (warp 0) only: waits for the round and returns entry `lane`
+    auto exchange_leader_wait = [&](float4 identity) -> float4 {
         const uint32_t s = round & 1u;
         // once a wait has expired the results are void and later rounds do not wait again
-        if (warp == 0 && !poisoned && !mbar_wait(xbar_addr[s], (round >> 1) & 1u)) poisoned = 1;
+        if (!poisoned && !mbar_wait(xbar_addr[s], (round >> 1) & 1u)) poisoned = 1;
+        return lane < n_entries ? xch.slot[s][lane] : identity;
+    };
+    // all warps: ends the round (the other warps have been waiting here for the leader)
+    auto exchange_release = [&]() {
         __syncthreads();
-        const float4 e = lane < n_entries ? xch.slot[s][lane] : identity;
         ++round;
-        return e;
     };
 
     // (sequence, node) of the items this cluster visits: the current one and the two after
@@ -630,8 +640,8 @@ node_kernel(const __grid_constant__ NodeParams P)
                 for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
             }
         }
-        // Each thread exponentiates relative to its own integer reference; the factor to
-        // the row's reference and the normaliser are applied as per-thread scalars later.
+        // Each warp exponentiates relative to its own integer reference; the factor to the
+        // row's reference and the normaliser are applied as per-warp scalars later.
         float rt, zt;
         {
             float m0 = -INFINITY, m1 = -INFINITY;
@@ -640,7 +650,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                 m0 = max3(m0, tv[p].x, tv[p].y);
                 m1 = max3(m1, tv[p + 1].x, tv[p + 1].y);
             }
-            rt = int_ref(fmaxf(m0, m1) * scale);
+            rt = int_ref(warp_max(fmaxf(m0, m1)) * scale);  // one reference per warp
             const float rt0 = (rt == -INFINITY) ? 0.f : rt;
             const f32x2 scale2 = pack2(scale, scale), nref2 = pack2(-rt0, -rt0);
             f32x2 z0 = pack2(0.f, 0.f), z1 = z0;
@@ -660,11 +670,10 @@ node_kernel(const __grid_constant__ NodeParams P)
             // A leaf decides nothing.  Its softmax statistics are only needed if a walk ends
             // here, so each warp leaves the partial statistics of its run in global memory
             // (the walk kernel combines them) and goes on: no exchange, no barrier.
-            const float Rt = warp_max(rt);
-            const float st = warp_sum(zt * exp2i(rt - Rt));
+            const float st = warp_sum(zt);
             if (lane == 0)
                 P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * 32 +
-                            crank * NW + warp] = make_float2(Rt, st);
+                            crank * NW + warp] = make_float2(rt, st);
             if (crank == 0 && tid == 0) P.node_accept[node_idx] = -1;
             look_ahead();
             next_item();
@@ -748,7 +757,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                 }
                 md = fmaxf(m0, m1);
             }
-            rd = int_ref(md * scale);
+            rd = int_ref(warp_max(md) * scale);
             const float rd0 = (rd == -INFINITY) ? 0.f : rd;
             const f32x2 scale2 = pack2(scale, scale), nref2 = pack2(-rd0, -rd0);
             f32x2 z0 = pack2(0.f, 0.f), z1 = z0;
@@ -771,61 +780,99 @@ node_kernel(const __grid_constant__ NodeParams P)
         }
 
         // ---- softmax statistics of both rows: one exchange round
-        {
-            const float Rt = warp_max(rt), Rd = warp_max(rd);
-            const float st = warp_sum(zt * exp2i(rt - Rt));
-            const float sd = warp_sum(zd * exp2i(rd - Rd));
-            exchange_send(make_float4(Rt, st, Rd, sd));  // per warp: (ref_t, z_t, ref_d, z_d)
-        }
+        exchange_send(make_float4(rt, warp_sum(zt), rd, warp_sum(zd)));  // per warp: (ref_t, z_t, ref_d, z_d)
         look_ahead();  // in the shadow of the exchange
-        // While the round is in flight: 2^(scaled logit) of the candidates' own logits as
-        // 2^int * frac (lane i = candidate i; every warp keeps its own copy so that no CTA
-        // barrier is needed).
-        int int_t = 0, int_d = 0;
-        bool cand_ok = false;
-        int my_tok = -1;
-        if (lane < k) {
-            float frac_t = 0.f, frac_d = 0.f;
-            my_tok = ring.tok[s3][lane];
-            cand_ok = my_tok >= 0 && my_tok < P.V;
-            if (cand_ok) {
-                const uint32_t wt = ring.tl[s2][lane], wd = ring.dl[s2][lane];
-                frac_t = split_exp2(DIRECT ? __uint_as_float(wt) : E::from_word(wt, my_tok), scale, P.scale_lo, int_t);
-                frac_d = split_exp2(DIRECT ? __uint_as_float(wd) : E::from_word(wd, my_tok), scale, P.scale_lo, int_d);
-            }
-            s_px[warp][lane] = static_cast<double>(frac_t);  // parked here until the exchange has completed
-            s_qx[warp][lane] = static_cast<double>(frac_d);
-        }
-        float4 ent = exchange_wait(make_float4(-INFINITY, 0.f, -INFINITY, 0.f));
-        // row references ceil(row maximum * scale) and normalisers, the same bits in every thread
-        const float R_t = warp_max(ent.x), R_d = warp_max(ent.z);
-        const float Z_t = warp_sum(ent.y * exp2i(ent.x - R_t));
-        const float Z_d = warp_sum(ent.w * exp2i(ent.z - R_d));
-        const bool t_ok = Z_t > 0.f && Z_t < INFINITY;            // false for an all -inf or NaN row
-        const bool d_ok = internal && Z_d > 0.f && Z_d < INFINITY;
-        if (!t_ok) status_bits |= MCSD_STATUS_NO_MASS;
-        // p(x) = tv * a, q(x) = dv * bq for this thread's elements
-        const float inv_zt = t_ok ? 1.f / Z_t : 0.f;
-        const float a = exp2i(rt - R_t) * inv_zt;
-        float b_over_a = 0.f;  // bq / a
-        if (a > 0.f && d_ok && rd != -INFINITY)
-            b_over_a = exp2i((rd - R_d) - (rt - R_t)) * (Z_t / Z_d);
-        if (crank == 0 && tid == 0)
-            *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
 
-        // Candidates' probabilities, both multiplied by K = Z_t * Z_d so that no division is
-        // needed: px' = 2^(l_t*scale - R_t) * Z_d, qx' = 2^(l_d*scale - R_d) * Z_t.
-        const double K = static_cast<double>(Z_t) * static_cast<double>(Z_d);
-        if (lane < k) {
-            double px = 0.0, qx = 0.0;
-            if (cand_ok && t_ok && d_ok) {
-                px = s_px[warp][lane] * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
-                qx = s_qx[warp][lane] * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
+        // From here on warp 0 of every CTA is the leader: it alone combines the exchanged
+        // values, evaluates the acceptance tests (Algorithm 1 / Algorithm 2) and tells the
+        // other warps through `act` what to do next; they only stream and reduce.  The
+        // leaders of a cluster work from bit-identical inputs and decide identically.
+        //
+        // leader state of the rejection loop, in units where W' = W * K, K = Z_t * Z_d:
+        double c = 0.0, S = 1.0, Wk = 0.0, K = 0.0, c_try = 0.0;
+        double px = 0.0, qx = 0.0;  // lane i of the leader: candidate i's p and q, times K
+        int cand_i = 0, attempt = 0, accepted = -1, my_tok = -1;
+        float u_acc = 2.f;
+        // tests candidates from cand_i on until one is accepted (returns 0), all are rejected
+        // (returns 0) or one is rejected and its residual sum is needed (returns 1, c_try set)
+        auto leader_decide = [&]() -> int {
+            while (cand_i < k) {
+                const int i = cand_i;
+                const int xi = __shfl_sync(0xffffffffu, my_tok, i);
+                const double ui = static_cast<double>(__shfl_sync(0xffffffffu, u_acc, i));
+                const double pxi = __shfl_sync(0xffffffffu, px, i), qxi = __shfl_sync(0xffffffffu, qx, i);
+                const bool valid = xi >= 0 && xi < P.V;
+                if (!valid) status_bits |= MCSD_STATUS_BAD_TOKEN;
+                // Algorithm 2: a token rejected earlier at this node has draft probability 0 now
+                const bool dup = P.mode == 1 &&
+                    (__ballot_sync(0xffffffffu, lane < i && my_tok == xi) != 0u);
+                const bool zero_q = !valid || dup || !(qxi > 0.0) || !(Wk > 0.0);
+                double Pn = pxi - c * qxi;
+                Pn = Pn > 0.0 ? Pn : 0.0;
+                // r <= [P_n(x~)/S_n] / [q(x~)/W_n] without divisions (all factors > 0)
+                const bool accept = !zero_q && ui * S * qxi * K <= Pn * Wk;
+                if (P.node_ratio && crank == 0 && lane == 0)
+                    P.node_ratio[static_cast<long long>(b) * P.n_nodes + first + i] =
+                        zero_q ? -1.f : static_cast<float>((Pn / S) / (qxi * K / Wk));
+                if (accept) { accepted = first + i; return 0; }
+                // rejected: p := norm(max(0, p - q)); Algorithm 2 also removes x~ from q
+                c_try = c;
+                if (Wk > 0.0) c_try = (P.mode == 1) ? c + S * K / Wk : c + S;
+                if (P.mode == 1 && !zero_q) { Wk -= qxi; if (!(Wk > 0.0)) Wk = 0.0; }
+                attempt = 0;
+                return 1;
             }
-            s_px[warp][lane] = px;
-            s_qx[warp][lane] = qx;
+            return 0;
+        };
+
+        if (warp == 0) {
+            // while the round is in flight: 2^(scaled logit) of the candidates' own logits as
+            // 2^int * frac (lane i = candidate i)
+            float frac_t = 0.f, frac_d = 0.f;
+            int int_t = 0, int_d = 0;
+            bool cand_ok = false;
+            if (lane < k) {
+                my_tok = ring.tok[s3][lane];
+                u_acc = ring.u[s3][lane];
+                cand_ok = my_tok >= 0 && my_tok < P.V;
+                if (cand_ok) {
+                    const uint32_t wt = ring.tl[s2][lane], wd = ring.dl[s2][lane];
+                    frac_t = split_exp2(DIRECT ? __uint_as_float(wt) : E::from_word(wt, my_tok), scale, P.scale_lo, int_t);
+                    frac_d = split_exp2(DIRECT ? __uint_as_float(wd) : E::from_word(wd, my_tok), scale, P.scale_lo, int_d);
+                }
+            }
+            const float4 ent = exchange_leader_wait(make_float4(-INFINITY, 0.f, -INFINITY, 0.f));
+            // row references ceil(row maximum * scale) and normalisers
+            const float R_t = warp_max(ent.x), R_d = warp_max(ent.z);
+            const float Z_t = warp_sum(ent.y * exp2i(ent.x - R_t));
+            const float Z_d = warp_sum(ent.w * exp2i(ent.z - R_d));
+            const bool t_ok = Z_t > 0.f && Z_t < INFINITY;  // false for an all -inf or NaN row
+            const bool d_ok = Z_d > 0.f && Z_d < INFINITY;
+            if (!t_ok) status_bits |= MCSD_STATUS_NO_MASS;
+            // candidates' probabilities, both multiplied by K so that no division is needed:
+            // px' = 2^(l_t*scale - R_t) * Z_d, qx' = 2^(l_d*scale - R_d) * Z_t
+            K = static_cast<double>(Z_t) * static_cast<double>(Z_d);
+            Wk = K;
+            if (cand_ok && t_ok && d_ok) {
+                px = static_cast<double>(frac_t) * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
+                qx = static_cast<double>(frac_d) * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
+            }
+            const int more = leader_decide();
+            if (lane == 0) {
+                act[round & 1u].stats = make_float4(R_t, R_d, t_ok ? 1.f / Z_t : 0.f, (t_ok && d_ok) ? Z_t / Z_d : 0.f);
+                act[round & 1u].c_try = static_cast<float>(c_try);
+                act[round & 1u].more = more;
+                if (crank == 0) *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
+            }
         }
-        __syncwarp();
+        exchange_release();  // CTA barrier: the leader's verdict is visible to all warps
+        const float4 st4 = act[(round - 1u) & 1u].stats;
+        int more = act[(round - 1u) & 1u].more;
+        float c_next = act[(round - 1u) & 1u].c_try;
+        // p(x) = tv * a, q(x) = dv * bq for this warp's elements
+        const float a = exp2i(rt - st4.x) * st4.z;
+        float b_over_a = 0.f;  // bq / a
+        if (a > 0.f && st4.w > 0.f && rd != -INFINITY) b_over_a = exp2i((rd - st4.y) - (rt - st4.x)) * st4.w;
 
         // residual mass of this warp's run for a given c
         auto residual_pass = [&](float c_f) -> float {
@@ -848,52 +895,42 @@ node_kernel(const __grid_constant__ NodeParams P)
             return warp_sum((t.x + t.y) * a);
         };
 
-        // ---- the rejection loop (Algorithm 1 / Algorithm 2), identical in every thread;
-        // state in units where W' = W * K
-        double c = 0.0, S = 1.0, Wk = K;
-        int accepted = -1;
-        for (int i = 0; i < k; ++i) {
-            const int xi = __shfl_sync(0xffffffffu, my_tok, i);
-            const double ui = static_cast<double>(ring.u[s3][i]);
-            const double pxi = s_px[warp][i], qxi = s_qx[warp][i];
-            const bool valid = xi >= 0 && xi < P.V;
-            if (!valid) status_bits |= MCSD_STATUS_BAD_TOKEN;
-            // Algorithm 2: a token rejected earlier at this node has draft probability 0 now
-            const bool dup = P.mode == 1 &&
-                (__ballot_sync(0xffffffffu, lane < i && my_tok == xi) != 0u);
-            const bool zero_q = !valid || dup || !(qxi > 0.0) || !(Wk > 0.0);
-            double Pn = pxi - c * qxi;
-            Pn = Pn > 0.0 ? Pn : 0.0;
-            // r <= [P_n(x~)/S_n] / [q(x~)/W_n] without divisions (all factors > 0)
-            const bool accept = !zero_q && ui * S * qxi * K <= Pn * Wk;
-            if (P.node_ratio && crank == 0 && tid == 0)
-                P.node_ratio[static_cast<long long>(b) * P.n_nodes + first + i] =
-                    zero_q ? -1.f : static_cast<float>((Pn / S) / (qxi * K / Wk));
-            if (accept) { accepted = first + i; break; }
-            // rejected: p := norm(max(0, p - q)); Algorithm 2 also removes x~ from q
-            double c_try = c;
-            if (Wk > 0.0) c_try = (P.mode == 1) ? c + S * K / Wk : c + S;
-            if (P.mode == 1 && !zero_q) { Wk -= qxi; if (!(Wk > 0.0)) Wk = 0.0; }
-            for (int attempt = 0; attempt < 2; ++attempt) {
-                exchange_send(make_float4(residual_pass(static_cast<float>(c_try)), 0.f, 0.f, 0.f));
-                ent = exchange_wait(make_float4(0.f, 0.f, 0.f, 0.f));
+        // ---- one round per rejection: all warps reduce, the leader decides what comes next
+#pragma unroll 1
+        while (more) {
+            exchange_send(make_float4(residual_pass(c_next), 0.f, 0.f, 0.f));
+            if (warp == 0) {
+                const float4 ent = exchange_leader_wait(make_float4(0.f, 0.f, 0.f, 0.f));
                 const float S_new = warp_sum(ent.x);
+                int next;
                 if (S_new > 0.f) {
                     if (attempt == 0) { c = c_try; S = static_cast<double>(S_new); }
-                    break;
+                    ++cand_i;
+                    next = leader_decide();
+                } else {
+                    // zero residual mass: keep the previous residual (recompute its sums once)
+                    status_bits |= MCSD_STATUS_DEGENERATE;
+                    if (attempt == 0) { attempt = 1; c_try = c; next = 1; }
+                    else { ++cand_i; next = leader_decide(); }
                 }
-                // zero residual mass: keep the previous residual (recompute its sums once)
-                status_bits |= MCSD_STATUS_DEGENERATE;
-                c_try = c;
+                if (lane == 0) {
+                    act[round & 1u].c_try = static_cast<float>(c_try);
+                    act[round & 1u].more = next;
+                }
             }
+            exchange_release();
+            more = act[(round - 1u) & 1u].more;
+            c_next = act[(round - 1u) & 1u].c_try;
         }
 
         // ---- per-node results (the endpoint token is drawn by the walk kernel, and only
         // for the node where a walk stops)
-        if (crank == 0 && tid == 0) {
-            P.node_accept[node_idx] = accepted;
-            reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
-                make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
+        if (warp == 0) {
+            if (crank == 0 && lane == 0) {
+                P.node_accept[node_idx] = accepted;
+                reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
+                    make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
+            }
         }
         if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
         status_bits = __reduce_or_sync(0xffffffffu, status_bits);
