@@ -425,6 +425,11 @@ node_kernel(const __grid_constant__ NodeParams P)
     constexpr int NG = EPT / GV;
     constexpr int H = GV / 4;  // float4 per group once exponentiated
     constexpr bool kRawZone = !DIRECT && E::kBytes == 2;
+    // L2 prefetch of the cluster's next item: with 2-byte logits the kernel is bound by the
+    // SMs and the prefetch takes DRAM latency off the per-node chain (measured +20 %); with
+    // 4-byte logits it is bound by HBM and the extra request stream only costs (-1 %, and
+    // -30 % on leaf-only trees), so it is left out there
+    constexpr bool kPrefetch = !DIRECT && E::kBytes == 2;
     static_assert(EPT % GV == 0, "EPT must be a whole number of 16-byte groups");
     static_assert(NW == 4, "the exchange buffers hold four warps per CTA");
 
@@ -564,7 +569,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         fetch_logits(b, n, 0, 0);
         fetch_tokens(b1, n1, 1);
     }
-    if (!DIRECT && tid == 0 && b < P.B && bulk_bytes) {
+    if (kPrefetch && tid == 0 && b < P.B && bulk_bytes) {
         bulk_prefetch_l2(t_slice(static_cast<long long>(b) * P.n_nodes + n), bulk_bytes);
         if (n < P.n_internal) bulk_prefetch_l2(d_slice(b, n), bulk_bytes);
     }
@@ -600,7 +605,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         // data of the next two items
         auto look_ahead = [&]() {
             if (warp == 0) {
-                if (!DIRECT && lane == 0 && b1 < P.B && bulk_bytes) {
+                if (kPrefetch && lane == 0 && b1 < P.B && bulk_bytes) {
                     bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
                     if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
                 }
@@ -1084,6 +1089,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
     using E = Elem<DT>;
     constexpr int GV = E::kVec;
     __shared__ int s_term, s_len;
+    __shared__ int32_t s_acc[MCSD_MAX_NODES], s_tok[MCSD_MAX_NODES];
     __shared__ float s_wtot[kWalkWarps];
     __shared__ float s_leaf[2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1099,13 +1105,20 @@ walk_kernel(const __grid_constant__ WalkParams P)
     int32_t *tok = P.out_tokens + static_cast<long long>(b) * (P.gamma + 1);
     int len = 0;
     if (!P.all_nodes) {
+        // the tree's decisions and tokens come into shared memory with one parallel load, so
+        // that the walk itself is not a chain of dependent global loads
+        for (int i = tid; i < P.n_nodes; i += kWalkThreads) {
+            s_acc[i] = P.node_accept[nb + i];
+            s_tok[i] = P.cand[nb + i];
+        }
+        __syncthreads();
         if (tid == 0) {
             // bounded by the depth of the tree even if node_accept were corrupt
             for (int hop = 0; hop < P.gamma; ++hop) {
-                const int nx = P.node_accept[nb + n];
+                const int nx = s_acc[n];
                 if (nx <= n || nx >= P.n_nodes) break;
                 n = nx;
-                tok[len] = P.cand[nb + n];
+                tok[len] = s_tok[n];
                 ++len;
             }
             for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
@@ -1189,6 +1202,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
 
     // pass 1: the distribution itself and the mass of every run
     float mass = 0.f;
+#pragma unroll 4
     for (int x0 = x_lo + lane * GV; x0 < x_hi; x0 += kStep) {
         float w[GV];
         weights(x0, w);
