@@ -386,6 +386,63 @@ def run_e2e(args, w, inp, dist, world, dev):
                     "kernels inside the timed region; bound by the host link"}
 
 
+# ----------------------------------------------------------------------------- sweep
+def run_sweep(args):
+    """The 300-point throughput sweep (dtype x batch x k-config x sigma x mode at vocabulary
+    32000, temperature 1).  Every call is timed on its own between CUDA events with L2
+    flushed before it (a 256 MB buffer is overwritten), so small points report their
+    cold-cache latency; each point is checked against the oracle on its first sequences.
+    Writes one JSON line per point to --sweep-out and prints a summary line per point."""
+    from paper_2401_06706_b200 import binding
+    import oracle
+    from oracle import compare
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    binding.load_library()
+    peak, peak_kind = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    points = [w for w in synth.sweep_workloads() if args.sweep_filter in w.name]
+    out = open(args.sweep_out, "w") if args.sweep_out else None
+    for w in points:
+        inp = synth.make_inputs(w, dev)
+        st = inp.stats
+        ver = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[w.dtype], dev)
+        for _ in range(5):
+            ver.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+        times = []
+        for _ in range(args.sweep_calls):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ver.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        med, best = statistics.median(times), min(times)
+        n_par = min(w.batch, args.sweep_parity_seqs)
+        t, d, c, u = inp.host_f32(0, n_par)
+        rep = compare.compare(t, d, inp.parent, c, u, w.temperature, w.mode, w.dtype,
+                              accept_len=ver.accept_len[:n_par].cpu().numpy(), tokens=ver.tokens[:n_par].cpu().numpy(),
+                              residual=ver.residual[:n_par].cpu().numpy(), status=ver.status[:n_par].cpu().numpy())
+        algo = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
+        rec = {"workload": w.name, "dtype": w.dtype, "batch": w.batch, "kconfig": w.kconfig, "sigma": w.draft_sigma,
+               "mode": w.mode, "algorithmic_mb": algo / 1e6, "us_median": med * 1e3, "us_min": best * 1e3,
+               "nodes_per_s": w.batch * st["n_draft"] / (med * 1e-3), "gbs": algo / (med * 1e-3) / 1e9,
+               "frac_of_peak": algo / (med * 1e-3) / 1e9 / peak, "peak_kind": peak_kind,
+               "regime": "hbm" if algo > 4 * 126e6 else "latency/L2-bound point (inputs < 4x L2)",
+               "accept_len_mean": float(ver.accept_len.float().mean().item()), "parity_ok": rep.ok,
+               "parity": rep.summary()}
+        if out:
+            out.write(json.dumps(rec) + "\n")
+            out.flush()
+        print(f"{w.name:40s} {rec['algorithmic_mb']:9.1f} MB {rec['us_median']:9.1f} us {rec['gbs']:7.0f} GB/s "
+              f"{rec['frac_of_peak']:.3f} tau-1={rec['accept_len_mean']:.2f} parity={'ok' if rep.ok else 'FAIL'}", flush=True)
+        del inp, ver
+        torch.cuda.empty_cache()
+    if out:
+        out.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -400,8 +457,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch of the workload (profiling)")
+    ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the bench line")
+    ap.add_argument("--sweep-filter", default="", help="only sweep points whose name contains this text")
+    ap.add_argument("--sweep-out", default="", help="file for one JSON line per sweep point")
+    ap.add_argument("--sweep-calls", type=int, default=20)
+    ap.add_argument("--sweep-parity-seqs", type=int, default=16)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

@@ -8,7 +8,8 @@ Rules
     that a node whose first differing test has |u - rho_oracle| < NEAR_TIE is
     counted as a flipped near-tie and the rest of that node is skipped.
   * Every test the oracle performed with |u - rho| < NEAR_TIE is counted as a
-    near-tie decision; these must stay below NEAR_TIE_SHARE of all decisions.
+    near-tie decision; these must stay below NEAR_TIE_SHARE of all decisions (small
+    samples: at most NEAR_TIE_MIN_EVENTS events).
   * A sequence whose oracle path crosses a flipped node is excluded from the path
     and residual comparison (and counted).  All other sequences must have the same
     accepted length and accepted tokens.
@@ -28,6 +29,10 @@ from . import verify as oracle_verify, softmax as oracle_softmax, mcss as oracle
 
 NEAR_TIE = 1e-5
 NEAR_TIE_SHARE = 1e-4
+# The share is a rate: on a sample of a few hundred tests one single event already exceeds
+# 0.01 %, which says nothing about the rate (uniforms on a 2^-23 grid put about 2e-5 of all
+# tests inside the band by chance alone).  Up to this many events are always allowed.
+NEAR_TIE_MIN_EVENTS = 3
 RESIDUAL_TOL = {"fp32": 1e-5, "bf16": 2e-3, "fp16": 2e-3}
 
 
@@ -111,7 +116,7 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
         u0 = unif[:, :, 0].astype(np.float64)
         near = tested & (ref.node_ratio >= 0) & (np.abs(u0 - ref.node_ratio) < NEAR_TIE)
         rep.n_near_tie = int(near.sum())
-        if rep.n_near_tie > NEAR_TIE_SHARE * max(rep.n_tests, 1):
+        if rep.n_near_tie > max(NEAR_TIE_MIN_EVENTS, NEAR_TIE_SHARE * rep.n_tests):
             fail(f"{rep.n_near_tie} near-tie decisions out of {rep.n_tests} exceed the allowed share")
 
     flipped = np.zeros((B, n_nodes), dtype=bool)
