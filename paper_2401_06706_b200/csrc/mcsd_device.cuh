@@ -1200,16 +1200,24 @@ walk_kernel(const __grid_constant__ WalkParams P)
     int x_hi = x_lo + run;
     x_hi = x_hi > P.V ? P.V : x_hi;
 
-    // pass 1: the distribution itself and the mass of every run
+    // pass 1: the distribution itself, the mass of every run, and per lane the mass of its
+    // group in every step of the run (kept for the search below)
+    constexpr int kMaxSteps = MCSD_MAX_VOCAB / kWalkWarps / kStep;
+    float g[kMaxSteps];
     float mass = 0.f;
-#pragma unroll 4
-    for (int x0 = x_lo + lane * GV; x0 < x_hi; x0 += kStep) {
-        float w[GV];
-        weights(x0, w);
 #pragma unroll
-        for (int e = 0; e < GV; ++e) {
-            mass += w[e];
-            if (out && x0 + e < P.V) out[x0 + e] = w[e] * inv_s;
+    for (int st = 0; st < kMaxSteps; ++st) {
+        g[st] = 0.f;
+        const int x0 = x_lo + st * kStep + lane * GV;
+        if (x0 < x_hi) {
+            float w[GV];
+            weights(x0, w);
+#pragma unroll
+            for (int e = 0; e < GV; ++e) {
+                g[st] += w[e];
+                if (out && x0 + e < P.V) out[x0 + e] = w[e] * inv_s;
+            }
+            mass += g[st];
         }
     }
     mass = warp_sum(mass);
@@ -1236,55 +1244,52 @@ walk_kernel(const __grid_constant__ WalkParams P)
     }
     if (warp != pick) return;
 
-    // pass 2 (one warp): 32 * GV elements at a time until the quantile is passed
-    float tgt = target - __shfl_sync(0xffffffffu, inc - m, pick);
-    int found = -1, last_x0 = -1;     // element index; start of the last step that had mass
-    float runsum = 0.f;
-    for (int x0 = x_lo; x0 < x_hi && found < 0; x0 += kStep) {
-        float w[GV];
-        weights(x0 + lane * GV, w);
-        float g = 0.f;
+    // the step of the run that holds the quantile, from the step totals; then the lane and
+    // the element inside that step (its weights are formed once more)
+    const float tgt = target - __shfl_sync(0xffffffffu, inc - m, pick);
+    float tj;
+    warp_multi_sum<kMaxSteps>(g, lane, tj);  // lane st * (32 / kMaxSteps) holds the total of step st
+    int ps = -1, last_s = -1;
+    float runsum = 0.f, ps_before = 0.f;
 #pragma unroll
-        for (int e = 0; e < GV; ++e) g += w[e];
-        const float gi = warp_scan_incl(g, lane);
-        const float step_total = __shfl_sync(0xffffffffu, gi, 31);
-        if (step_total > 0.f) {
-            last_x0 = x0;
-            if (runsum + step_total > tgt) {
-                const float t2 = tgt - runsum;
-                const unsigned h2 = __ballot_sync(0xffffffffu, g > 0.f && gi > t2);
-                const unsigned p2 = __ballot_sync(0xffffffffu, g > 0.f);
-                const int l = h2 ? __ffs(h2) - 1 : 31 - __clz(p2);
-                int pe = -1, last = -1;
-                if (lane == l) {
-                    const float rem = t2 - (gi - g);
-                    float acc = 0.f;
-#pragma unroll
-                    for (int e = 0; e < GV; ++e) {
-                        if (w[e] > 0.f) {
-                            acc += w[e];
-                            last = e;
-                            if (pe < 0 && acc > rem) pe = e;
-                        }
-                    }
-                    if (pe < 0) pe = last;
-                }
-                found = __shfl_sync(0xffffffffu, x0 + lane * GV + pe, l);
-            }
+    for (int st = 0; st < kMaxSteps; ++st) {
+        const float ms = __shfl_sync(0xffffffffu, tj, st * (32 / kMaxSteps));
+        if (ms > 0.f) {
+            last_s = st;
+            if (ps < 0 && runsum + ms > tgt) { ps = st; ps_before = runsum; }
         }
-        runsum += step_total;
+        runsum += ms;
     }
-    if (found < 0 && last_x0 >= 0) {
-        // rounding: the quantile lies past the run's own sum; take its last element with mass
-        float w[GV];
-        weights(last_x0 + lane * GV, w);
-        int last = -1;
+    // rounding may leave the quantile past the run's own sum: take its last element with mass
+    float t2 = tgt - ps_before;
+    if (ps < 0) { ps = last_s; t2 = INFINITY; }
+    int found = -1;
+    if (ps >= 0) {
+        float gs = g[0];
 #pragma unroll
-        for (int e = 0; e < GV; ++e) if (w[e] > 0.f) last = e;
-        const unsigned p2 = __ballot_sync(0xffffffffu, last >= 0);
+        for (int st = 1; st < kMaxSteps; ++st) gs = (ps == st) ? g[st] : gs;
+        const float gi = warp_scan_incl(gs, lane);
+        const unsigned h2 = __ballot_sync(0xffffffffu, gs > 0.f && gi > t2);
+        const unsigned p2 = __ballot_sync(0xffffffffu, gs > 0.f);
         if (p2) {
-            const int l = 31 - __clz(p2);
-            found = __shfl_sync(0xffffffffu, last_x0 + lane * GV + last, l);
+            const int l = h2 ? __ffs(h2) - 1 : 31 - __clz(p2);
+            int pe = -1, last = -1;
+            if (lane == l) {
+                float w[GV];
+                weights(x_lo + ps * kStep + lane * GV, w);
+                const float rem = t2 - (gi - gs);
+                float acc = 0.f;
+#pragma unroll
+                for (int e = 0; e < GV; ++e) {
+                    if (w[e] > 0.f) {
+                        acc += w[e];
+                        last = e;
+                        if (pe < 0 && acc > rem) pe = e;
+                    }
+                }
+                if (pe < 0) pe = last;
+            }
+            found = __shfl_sync(0xffffffffu, pe < 0 ? -1 : x_lo + ps * kStep + lane * GV + pe, l);
         }
     }
     if (lane == 0) {
