@@ -244,6 +244,13 @@ def run_cuda(args):
     nodes_per_step = w.batch * st["n_draft"]
 
     def step(events=None):
+        if args.form == "path":
+            if events is not None:
+                events[0].record()
+            ver.mcsd_verify_path(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
+            if events is not None:
+                events[1].record()
+            return
         if events is None:
             ver.mcsd_verify(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
             return
@@ -257,10 +264,14 @@ def run_cuda(args):
         step()
     torch.cuda.synchronize()
     launches_per_step = 0
-    ver.mcsd_verify_nodes(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
-    launches_per_step += binding.mcsd_last_launch_count()
-    ver.mcsd_verify_walk(inp.target, draft, inp.cand, inp.unif, w.temperature)
-    launches_per_step += binding.mcsd_last_launch_count()
+    if args.form == "path":
+        ver.mcsd_verify_path(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
+        launches_per_step += binding.mcsd_last_launch_count()
+    else:
+        ver.mcsd_verify_nodes(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
+        launches_per_step += binding.mcsd_last_launch_count()
+        ver.mcsd_verify_walk(inp.target, draft, inp.cand, inp.unif, w.temperature)
+        launches_per_step += binding.mcsd_last_launch_count()
     torch.cuda.synchronize()
 
     # timed region: K steps between barriers and synchronisations, CUDA events on the
@@ -297,15 +308,25 @@ def run_cuda(args):
     # every target row once + every draft row once (none at temperature 0) + 12 bytes of
     # candidate token and uniforms per node
     algo_bytes = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
+    if args.form == "path":
+        # only the rows of visited nodes are read: len+1 target rows per sequence and one draft
+        # row per visited node that has children (every node above the leaf level)
+        ln = ver.accept_len.to(torch.int64)
+        rows = int((ln + 1).sum().item()) + (int(torch.clamp(ln + 1, max=st["gamma"]).sum().item())
+                                             if w.temperature > 0 else 0)
+        algo_bytes = rows * w.vocab * inp.target.element_size()
     node_ms_avg = sum(node_ms) / len(node_ms)
     achieved = algo_bytes / (node_ms_avg * 1e-3) / 1e9
     peak, peak_kind = measured_peaks()
-    roofline = {"bound": "hbm", "kernel": "node_kernel" if w.temperature > 0 else "argmax_kernel",
+    roofline = {"bound": "hbm", "kernel": ("node_kernel" if w.temperature > 0 else "argmax_kernel") +
+                (" (one launch per level; the figure covers the whole call, which is bound by launch and "
+                 "exchange latency, not by HBM)" if args.form == "path" else ""),
                 "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_avg": node_ms_avg,
                 "kernel_ms_min": min(node_ms), "step_share": node_ms_avg / ms_per_step,
-                "traffic": recorded_traffic(w.batch * st["n_nodes"]) if w.name == "cfg5_largest" else None}
+                "traffic": recorded_traffic(w.batch * st["n_nodes"])
+                if (w.name == "cfg5_largest" and args.form == "all_node") else None}
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside
     e2e = None
@@ -322,7 +343,7 @@ def run_cuda(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": workload_config(w, st, parallelism=f"replicas x{world} (batch split, no collective)",
+                "config": workload_config(w, st, form=args.form, parallelism=f"replicas x{world} (batch split, no collective)",
                                           l2="inputs (%.2f GB per GPU) far larger than the 126 MB L2" %
                                           (inp.logit_bytes() / 1e9) if inp.logit_bytes() > 4 * 126e6 else
                                           "inputs smaller than 4x L2: latency/L2-bound point",
@@ -457,6 +478,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch of the workload (profiling)")
+    ap.add_argument("--form", default="all_node", choices=["all_node", "path"],
+                    help="all_node: every node of every tree is evaluated (the measured configuration); "
+                         "path: mcsd_verify_path, only the nodes the walks visit, one launch per level")
     ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the bench line")
     ap.add_argument("--sweep-filter", default="", help="only sweep points whose name contains this text")
     ap.add_argument("--sweep-out", default="", help="file for one JSON line per sweep point")

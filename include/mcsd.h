@@ -168,6 +168,23 @@ int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const voi
                      float temperature, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual);
 
 /*
+ * The same result computed the way Section 3 describes the procedure: only the nodes a
+ * walk actually visits are evaluated.  Level by level (one kernel launch per level of the
+ * tree, gamma + 1 in all), every sequence evaluates the node its walk stands on
+ * (softmax of that node's two rows, Algorithm 1 / 2 on its candidates) and moves to the
+ * accepted child; then the walk stage runs as in mcsd_verify.  At most 2 * gamma + 1 logit
+ * rows per tree are read instead of all of them, at the price of gamma + 1 dependent
+ * launches, so this is the form to use when the tree is large or latency matters more
+ * than the node rate.  Outputs are identical to those of mcsd_verify (the same tests with
+ * the same uniforms).  The optional per-node outputs of the descriptor are filled for
+ * visited nodes only and node_bonus is not produced.  Arguments as in mcsd_verify.
+ */
+int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int replacement_mode, int32_t *out_accept_len,
+                     int32_t *out_tokens, float *out_residual);
+
+/*
  * The same step for callers whose data lives in HOST memory: every pointer below
  * is a host pointer.  The library allocates device buffers for a slice of the
  * batch, copies the slice in, verifies it and copies the results back, slice

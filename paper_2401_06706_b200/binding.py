@@ -22,7 +22,7 @@ MCSD_DTYPE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 STATUS_DEGENERATE, STATUS_BAD_TOKEN, STATUS_NO_MASS, STATUS_TIMEOUT = 1, 2, 4, 8
 MAX_NODES, MAX_CHILDREN, MAX_VOCAB = 512, 32, 65536
 
-EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static",
+EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path",
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
            "mcsd_version")
 
@@ -60,6 +60,8 @@ def load_library(path: Optional[str] = None):
     dp = ctypes.POINTER(McsdDesc)
     lib.mcsd_verify.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
     lib.mcsd_verify.restype = ctypes.c_int
+    lib.mcsd_verify_path.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
+    lib.mcsd_verify_path.restype = ctypes.c_int
     lib.mcsd_verify_static.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
     lib.mcsd_verify_static.restype = ctypes.c_int
     lib.mcsd_verify_nodes.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int]
@@ -208,6 +210,16 @@ class Verifier:
         _check(self.lib.mcsd_verify(ctypes.byref(self.desc), _ptr(target), _ptr(draft), self.parent.ctypes.data,
                                     _ptr(cand), _ptr(unif), float(temperature), int(mode),
                                     _ptr(self.accept_len), _ptr(self.tokens), _ptr(self.residual)))
+        return self._out()
+
+    def mcsd_verify_path(self, target, draft, cand, unif, temperature: float, mode: int) -> VerifyOutput:
+        """Level-by-level form: only the nodes the walks visit are evaluated (see mcsd.h)."""
+        self._bind(target, draft)
+        if self.node_ratio is not None:
+            self.node_ratio.fill_(float("nan"))
+        _check(self.lib.mcsd_verify_path(ctypes.byref(self.desc), _ptr(target), _ptr(draft),
+                                         self.parent.ctypes.data, _ptr(cand), _ptr(unif), float(temperature),
+                                         int(mode), _ptr(self.accept_len), _ptr(self.tokens), _ptr(self.residual)))
         return self._out()
 
     def mcsd_verify_static(self, target, draft, cand, unif, temperature: float, mode: int) -> VerifyOutput:

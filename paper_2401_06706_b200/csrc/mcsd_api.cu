@@ -58,6 +58,7 @@ struct Workspace {
     NodeStats *stats;
     float2 *leaf_part;
     int32_t *status;
+    int32_t *path[2];
     size_t bytes;
 };
 
@@ -75,6 +76,8 @@ Workspace carve(void *base, long long n_items, long long n_leaf_items, int batch
     w.stats = reinterpret_cast<NodeStats *>(take(sizeof(NodeStats) * n_items));
     w.leaf_part = reinterpret_cast<float2 *>(take(sizeof(float2) * 32 * n_leaf_items));
     w.status = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
+    w.path[0] = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
+    w.path[1] = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
     w.bytes = off;
     return w;
 }
@@ -268,14 +271,24 @@ int check_common(const mcsd_desc *d, const void *target, const void *draft, cons
     return MCSD_OK;
 }
 
+// level < 0: the all-node form (every node of every tree is an item).  level >= 0: path
+// mode, the items are the sequences and each works on the node its walk stands on at
+// that level (path arrays in the workspace, swapped level by level).
 int launch_nodes(const Call &c, const void *target, const void *draft, const int32_t *cand,
-                 const float *unif, float T, int mode)
+                 const float *unif, float T, int mode, int level = -1)
 {
     const mcsd_desc *d = c.d;
-    const long long n_items = static_cast<long long>(d->batch) * d->n_nodes;
+    const bool path = level >= 0;
+    const long long n_items = path ? d->batch : static_cast<long long>(d->batch) * d->n_nodes;
     if (n_items == 0) return MCSD_OK;
-    if (cudaMemsetAsync(c.status, 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
-        return MCSD_ERR_CUDA;
+    const int32_t *path_cur = path ? c.ws.path[level & 1] : nullptr;
+    int32_t *path_next = path ? c.ws.path[(level + 1) & 1] : nullptr;
+    if (level <= 0) {
+        if (cudaMemsetAsync(c.status, 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
+            return MCSD_ERR_CUDA;
+        if (path && cudaMemsetAsync(c.ws.path[0], 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
+            return MCSD_ERR_CUDA;  // every walk starts at the root
+    }
 
     if (T == 0.f) {
         ArgmaxParams p = {};
@@ -285,6 +298,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
         p.n_rows = static_cast<int32_t>(n_items);
         p.vector_ok = rows_aligned16(target, d->ld_target, d->dtype) ? 1 : 0;
+        p.path_cur = path_cur; p.path_next = path_next;
         std::memcpy(p.child_first, c.plan.child_first, sizeof(p.child_first));
         std::memcpy(p.child_count, c.plan.child_count, sizeof(p.child_count));
         int dev = 0, n_sm = 148;
@@ -321,8 +335,9 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     p.B = d->batch; p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
     p.slice = cfg.slice;
     p.n_items = static_cast<int32_t>(n_items);
-    p.step_b = static_cast<int32_t>(n_clusters / d->n_nodes);
-    p.step_n = static_cast<int32_t>(n_clusters % d->n_nodes);
+    p.step_b = static_cast<int32_t>(path ? n_clusters : n_clusters / d->n_nodes);
+    p.step_n = static_cast<int32_t>(path ? 0 : n_clusters % d->n_nodes);
+    p.path_cur = path_cur; p.path_next = path_next;
     p.mode = mode;
     const double scale_d = 1.4426950408889634 / static_cast<double>(T);
     p.scale = static_cast<float>(scale_d);
@@ -351,7 +366,8 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
 }
 
 int launch_walk(const Call &c, const void *target, const void *draft, const int32_t *cand,
-                const float *unif, float T, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
+                const float *unif, float T, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual,
+                bool all_nodes_allowed = true)
 {
     const mcsd_desc *d = c.d;
     if (d->batch == 0) return MCSD_OK;
@@ -376,7 +392,7 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
         p.n_entries = cfg.cluster * kNodeWarps;
     }
     // all-nodes pass first (only when per-node endpoint tokens were asked for), then the walks
-    for (int all = (T > 0.f && d->node_bonus) ? 1 : 0; all >= 0; --all) {
+    for (int all = (T > 0.f && d->node_bonus && all_nodes_allowed) ? 1 : 0; all >= 0; --all) {
         p.all_nodes = all;
         const unsigned grid = static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch);
         switch (d->dtype) {
@@ -484,6 +500,30 @@ int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *dr
     if (rc != MCSD_OK) return rc;
     return launch_walk(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, out_accept_len,
                        out_tokens, out_residual);
+}
+
+int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int replacement_mode, int32_t *out_accept_len,
+                     int32_t *out_tokens, float *out_residual)
+{
+    Call c;
+    int rc = prepare(desc, tree_parent, &c);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0) return MCSD_OK;
+    rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
+                      replacement_mode, true);
+    if (rc != MCSD_OK) return rc;
+    if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
+    // one launch per level of the tree: level l evaluates, for every sequence, the node its
+    // walk stands on after l accepted tokens (nothing for walks that have ended)
+    for (int level = 0; level <= c.plan.gamma; ++level) {
+        rc = launch_nodes(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, replacement_mode, level);
+        if (rc != MCSD_OK) return rc;
+    }
+    return launch_walk(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, out_accept_len,
+                       out_tokens, out_residual, false);
 }
 
 // ---- mcsd_verify_static: the scratch memory is an array built into the library --------

@@ -71,6 +71,11 @@ struct NodeParams {
     int32_t slice;   // vocabulary elements owned by one CTA of the cluster
     int32_t n_items; // B * n_nodes
     int32_t step_b, step_n;  // quotient and remainder of (clusters in the grid) / n_nodes
+    // Path mode (one launch per tree level): the items are the sequences, item b works on node
+    // path_cur[b] (negative: that walk has ended, nothing to do) and leaves in path_next[b] the
+    // accepted child, or -1.  Null for the all-node form.  Then step_b = clusters, step_n = 0.
+    const int32_t *path_cur;
+    int32_t *path_next;
     int32_t mode;
     float scale;     // log2(e) / T rounded to float ...
     float scale_lo;  // ... and what the rounding dropped (for the candidates' own probabilities)
@@ -519,12 +524,13 @@ node_kernel(const __grid_constant__ NodeParams P)
         b += P.step_b;
         n += P.step_n;
         if (n >= P.n_nodes) { n -= P.n_nodes; ++b; }
+        if (P.path_cur) n = b < P.B ? __ldg(P.path_cur + b) : 0;
     };
 
     // ---- candidate pipeline (warp 0 only) -------------------------------------------
     auto fetch_tokens = [&](int b, int n, int slot3) {
         if (b < P.B) {
-            const int k = n < P.n_internal ? P.child_count[n] : 0;
+            const int k = (n >= 0 && n < P.n_internal) ? P.child_count[n] : 0;
             if (lane < k) {
                 const long long ci = static_cast<long long>(b) * P.n_nodes + P.child_first[n] + lane;
                 cp_async4(&ring.tok[slot3][lane], P.cand + ci);
@@ -535,7 +541,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     // needs the item's tokens to have arrived (cp_async_wait_all by this thread)
     auto fetch_logits = [&](int b, int n, int slot3, int slot2) {
         if (b < P.B) {
-            const int k = n < P.n_internal ? P.child_count[n] : 0;
+            const int k = (n >= 0 && n < P.n_internal) ? P.child_count[n] : 0;
             if (lane < k) {
                 const int xt = ring.tok[slot3][lane];
                 if (xt >= 0 && xt < P.V) {
@@ -556,6 +562,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     };
 
     int b = cluster_id / P.n_nodes, n = cluster_id - b * P.n_nodes;  // current item
+    if (P.path_cur) { b = cluster_id; n = b < P.B ? __ldg(P.path_cur + b) : 0; }
     int b1 = b, n1 = n;                                              // the next one
     advance(b1, n1);
     int b2 = b1, n2 = n1;                                            // the one after
@@ -575,9 +582,9 @@ node_kernel(const __grid_constant__ NodeParams P)
     }
 
     for (; b < P.B; ++it) {
-        const bool internal = n < P.n_internal;
+        const bool internal = n >= 0 && n < P.n_internal;
         const int k = internal ? P.child_count[n] : 0;
-        const int first = P.child_first[n];
+        const int first = internal ? P.child_first[n] : 0;
         const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
         const int s3 = it % 3u, s2 = it & 1u;
         int status_bits = 0;
@@ -618,6 +625,13 @@ node_kernel(const __grid_constant__ NodeParams P)
             b1 = b2; n1 = n2;
             advance(b2, n2);
         };
+
+        if (n < 0) {  // path mode: this walk ended at an earlier level
+            if (crank == 0 && tid == 0) P.path_next[b] = -1;
+            look_ahead();
+            next_item();
+            continue;
+        }
 
         // ---- target slice -> registers, as packed pairs
         f32x2 tv[EPT / 2];
@@ -679,7 +693,10 @@ node_kernel(const __grid_constant__ NodeParams P)
             if (lane == 0)
                 P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * 32 +
                             crank * NW + warp] = make_float2(rt, st);
-            if (crank == 0 && tid == 0) P.node_accept[node_idx] = -1;
+            if (crank == 0 && tid == 0) {
+                P.node_accept[node_idx] = -1;
+                if (P.path_next) P.path_next[b] = -1;
+            }
             look_ahead();
             next_item();
             continue;
@@ -933,6 +950,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (warp == 0) {
             if (crank == 0 && lane == 0) {
                 P.node_accept[node_idx] = accepted;
+                if (P.path_next) P.path_next[b] = accepted;
                 reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
                     make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
             }
@@ -958,6 +976,9 @@ struct ArgmaxParams {
     long long ld_t;
     int32_t n_nodes, n_internal, V, n_rows;
     int32_t vector_ok;  // rows are 16-byte aligned
+    // path mode, as in NodeParams: n_rows = sequences, item b works on node path_cur[b]
+    const int32_t *path_cur;
+    int32_t *path_next;
     uint16_t child_first[MCSD_MAX_NODES];
     uint8_t child_count[MCSD_MAX_NODES];
 };
@@ -971,7 +992,16 @@ argmax_kernel(const __grid_constant__ ArgmaxParams P)
     __shared__ float s_val[kWarps];
     __shared__ int s_idx[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int row = blockIdx.x; row < P.n_rows; row += gridDim.x) {
+    for (int item = blockIdx.x; item < P.n_rows; item += gridDim.x) {
+        int row = item;
+        if (P.path_cur) {
+            const int pn = __ldg(P.path_cur + item);
+            if (pn < 0) {  // this walk ended at an earlier level
+                if (tid == 0) P.path_next[item] = -1;
+                continue;
+            }
+            row = item * P.n_nodes + pn;
+        }
         const unsigned char *t_row = reinterpret_cast<const unsigned char *>(P.target) +
             static_cast<long long>(row) * P.ld_t * E::kBytes;
         float best = -INFINITY;
@@ -1043,6 +1073,7 @@ argmax_kernel(const __grid_constant__ ArgmaxParams P)
             if (lane == 0) {
                 P.node_accept[row] = acc;
                 P.node_bonus[row] = acc >= 0 ? -1 : a;
+                if (P.path_next) P.path_next[item] = acc;
             }
         }
         __syncthreads();
