@@ -52,6 +52,12 @@ def _bind(lib):
     lib.mcsd_oracle_invcdf.restype = c_i32
     lib.mcsd_oracle_mcss.argtypes = [P, P, c_i32, P, P, c_i32, c_i32, P, P, P]
     lib.mcsd_oracle_mcss.restype = c_i32
+    lib.mcsd_oracle_draw.argtypes = [P, c_i32, P, c_i32, c_i32, P]
+    lib.mcsd_oracle_draw.restype = c_i32
+    lib.mcsd_oracle_topk.argtypes = [P, c_i32, c_i32, P]
+    lib.mcsd_oracle_topk.restype = None
+    lib.mcsd_oracle_sample.argtypes = [c_i32, c_i32, c_i32, c_i32, P, P, P, c_dbl, c_i32, c_i32, c_i32, P]
+    lib.mcsd_oracle_sample.restype = c_i32
     lib.mcsd_oracle_verify.argtypes = [c_i32, c_i32, c_i32, c_i32, P, P, P, P, P, c_dbl, c_i32,
                                        c_i32, P, P, P, P, P, P, P]
     lib.mcsd_oracle_verify.restype = c_i32
@@ -88,6 +94,41 @@ def argmax(logits) -> int:
 def invcdf(P, u: float) -> int:
     P = np.ascontiguousarray(P, dtype=np.float64)
     return int(_load().mcsd_oracle_invcdf(_ptr(P), P.shape[0], float(u)))
+
+
+def draw(q, u, mode: int) -> np.ndarray:
+    """k draws from q by inverse CDF with the uniforms u: with replacement (mode 0) or without,
+    Eq. 1 (mode 1).  Returns the k tokens (-1 where no mass was left)."""
+    q = np.array(q, dtype=np.float64, copy=True)
+    u = np.ascontiguousarray(u, dtype=np.float64)
+    x = np.empty(u.shape[0], dtype=np.int32)
+    _load().mcsd_oracle_draw(_ptr(q), q.shape[0], _ptr(u), u.shape[0], int(mode), _ptr(x))
+    return x
+
+
+def topk(logits, k: int) -> np.ndarray:
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    x = np.empty(k, dtype=np.int32)
+    _load().mcsd_oracle_topk(_ptr(logits), logits.shape[0], int(k), _ptr(x))
+    return x
+
+
+def sample(draft, parent, unif_draw, T: float, mode: int, node_begin: int = 0, node_end=None, cand=None) -> np.ndarray:
+    """Candidate tokens of the children of the nodes [node_begin, node_end) of every tree; see
+    ``mcsd_oracle_sample``.  Returns cand [B, n_nodes] (entries outside the range keep -1 / their input)."""
+    draft = np.ascontiguousarray(draft, dtype=np.float32)
+    B, n_internal, V = draft.shape
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    n_nodes = parent.shape[0]
+    unif_draw = np.ascontiguousarray(unif_draw, dtype=np.float32)
+    assert unif_draw.shape == (B, n_nodes)
+    node_end = n_internal if node_end is None else node_end
+    out = np.full((B, n_nodes), -1, dtype=np.int32) if cand is None else np.ascontiguousarray(cand, dtype=np.int32)
+    rc = _load().mcsd_oracle_sample(B, n_nodes, n_internal, V, _ptr(draft), _ptr(parent), _ptr(unif_draw),
+                                    float(T), int(mode), int(node_begin), int(node_end), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"mcsd_oracle_sample rejected its arguments (code {rc})")
+    return out
 
 
 @dataclass

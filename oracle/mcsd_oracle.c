@@ -16,6 +16,8 @@
  *     algorithm on that node's (p, q, candidates); move to the accepted child or
  *     stop; a node where everything is rejected returns a token from the final
  *     residual; a leaf returns a token from its own target distribution.
+ *   - Section 3.2, Eq. 1 (how the k candidates of a node are drawn without replacement);
+ *     the draws themselves are made deterministic by supplied uniforms.
  *   - Section 4.1 (sampling setups): temperature 1 is plain softmax sampling,
  *     temperature 0 is argmax.  Section 4.4 states that at temperature 0 the
  *     with-replacement algorithm degenerates to standard speculative decoding and
@@ -168,6 +170,86 @@ int32_t mcsd_oracle_mcss(double *p, double *q, int32_t V, const int32_t *cand,
         }
     }
     return -1;
+}
+
+/*
+ * Drawing the k candidates of one node from the draft distribution q (Section 3.2).
+ *   mode 0: k independent draws from q (sampling with replacement, the input of
+ *           Algorithm 1): x_i is the inverse-CDF image of u[i] under q.
+ *   mode 1: sampling without replacement, Eq. 1: x_1 is drawn from q; before each later
+ *           draw the tokens already drawn get probability 0 and the rest is renormalised
+ *           (the inverse CDF works on unnormalised weights, so zeroing is enough).
+ * q [V] is used as scratch in mode 1 (drawn entries are zeroed).  Returns the number of
+ * draws that found no mass (their token is -1).
+ */
+int32_t mcsd_oracle_draw(double *q, int32_t V, const double *u, int32_t k, int32_t mode, int32_t *x_out)
+{
+    int32_t failed = 0;
+    for (int32_t i = 0; i < k; ++i) {
+        int32_t x = mcsd_oracle_invcdf(q, V, u[i]);
+        x_out[i] = x;
+        if (x < 0) { ++failed; continue; }
+        if (mode == 1) q[x] = 0.0;
+    }
+    return failed;
+}
+
+/* The k largest logits in descending order, equal logits by ascending index: what the
+ * draws of a node become at temperature 0 (every draw takes the most probable token that
+ * is still available). */
+void mcsd_oracle_topk(const float *logits, int32_t V, int32_t k, int32_t *x_out)
+{
+    for (int32_t i = 0; i < k; ++i) {
+        int32_t best = -1;
+        for (int32_t x = 0; x < V; ++x) {
+            int32_t taken = 0;
+            for (int32_t j = 0; j < i; ++j) taken |= (x_out[j] == x);
+            if (taken) continue;
+            if (best < 0 || (double)logits[x] > (double)logits[best]) best = x;
+        }
+        x_out[i] = best;
+    }
+}
+
+/*
+ * Candidate tokens of every child of the nodes [node_begin, node_end) of every tree.
+ *   draft  [B][n_internal][V]  float32 draft logits
+ *   unif   [B][n_nodes]        the uniform that draws the token of each draft node
+ *   cand   [B][n_nodes]        out: cand[b][c] for every child c of the nodes in range;
+ *                              other entries are left untouched
+ * T > 0: draws from softmax(draft / T) as in mcsd_oracle_draw; T == 0: top-k.
+ * Returns 0, or -1 on malformed arguments.
+ */
+int32_t mcsd_oracle_sample(int32_t B, int32_t n_nodes, int32_t n_internal, int32_t V,
+                           const float *draft, const int32_t *parent, const float *unif, double T,
+                           int32_t mode, int32_t node_begin, int32_t node_end, int32_t *cand)
+{
+    if (B < 0 || n_nodes < 1 || V < 1 || n_internal < 0 || n_internal > n_nodes) return -1;
+    if (!(T >= 0.0) || (mode != 0 && mode != 1)) return -1;
+    if (node_begin < 0 || node_end > n_internal || node_begin > node_end) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t b = 0; b < B; ++b) {
+        double *q = (double *)malloc((size_t)V * sizeof(double));
+        for (int32_t n = node_begin; n < node_end; ++n) {
+            int32_t first = -1, k = 0;
+            for (int32_t c = n + 1; c < n_nodes; ++c)
+                if (parent[c] == n) { if (k == 0) first = c; ++k; }
+            if (k == 0 || k > 64) continue;
+            const float *d = draft + ((size_t)b * n_internal + n) * V;
+            int32_t x[64];
+            if (T == 0.0) {
+                mcsd_oracle_topk(d, V, k, x);
+            } else {
+                double u[64];
+                for (int32_t i = 0; i < k; ++i) u[i] = (double)unif[(size_t)b * n_nodes + first + i];
+                mcsd_oracle_softmax(d, V, T, q);
+                mcsd_oracle_draw(q, V, u, k, mode, x);
+            }
+            for (int32_t i = 0; i < k; ++i) cand[(size_t)b * n_nodes + first + i] = x[i];
+        }
+        free(q);
+    }
+    return 0;
 }
 
 /* Children of node n in a level-ordered tree: the contiguous run of nodes whose

@@ -8,6 +8,7 @@ import pytest
 
 import oracle
 import test_oracle_pins as pins
+import test_oracle_sample_pins as spins
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "mcsd_oracle.c")
 
@@ -53,6 +54,18 @@ MUTANTS = [
      [pins.test_output_marginal_through_verify_on_uniform_grid]),
     ("t0_accepts_any_candidate", "int32_t match = cand_b[first + i] == a;", "int32_t match = 1;",
      [pins.test_temperature_zero_is_greedy_matching]),
+    ("eq1_drawn_token_not_removed", "if (mode == 1) q[x] = 0.0;", ";",
+     [spins.test_hand_computed_draws_without_replacement]),
+    ("eq1_removal_applied_with_replacement", "if (mode == 1) q[x] = 0.0;", "q[x] = 0.0;",
+     [spins.test_draws_with_replacement_reproduce_q]),
+    ("draw_uses_wrong_uniform", "int32_t x = mcsd_oracle_invcdf(q, V, u[i]);", "int32_t x = mcsd_oracle_invcdf(q, V, u[0]);",
+     [spins.test_hand_computed_draws_without_replacement]),
+    ("topk_ascending", "(double)logits[x] > (double)logits[best]) best = x;", "(double)logits[x] < (double)logits[best]) best = x;",
+     [spins.test_temperature_zero_is_top_k_with_lowest_index_on_ties]),
+    ("topk_highest_index_on_ties", "(double)logits[x] > (double)logits[best]) best = x;", "(double)logits[x] >= (double)logits[best]) best = x;",
+     [spins.test_temperature_zero_is_top_k_with_lowest_index_on_ties]),
+    ("sample_children_of_wrong_node", "const float *d = draft + ((size_t)b * n_internal + n) * V;", "const float *d = draft + ((size_t)b * n_internal) * V;",
+     [lambda: spins.test_tree_level_routine_is_the_node_routine_in_child_order(1, 0.7)]),
 ]
 
 
