@@ -185,6 +185,29 @@ int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const voi
                      int32_t *out_tokens, float *out_residual);
 
 /*
+ * The step before verification: drawing the candidate tokens (Section 3.2).  For every
+ * node n in [node_begin, node_end) of every tree (node indices < n_internal) the tokens
+ * of its k children are drawn from softmax(draft_logits[b][n] / temperature) by inverse
+ * CDF in token order (see "Endpoint draw" above), child c with the uniform
+ * uniforms_draw[b][c]:
+ *   MCSD_MODE_WITH_REPLACEMENT     k independent draws (the input of Algorithm 1)
+ *   MCSD_MODE_WITHOUT_REPLACEMENT  Eq. 1: every drawn token gets probability 0 before the
+ *                                  next draw, so the k tokens are distinct
+ *   temperature 0                  the k largest draft logits in descending order, lowest
+ *                                  index first among equals; uniforms_draw may be NULL
+ * A draft model produces the rows of one tree level at a time, hence the node range.
+ *   draft_logits   device [B][n_internal][ld_draft]
+ *   tree_parent    HOST   [n_nodes]
+ *   uniforms_draw  device [B][n_nodes] float32 in (0, 1)
+ *   cand_tokens    device [B][n_nodes], written for the children of the nodes in range
+ * Of the descriptor only batch, n_nodes, n_internal, vocab, dtype, ld_draft, stream and
+ * out_status (MCSD_STATUS_NO_MASS if a draw finds no mass; not cleared here) are read.
+ */
+int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, const int32_t *tree_parent,
+                           const float *uniforms_draw, float temperature, int replacement_mode,
+                           int32_t node_begin, int32_t node_end, int32_t *cand_tokens);
+
+/*
  * The same step for callers whose data lives in HOST memory: every pointer below
  * is a host pointer.  The library allocates device buffers for a slice of the
  * batch, copies the slice in, verifies it and copies the results back, slice

@@ -192,3 +192,48 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
         if status is not None and int(status[b]) != int(ref.status[b]):
             fail(f"seq {b}: status {int(status[b])}, oracle {int(ref.status[b])}")
     return rep
+
+
+@dataclass
+class SampleReport:
+    n_draws: int = 0
+    n_tolerated: int = 0      # first differing draw of a node lies within NEAR_TIE of a CDF boundary
+    failures: List[str] = field(default_factory=list)
+
+    @property
+    def ok(self) -> bool:
+        return not self.failures
+
+
+def compare_samples(draft, parent, unif_draw, T: float, mode: int, cand, node_begin: int = 0, node_end=None,
+                    max_failures: int = 20) -> SampleReport:
+    """Candidate tokens drawn by another implementation against the oracle's (Section 3.2, Eq. 1).
+    Tokens must be identical, except that at the first differing draw of a node the other token is
+    accepted if it has positive probability under the distribution of that draw and the uniform lies
+    within NEAR_TIE (CDF units) of its interval; the later draws of that node (which depend on the
+    earlier ones when drawing without replacement) are then not compared.  Temperature 0: exact."""
+    from . import sample as oracle_sample
+    parent = np.asarray(parent, dtype=np.int32)
+    B, n_internal, V = draft.shape
+    node_end = n_internal if node_end is None else node_end
+    ref = oracle_sample(draft, parent, unif_draw, T, mode, node_begin, node_end)
+    first, count = _children(parent)
+    rep = SampleReport()
+    for b in range(B):
+        for n in range(node_begin, node_end):
+            ch = np.arange(first[n], first[n] + count[n])
+            rep.n_draws += len(ch)
+            if np.array_equal(cand[b, ch], ref[b, ch]):
+                continue
+            i = int(np.argmax(cand[b, ch] != ref[b, ch]))
+            g, okk = int(cand[b, ch[i]]), False
+            if T > 0:
+                q = oracle_softmax(draft[b, n], T)
+                if mode == 1:
+                    q[ref[b, ch[:i]]] = 0.0      # the tokens drawn before (identical on both sides)
+                okk = _bonus_tolerated(q, g, float(unif_draw[b, ch[i]]))
+            if okk:
+                rep.n_tolerated += 1
+            elif len(rep.failures) < max_failures:
+                rep.failures.append(f"seq {b} node {n} draw {i}: token {g}, oracle {int(ref[b, ch[i]])}")
+    return rep

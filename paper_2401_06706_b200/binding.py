@@ -22,7 +22,7 @@ MCSD_DTYPE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 STATUS_DEGENERATE, STATUS_BAD_TOKEN, STATUS_NO_MASS, STATUS_TIMEOUT = 1, 2, 4, 8
 MAX_NODES, MAX_CHILDREN, MAX_VOCAB = 512, 32, 65536
 
-EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path",
+EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path", "mcsd_sample_candidates",
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
            "mcsd_version")
 
@@ -62,6 +62,8 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_verify.restype = ctypes.c_int
     lib.mcsd_verify_path.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
     lib.mcsd_verify_path.restype = ctypes.c_int
+    lib.mcsd_sample_candidates.argtypes = [dp, vp, vp, vp, f32, ctypes.c_int, i32, i32, vp]
+    lib.mcsd_sample_candidates.restype = ctypes.c_int
     lib.mcsd_verify_static.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
     lib.mcsd_verify_static.restype = ctypes.c_int
     lib.mcsd_verify_nodes.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int]
@@ -255,6 +257,30 @@ def mcsd_verify(target, draft, parent, cand, unif, temperature: float, mode: int
     v = Verifier(B, parent, V, target.dtype, target.device, want_residual=want_residual,
                  node_outputs=node_outputs)
     return v.mcsd_verify(target, draft, cand, unif, temperature, mode)
+
+
+def mcsd_sample_candidates(draft, parent, unif_draw, temperature: float, mode: int, *, node_begin: int = 0,
+                           node_end: Optional[int] = None, cand: Optional[torch.Tensor] = None,
+                           status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Candidate tokens of the children of nodes [node_begin, node_end): device tensors in, the
+    [B, n_nodes] int32 token tensor out (entries outside the range keep their value, -1 if new)."""
+    lib = load_library()
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    B, n_internal, V = draft.shape
+    n_nodes = int(parent.shape[0])
+    d = McsdDesc()
+    d.batch, d.n_nodes, d.n_internal, d.vocab = B, n_nodes, n_internal, V
+    d.dtype = MCSD_DTYPE[draft.dtype]
+    d.ld_target = V
+    d.ld_draft = _row_stride(draft) if n_internal else V
+    d.stream = torch.cuda.current_stream(draft.device).cuda_stream
+    d.out_status = _ptr(status)
+    if cand is None:
+        cand = torch.full((B, n_nodes), -1, dtype=torch.int32, device=draft.device)
+    _check(lib.mcsd_sample_candidates(ctypes.byref(d), _ptr(draft), parent.ctypes.data, _ptr(unif_draw),
+                                      float(temperature), int(mode), int(node_begin),
+                                      int(n_internal if node_end is None else node_end), _ptr(cand)))
+    return cand
 
 
 def mcsd_verify_host(target, draft, parent, cand, unif, temperature: float, mode: int, *,

@@ -526,6 +526,47 @@ int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const voi
                        out_tokens, out_residual, false);
 }
 
+int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, const int32_t *tree_parent,
+                           const float *uniforms_draw, float temperature, int replacement_mode,
+                           int32_t node_begin, int32_t node_end, int32_t *cand_tokens)
+{
+    int rc = check_desc(desc);
+    if (rc != MCSD_OK) return rc;
+    TreePlan plan;
+    rc = plan_tree(tree_parent, desc->n_nodes, desc->n_internal, &plan);
+    if (rc != MCSD_OK) return rc;
+    if (!(temperature >= 0.f) || std::isinf(temperature)) return MCSD_ERR_TEMPERATURE;
+    if (replacement_mode != MCSD_MODE_WITH_REPLACEMENT && replacement_mode != MCSD_MODE_WITHOUT_REPLACEMENT)
+        return MCSD_ERR_MODE;
+    if (node_begin < 0 || node_end > desc->n_internal || node_begin > node_end) return MCSD_ERR_SHAPE;
+    g_last_launches = 0;
+    const long long n_ctas = static_cast<long long>(desc->batch) * (node_end - node_begin);
+    if (n_ctas == 0) return MCSD_OK;
+    if (!draft_logits || !cand_tokens || (temperature > 0.f && !uniforms_draw)) return MCSD_ERR_NULL;
+    if (desc->ld_draft < desc->vocab) return MCSD_ERR_STRIDE;
+    if (n_ctas > 0x7fffffffLL) return MCSD_ERR_UNSUPPORTED;
+    SampleParams p = {};
+    p.draft = draft_logits; p.unif_draw = uniforms_draw; p.cand = cand_tokens; p.status = desc->out_status;
+    p.ld_d = desc->ld_draft;
+    p.n_nodes = desc->n_nodes; p.n_internal = desc->n_internal; p.V = desc->vocab;
+    p.node_begin = node_begin; p.n_range = node_end - node_begin;
+    p.mode = replacement_mode;
+    p.vector_ok = rows_aligned16(draft_logits, desc->ld_draft, desc->dtype) ? 1 : 0;
+    p.scale = temperature > 0.f ? static_cast<float>(1.4426950408889634 / static_cast<double>(temperature)) : 0.f;
+    std::memcpy(p.child_first, plan.child_first, sizeof(p.child_first));
+    std::memcpy(p.child_count, plan.child_count, sizeof(p.child_count));
+    cudaStream_t stream = static_cast<cudaStream_t>(desc->stream);
+    const unsigned grid = static_cast<unsigned>(n_ctas);
+    switch (desc->dtype) {
+    case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32><<<grid, kWalkThreads, 0, stream>>>(p); break;
+    case MCSD_DTYPE_BF16: sample_kernel<MCSD_DTYPE_BF16><<<grid, kWalkThreads, 0, stream>>>(p); break;
+    default: sample_kernel<MCSD_DTYPE_F16><<<grid, kWalkThreads, 0, stream>>>(p); break;
+    }
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches = 1;
+    return MCSD_OK;
+}
+
 // ---- mcsd_verify_static: the scratch memory is an array built into the library --------
 // In host code the name below is only a handle for the runtime; the address kernels can
 // use comes from cudaGetSymbolAddress, looked up once per device.
