@@ -306,6 +306,21 @@ static int32_t verify_node(int32_t n, int32_t n_nodes, int32_t n_internal, int32
         return -1;
     }
     mcsd_oracle_softmax(t, V, T, residual); /* p */
+    if (mode == 2 && k > 0) {
+        /* Naive sampling (the baseline of Section 2 that Section 4.4 and Appendix C compare
+         * with): draw x from the target distribution itself; if one of the candidates
+         * carries x the walk moves to (the first) such child, otherwise x is the endpoint
+         * token.  The draft distribution plays no part. */
+        int32_t x = mcsd_oracle_invcdf(residual, V, (double)unif_b[2 * n + 1]);
+        if (x < 0) { *status |= ORACLE_STATUS_NO_MASS; *bonus = -1; return -1; }
+        for (int32_t i = 0; i < k; ++i) {
+            int32_t match = cand_b[first + i] == x;
+            if (ratio_b) ratio_b[first + i] = match ? 1.0 : 0.0;
+            if (match) { *bonus = -1; return first + i; }
+        }
+        *bonus = x;
+        return -1;
+    }
     if (k == 0) {
         /* leaf: endpoint from its own target distribution */
         *bonus = mcsd_oracle_invcdf(residual, V, (double)unif_b[2 * n + 1]);
@@ -344,6 +359,8 @@ static int32_t verify_node(int32_t n, int32_t n_nodes, int32_t n_internal, int32
  *   unif    [B][n_nodes][2]     [..][0]: uniform of the test of node n as a
  *                               candidate; [..][1]: uniform of the endpoint draw
  *                               when the walk stops at n
+ *   mode 0 / 1: Algorithm 1 / Algorithm 2; mode 2: naive sampling (draw from the target
+ *   distribution, accept if a candidate carries the drawn token; draft unused, may be NULL)
  *   sequential = 0: evaluate every node, then walk (the data-parallel form);
  *   sequential = 1: the paper's literal procedure, evaluating only the nodes the
  *                   walk stands on.  Per-node outputs of unvisited nodes are then
@@ -367,7 +384,7 @@ int32_t mcsd_oracle_verify(int32_t B, int32_t n_nodes, int32_t n_internal, int32
                            int32_t *node_bonus, double *node_ratio, int32_t *out_status)
 {
     if (B < 0 || n_nodes < 1 || V < 1 || n_internal < 0 || n_internal > n_nodes) return -1;
-    if (!(T >= 0.0) || (mode != 0 && mode != 1)) return -1;
+    if (!(T >= 0.0) || (mode != 0 && mode != 1 && mode != 2)) return -1;
     if (parent[0] != -1) return -1;
     for (int32_t n = 1; n < n_nodes; ++n)
         if (parent[n] < 0 || parent[n] >= n || parent[n] < parent[n - 1]) return -1;
@@ -376,7 +393,7 @@ int32_t mcsd_oracle_verify(int32_t B, int32_t n_nodes, int32_t n_internal, int32
         if (k > 64) return -1;
         if ((k > 0) != (n < n_internal)) return -1;
     }
-    if (T > 0.0 && n_internal > 0 && !draft) return -1;
+    if (T > 0.0 && mode != 2 && n_internal > 0 && !draft) return -1;
     const int32_t gamma = tree_depth(parent, n_nodes);
     int32_t fail = 0;
 

@@ -9,6 +9,7 @@ import pytest
 import oracle
 import test_oracle_pins as pins
 import test_oracle_sample_pins as spins
+import test_oracle_mcns_pins as npins
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "mcsd_oracle.c")
 
@@ -64,6 +65,13 @@ MUTANTS = [
      [spins.test_temperature_zero_is_top_k_with_lowest_index_on_ties]),
     ("topk_highest_index_on_ties", "(double)logits[x] > (double)logits[best]) best = x;", "(double)logits[x] >= (double)logits[best]) best = x;",
      [spins.test_temperature_zero_is_top_k_with_lowest_index_on_ties]),
+    ("naive_draw_uses_acceptance_uniform", "int32_t x = mcsd_oracle_invcdf(residual, V, (double)unif_b[2 * n + 1]);\n        if (x < 0) { *status",
+     "int32_t x = mcsd_oracle_invcdf(residual, V, (double)unif_b[2 * n]);\n        if (x < 0) { *status",
+     [npins.test_emitted_token_is_a_draw_from_p_and_accepted_iff_a_candidate_carries_it]),
+    ("naive_match_inverted", "int32_t match = cand_b[first + i] == x;", "int32_t match = cand_b[first + i] != x;",
+     [npins.test_emitted_token_is_a_draw_from_p_and_accepted_iff_a_candidate_carries_it]),
+    ("naive_endpoint_not_the_draw", "        *bonus = x;\n        return -1;", "        *bonus = cand_b[first];\n        return -1;",
+     [npins.test_walk_over_levels_and_leaf_endpoint]),
     ("sample_children_of_wrong_node", "const float *d = draft + ((size_t)b * n_internal + n) * V;", "const float *d = draft + ((size_t)b * n_internal) * V;",
      [lambda: spins.test_tree_level_routine_is_the_node_routine_in_child_order(1, 0.7)]),
 ]
