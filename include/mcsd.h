@@ -58,6 +58,12 @@ extern "C" {
 /* replacement_mode */
 #define MCSD_MODE_WITH_REPLACEMENT 0    /* Algorithm 1 */
 #define MCSD_MODE_WITHOUT_REPLACEMENT 1 /* Algorithm 2 */
+#define MCSD_MODE_NAIVE 2 /* multi-candidate naive sampling, the ablation baseline of Section 4.4:
+                             draw x from the target distribution (second uniform of the node);
+                             accept the first child that carries x, else x is the endpoint token.
+                             mcsd_verify, mcsd_verify_path and mcsd_verify_host only; draft_logits
+                             are not read and may be NULL; out_residual is the stopping node's
+                             target distribution; per-node outputs cover visited nodes */
 
 /* limits */
 #define MCSD_MAX_NODES 512     /* nodes per tree, root included            */

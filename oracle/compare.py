@@ -17,6 +17,8 @@ Rules
     if it has positive oracle probability and u lies within NEAR_TIE (in CDF
     units) of that token's oracle CDF interval.  Such cases are counted.
   * Residual distributions agree within `residual_tol` max abs error.
+  * Naive sampling (mode 2): every emitted token is such a draw; the first differing token of a
+    sequence is judged by the endpoint rule and the rest of that sequence is skipped.
 """
 from __future__ import annotations
 
@@ -169,6 +171,21 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
             rep.n_excluded_sequences += 1
             continue
         L = int(ref.accept_len[b])
+        if mode == 2 and T > 0 and not np.array_equal(tokens[b], ref.tokens[b]):
+            # naive sampling: every emitted token is itself a draw by inverse CDF.  At the first
+            # position where the token sequences differ, the other token passes under the same
+            # rule as an endpoint token; what follows depends on it and is not compared.
+            i = int(np.argmax(tokens[b] != ref.tokens[b]))
+            node = 0
+            for _ in range(i):
+                node = int(ref.node_accept[b, node])
+            if node >= 0 and _bonus_tolerated(oracle_softmax(target[b, node], T), int(tokens[b, i]),
+                                              float(unif[b, node, 1])):
+                rep.n_bonus_tolerated += 1
+                rep.n_excluded_sequences += 1
+            else:
+                fail(f"seq {b}: tokens {tokens[b].tolist()}, oracle {ref.tokens[b].tolist()}")
+            continue
         if int(accept_len[b]) != L:
             fail(f"seq {b}: accepted length {int(accept_len[b])}, oracle {L}")
             continue

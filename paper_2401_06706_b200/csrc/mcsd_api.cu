@@ -256,14 +256,16 @@ int prepare(const mcsd_desc *d, const int32_t *parent, Call *c)
 }
 
 int check_common(const mcsd_desc *d, const void *target, const void *draft, const int32_t *cand,
-                 const float *unif, float T, int mode, bool need_unif)
+                 const float *unif, float T, int mode, bool need_unif, bool naive_ok = false)
 {
     if (!target || !cand) return MCSD_ERR_NULL;
     if (!(T >= 0.f) || std::isinf(T)) return MCSD_ERR_TEMPERATURE;
-    if (mode != MCSD_MODE_WITH_REPLACEMENT && mode != MCSD_MODE_WITHOUT_REPLACEMENT) return MCSD_ERR_MODE;
+    if (mode != MCSD_MODE_WITH_REPLACEMENT && mode != MCSD_MODE_WITHOUT_REPLACEMENT &&
+        !(naive_ok && mode == MCSD_MODE_NAIVE))
+        return MCSD_ERR_MODE;
     if (T > 0.f) {
         if (need_unif && !unif) return MCSD_ERR_NULL;
-        if (d->n_internal > 0) {
+        if (d->n_internal > 0 && mode != MCSD_MODE_NAIVE) {
             if (!draft) return MCSD_ERR_NULL;
             if (d->ld_draft < d->vocab) return MCSD_ERR_STRIDE;
         }
@@ -361,6 +363,35 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         cudaGetLastError();
         return MCSD_ERR_CUDA;
     }
+    g_last_launches += 1;
+    return MCSD_OK;
+}
+
+// Naive sampling: one kernel walks every tree level by level (nothing else is launched).
+int launch_naive(const Call &c, const void *target, const int32_t *cand, const float *unif, float T,
+                 int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
+{
+    const mcsd_desc *d = c.d;
+    if (d->batch == 0) return MCSD_OK;
+    if (cudaMemsetAsync(c.status, 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess) return MCSD_ERR_CUDA;
+    NaiveParams p = {};
+    p.target = target; p.cand = cand; p.unif = unif;
+    p.node_accept = c.node_accept;
+    p.out_accept_len = out_accept_len; p.out_tokens = out_tokens; p.out_residual = out_residual;
+    p.status = c.status;
+    p.ld_t = d->ld_target;
+    p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab; p.gamma = c.plan.gamma;
+    p.vector_ok = rows_aligned16(target, d->ld_target, d->dtype) ? 1 : 0;
+    p.scale = static_cast<float>(1.4426950408889634 / static_cast<double>(T));
+    std::memcpy(p.child_first, c.plan.child_first, sizeof(p.child_first));
+    std::memcpy(p.child_count, c.plan.child_count, sizeof(p.child_count));
+    const unsigned grid = static_cast<unsigned>(d->batch);
+    switch (d->dtype) {
+    case MCSD_DTYPE_F32: naive_kernel<MCSD_DTYPE_F32><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
+    case MCSD_DTYPE_BF16: naive_kernel<MCSD_DTYPE_BF16><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
+    default: naive_kernel<MCSD_DTYPE_F16><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
+    }
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
     g_last_launches += 1;
     return MCSD_OK;
 }
@@ -493,9 +524,16 @@ int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *dr
     g_last_launches = 0;
     if (desc->batch == 0) return MCSD_OK;
     rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
-                      replacement_mode, true);
+                      replacement_mode, true, true);
     if (rc != MCSD_OK) return rc;
     if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
+    if (replacement_mode == MCSD_MODE_NAIVE) {
+        // at temperature 0 the draw is the target argmax: the ordinary argmax rule
+        if (temperature > 0.f)
+            return launch_naive(c, target_logits, cand_tokens, uniforms, temperature, out_accept_len, out_tokens,
+                                out_residual);
+        replacement_mode = MCSD_MODE_WITH_REPLACEMENT;
+    }
     rc = launch_nodes(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, replacement_mode);
     if (rc != MCSD_OK) return rc;
     return launch_walk(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, out_accept_len,
@@ -513,9 +551,16 @@ int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const voi
     g_last_launches = 0;
     if (desc->batch == 0) return MCSD_OK;
     rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
-                      replacement_mode, true);
+                      replacement_mode, true, true);
     if (rc != MCSD_OK) return rc;
     if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
+    if (replacement_mode == MCSD_MODE_NAIVE) {
+        // at temperature 0 the draw is the target argmax: the ordinary argmax rule
+        if (temperature > 0.f)
+            return launch_naive(c, target_logits, cand_tokens, uniforms, temperature, out_accept_len, out_tokens,
+                                out_residual);
+        replacement_mode = MCSD_MODE_WITH_REPLACEMENT;
+    }
     // one launch per level of the tree: level l evaluates, for every sequence, the node its
     // walk stands on after l accepted tokens (nothing for walks that have ended)
     for (int level = 0; level <= c.plan.gamma; ++level) {
@@ -625,14 +670,14 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
     rc = plan_tree(tree_parent, desc->n_nodes, desc->n_internal, &plan);
     if (rc != MCSD_OK) return rc;
     rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
-                      replacement_mode, true);
+                      replacement_mode, true, true);
     if (rc != MCSD_OK) return rc;
     if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
     const int B = desc->batch;
     if (B == 0) return MCSD_OK;
 
     const size_t es = elem_bytes(desc->dtype);
-    const bool use_draft = temperature > 0.f && desc->n_internal > 0;
+    const bool use_draft = temperature > 0.f && desc->n_internal > 0 && replacement_mode != MCSD_MODE_NAIVE;
     const size_t t_seq = static_cast<size_t>(desc->n_nodes) * desc->ld_target * es;
     const size_t d_seq = use_draft ? static_cast<size_t>(desc->n_internal) * desc->ld_draft * es : 0;
     const size_t c_seq = sizeof(int32_t) * desc->n_nodes, u_seq = sizeof(float) * 2 * desc->n_nodes;
