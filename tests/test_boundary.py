@@ -100,7 +100,7 @@ def test_host_validation_codes(lib):
     assert call(d, parent, T=-0.5) == -5
     assert call(d, parent, T=float("nan")) == -5
     assert call(d, parent, T=float("inf")) == -5
-    assert call(d, parent, mode=2) == -4
+    assert call(d, parent, mode=3) == -4
     d2, _ = _desc(ws=ws); d2.dtype = 7
     assert call(d2, parent) == -3
     d2, _ = _desc(ws=ws); d2.vocab = 0
