@@ -114,6 +114,11 @@ typedef struct mcsd_desc {
     float *node_ratio;    /* [B][n_nodes] p/q seen by the test of each draft node; -1
                              for a forced rejection; untouched if never tested      */
     int32_t *out_status;  /* [B] MCSD_STATUS_* bits (device), NULL to skip            */
+    int32_t *out_path_nodes; /* [B][gamma+1] (device), NULL to skip: entry i < accept_len
+                             is the tree node whose token is out_tokens[i], the rest is
+                             -1.  With the flattened-tree layout of Section 3.3 (node n
+                             at sequence position prefix_len + n) these are the key/value
+                             cache rows that stay after verification.                */
 } mcsd_desc;
 
 /*
@@ -261,6 +266,20 @@ int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const v
                        const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                        float temperature, int replacement_mode, int32_t *out_accept_len,
                        int32_t *out_tokens, float *out_residual);
+
+/*
+ * Tree Attention layout (Section 3.3): the tree is fed to the target model as one flattened
+ * sequence in node order, every node attending only to itself and its ancestors (and to the
+ * whole prefix), with the position ids it would have in its own root-to-node sequence.
+ *   tree_parent   HOST   [n_nodes]
+ *   prefix_len    position id of the root (node 0 is the last committed token)
+ *   mask          device [n_nodes][n_nodes] bytes: mask[i][j] = 1 iff j == i or j is an
+ *                 ancestor of i, else 0
+ *   position_ids  device [n_nodes]: prefix_len + depth of the node
+ * Either output may be NULL.  stream: cudaStream_t the work is enqueued on.
+ */
+int mcsd_tree_attention_layout(const int32_t *tree_parent, int32_t n_nodes, int32_t prefix_len,
+                               uint8_t *mask, int32_t *position_ids, void *stream);
 
 /* Bytes of device workspace mcsd_verify needs for this descriptor (batch and
  * n_nodes are read); 0 if the descriptor is NULL or its shape is invalid. */

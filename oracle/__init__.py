@@ -207,3 +207,36 @@ def verify(target, draft, parent, cand, unif, T: float, mode: int, *, sequential
     if rc != 0:
         raise ValueError(f"mcsd_oracle_verify rejected its arguments (code {rc})")
     return VerifyResult(accept_len, tokens, residual, node_accept, node_bonus, node_ratio, status)
+
+
+def tree_attention_layout(parent, prefix_len: int):
+    """Section 3.3 written out: mask[i][j] = 1 iff j is i or an ancestor of i (the reflexive and
+    transitive closure of the parent relation, by following parents), position id = prefix_len +
+    depth.  Returns (mask uint8 [n, n], position_ids int32 [n])."""
+    parent = np.asarray(parent, dtype=np.int64)
+    n = parent.shape[0]
+    mask = np.zeros((n, n), dtype=np.uint8)
+    pos = np.zeros(n, dtype=np.int32)
+    for i in range(n):
+        a, depth = i, 0
+        while a >= 0:
+            mask[i, a] = 1
+            a = int(parent[a])
+            if a >= 0:
+                depth += 1
+        pos[i] = prefix_len + depth
+    return mask, pos
+
+
+def path_nodes(result: "VerifyResult", gamma: int) -> np.ndarray:
+    """Tree nodes of the accepted tokens of every sequence, -1 padded to gamma + 1 columns: the walk
+    of Section 3 followed through node_accept."""
+    B = result.accept_len.shape[0]
+    out = np.full((B, gamma + 1), -1, dtype=np.int32)
+    for b in range(B):
+        n, i = 0, 0
+        while result.node_accept[b, n] >= 0:
+            n = int(result.node_accept[b, n])
+            out[b, i] = n
+            i += 1
+    return out

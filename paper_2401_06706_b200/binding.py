@@ -22,7 +22,7 @@ MCSD_DTYPE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 STATUS_DEGENERATE, STATUS_BAD_TOKEN, STATUS_NO_MASS, STATUS_TIMEOUT = 1, 2, 4, 8
 MAX_NODES, MAX_CHILDREN, MAX_VOCAB = 512, 32, 65536
 
-EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path", "mcsd_sample_candidates",
+EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path", "mcsd_sample_candidates", "mcsd_tree_attention_layout",
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
            "mcsd_version")
 
@@ -34,7 +34,8 @@ class McsdDesc(ctypes.Structure):
                 ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
                 ("workspace_bytes", ctypes.c_size_t),
                 ("node_accept", ctypes.c_void_p), ("node_bonus", ctypes.c_void_p),
-                ("node_ratio", ctypes.c_void_p), ("out_status", ctypes.c_void_p)]
+                ("node_ratio", ctypes.c_void_p), ("out_status", ctypes.c_void_p),
+                ("out_path_nodes", ctypes.c_void_p)]
 
 
 class McsdError(RuntimeError):
@@ -64,6 +65,8 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_verify_path.restype = ctypes.c_int
     lib.mcsd_sample_candidates.argtypes = [dp, vp, vp, vp, f32, ctypes.c_int, i32, i32, vp]
     lib.mcsd_sample_candidates.restype = ctypes.c_int
+    lib.mcsd_tree_attention_layout.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.mcsd_tree_attention_layout.restype = ctypes.c_int
     lib.mcsd_verify_static.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
     lib.mcsd_verify_static.restype = ctypes.c_int
     lib.mcsd_verify_nodes.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int]
@@ -145,6 +148,7 @@ class VerifyOutput:
     node_accept: Optional[torch.Tensor] = None
     node_bonus: Optional[torch.Tensor] = None
     node_ratio: Optional[torch.Tensor] = None
+    path_nodes: Optional[torch.Tensor] = None  # [B, gamma+1] tree nodes of the accepted tokens, -1 padded
 
 
 class Verifier:
@@ -183,6 +187,8 @@ class Verifier:
                          if want_residual else None)
         self.status = torch.zeros(self.batch, **i32)
         d.out_status = self.status.data_ptr()
+        self.path_nodes = torch.empty((self.batch, self.gamma + 1), **i32)
+        d.out_path_nodes = self.path_nodes.data_ptr()
         self.node_accept = self.node_bonus = self.node_ratio = None
         if node_outputs:
             self.node_accept = torch.empty((self.batch, self.n_nodes), **i32)
@@ -203,7 +209,7 @@ class Verifier:
 
     def _out(self) -> VerifyOutput:
         return VerifyOutput(self.accept_len, self.tokens, self.residual, self.status, self.node_accept,
-                            self.node_bonus, self.node_ratio)
+                            self.node_bonus, self.node_ratio, self.path_nodes)
 
     def mcsd_verify(self, target, draft, cand, unif, temperature: float, mode: int) -> VerifyOutput:
         self._bind(target, draft)
@@ -257,6 +263,18 @@ def mcsd_verify(target, draft, parent, cand, unif, temperature: float, mode: int
     v = Verifier(B, parent, V, target.dtype, target.device, want_residual=want_residual,
                  node_outputs=node_outputs)
     return v.mcsd_verify(target, draft, cand, unif, temperature, mode)
+
+
+def mcsd_tree_attention_layout(parent, prefix_len: int, device="cuda"):
+    """Ancestor-only attention mask [n, n] (uint8) and position ids [n] (int32) of the flattened tree."""
+    lib = load_library()
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    n = int(parent.shape[0])
+    mask = torch.empty((n, n), dtype=torch.uint8, device=device)
+    pos = torch.empty(n, dtype=torch.int32, device=device)
+    _check(lib.mcsd_tree_attention_layout(parent.ctypes.data, n, int(prefix_len), _ptr(mask), _ptr(pos),
+                                          torch.cuda.current_stream(torch.device(device)).cuda_stream))
+    return mask, pos
 
 
 def mcsd_sample_candidates(draft, parent, unif_draw, temperature: float, mode: int, *, node_begin: int = 0,

@@ -378,6 +378,7 @@ int launch_naive(const Call &c, const void *target, const int32_t *cand, const f
     p.target = target; p.cand = cand; p.unif = unif;
     p.node_accept = c.node_accept;
     p.out_accept_len = out_accept_len; p.out_tokens = out_tokens; p.out_residual = out_residual;
+    p.out_path_nodes = d->out_path_nodes;
     p.status = c.status;
     p.ld_t = d->ld_target;
     p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab; p.gamma = c.plan.gamma;
@@ -407,6 +408,7 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
     p.node_accept = c.node_accept; p.node_bonus = c.node_bonus;
     p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part; p.status = c.status;
     p.out_accept_len = out_accept_len; p.out_tokens = out_tokens; p.out_residual = out_residual;
+    p.out_path_nodes = d->out_path_nodes;
     p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
     p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab; p.gamma = c.plan.gamma;
     p.scale = T > 0.f ? static_cast<float>(1.4426950408889634 / static_cast<double>(T)) : 0.f;
@@ -612,6 +614,23 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
     return MCSD_OK;
 }
 
+int mcsd_tree_attention_layout(const int32_t *tree_parent, int32_t n_nodes, int32_t prefix_len,
+                               uint8_t *mask, int32_t *position_ids, void *stream)
+{
+    TreePlan plan;
+    const int rc = plan_tree(tree_parent, n_nodes, -1, &plan);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (!mask && !position_ids) return MCSD_OK;
+    LayoutParams p = {};
+    p.mask = mask; p.position_ids = position_ids; p.n_nodes = n_nodes; p.prefix_len = prefix_len;
+    for (int n = 0; n < n_nodes; ++n) p.parent[n] = static_cast<int16_t>(tree_parent[n]);
+    layout_kernel<<<static_cast<unsigned>(n_nodes), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches = 1;
+    return MCSD_OK;
+}
+
 // ---- mcsd_verify_static: the scratch memory is an array built into the library --------
 // In host code the name below is only a handle for the runtime; the address kernels can
 // use comes from cudaGetSymbolAddress, looked up once per device.
@@ -698,7 +717,7 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
     } slot[2];
     mcsd_desc cd = *desc;
     cd.batch = chunk;
-    cd.node_accept = nullptr; cd.node_bonus = nullptr; cd.node_ratio = nullptr;
+    cd.node_accept = nullptr; cd.node_bonus = nullptr; cd.node_ratio = nullptr; cd.out_path_nodes = nullptr;
     const size_t ws_bytes = mcsd_workspace_bytes(&cd);
     bool ok = true;
     auto chk = [&](cudaError_t e) { if (e != cudaSuccess) ok = false; return e == cudaSuccess; };

@@ -1093,6 +1093,7 @@ struct WalkParams {
     int32_t *out_accept_len;
     int32_t *out_tokens;
     float *out_residual;  // may be null
+    int32_t *out_path_nodes;  // may be null
     int32_t *status;      // [B]
     long long ld_t, ld_d;
     int32_t n_nodes, n_internal, V, gamma;
@@ -1150,9 +1151,12 @@ walk_kernel(const __grid_constant__ WalkParams P)
                 if (nx <= n || nx >= P.n_nodes) break;
                 n = nx;
                 tok[len] = s_tok[n];
+                if (P.out_path_nodes) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + len] = n;
                 ++len;
             }
             for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
+            if (P.out_path_nodes)
+                for (int i = len; i <= P.gamma; ++i) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + i] = -1;
             P.out_accept_len[b] = len;
             s_term = n;
             s_len = len;
@@ -1572,6 +1576,7 @@ struct NaiveParams {
     int32_t *out_accept_len;
     int32_t *out_tokens;
     float *out_residual;    // may be null
+    int32_t *out_path_nodes;  // may be null
     int32_t *status;
     long long ld_t;
     int32_t n_nodes, n_internal, V, gamma;
@@ -1730,13 +1735,18 @@ naive_kernel(const __grid_constant__ NaiveParams P)
         __syncthreads();
         const int nx = s_next;
         if (nx <= n || nx >= P.n_nodes) break;
-        if (tid == 0) tok[len] = x;
+        if (tid == 0) {
+            tok[len] = x;
+            if (P.out_path_nodes) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + len] = nx;
+        }
         ++len;
         n = nx;
     }
     if (tid == 0) {
         tok[len] = x;
         for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
+        if (P.out_path_nodes)
+            for (int i = len; i <= P.gamma; ++i) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + i] = -1;
         P.out_accept_len[b] = len;
         if (x < 0) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
     }
@@ -1752,6 +1762,39 @@ naive_kernel(const __grid_constant__ NaiveParams P)
                 if (x0 + e < P.V) out[x0 + e] = w[e] * inv;
         }
     }
+}
+
+// ------------------------------------------------------------------ tree attention layout
+struct LayoutParams {
+    uint8_t *mask;          // [n_nodes][n_nodes] or null
+    int32_t *position_ids;  // [n_nodes] or null
+    int32_t n_nodes, prefix_len;
+    int16_t parent[MCSD_MAX_NODES];
+};
+
+// Section 3.3: row i of the mask marks node i and its ancestors; the position id of a node
+// is the root's plus its depth.  One CTA per node: thread 0 climbs to the root marking the
+// way in shared memory, then the CTA writes the row.
+__global__ void __launch_bounds__(kThreads)
+layout_kernel(const __grid_constant__ LayoutParams P)
+{
+    __shared__ uint8_t s_row[MCSD_MAX_NODES];
+    const int i = blockIdx.x;
+    for (int j = threadIdx.x; j < P.n_nodes; j += kThreads) s_row[j] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int depth = 0;
+        int a = i;
+        for (int hop = 0; hop < P.n_nodes && a >= 0; ++hop) {  // bounded even for a corrupt tree
+            s_row[a] = 1;
+            a = P.parent[a];
+            if (a >= 0) ++depth;
+        }
+        if (P.position_ids) P.position_ids[i] = P.prefix_len + depth;
+    }
+    __syncthreads();
+    if (P.mask)
+        for (int j = threadIdx.x; j < P.n_nodes; j += kThreads) P.mask[static_cast<long long>(i) * P.n_nodes + j] = s_row[j];
 }
 
 }  // namespace mcsd
