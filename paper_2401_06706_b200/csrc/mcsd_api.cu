@@ -604,10 +604,21 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
     std::memcpy(p.child_count, plan.child_count, sizeof(p.child_count));
     cudaStream_t stream = static_cast<cudaStream_t>(desc->stream);
     const unsigned grid = static_cast<unsigned>(n_ctas);
-    switch (desc->dtype) {
-    case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32><<<grid, kWalkThreads, 0, stream>>>(p); break;
-    case MCSD_DTYPE_BF16: sample_kernel<MCSD_DTYPE_BF16><<<grid, kWalkThreads, 0, stream>>>(p); break;
-    default: sample_kernel<MCSD_DTYPE_F16><<<grid, kWalkThreads, 0, stream>>>(p); break;
+    // 16 warps cover the row within the per-warp step budget (half of MCSD_MAX_VOCAB / 32 elements
+    // per warp at 1024 threads) when the vocabulary is at most half the maximum
+    const bool small = desc->vocab <= MCSD_MAX_VOCAB / 2;
+    if (small) {
+        switch (desc->dtype) {
+        case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32, 512><<<grid, 512, 0, stream>>>(p); break;
+        case MCSD_DTYPE_BF16: sample_kernel<MCSD_DTYPE_BF16, 512><<<grid, 512, 0, stream>>>(p); break;
+        default: sample_kernel<MCSD_DTYPE_F16, 512><<<grid, 512, 0, stream>>>(p); break;
+        }
+    } else {
+        switch (desc->dtype) {
+        case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32, 1024><<<grid, 1024, 0, stream>>>(p); break;
+        case MCSD_DTYPE_BF16: sample_kernel<MCSD_DTYPE_BF16, 1024><<<grid, 1024, 0, stream>>>(p); break;
+        default: sample_kernel<MCSD_DTYPE_F16, 1024><<<grid, 1024, 0, stream>>>(p); break;
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
     g_last_launches = 1;

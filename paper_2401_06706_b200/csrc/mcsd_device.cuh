@@ -1356,17 +1356,20 @@ struct SampleParams {
 // subtracting its weight from the partial sums of its lane, its warp's run and the
 // element scan.  The row is read once (twice for its maximum, the second time from L2);
 // temperature 0 takes the k largest logits instead (lowest index first on ties).
-template <int DT>
-__global__ void __launch_bounds__(kWalkThreads)
+// NT threads per CTA: 512 (two CTAs per SM, two independent chains) when the vocabulary fits
+// 16 steps per warp, else 1024.
+template <int DT, int NT>
+__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
 sample_kernel(const __grid_constant__ SampleParams P)
 {
     using E = Elem<DT>;
     constexpr int GV = E::kVec;
     constexpr int kStep = 32 * GV;
-    constexpr int kMaxSteps = MCSD_MAX_VOCAB / kWalkWarps / kStep;
-    __shared__ float s_wtot[kWalkWarps];
-    __shared__ float s_red[kWalkWarps];
-    __shared__ int s_redi[kWalkWarps];
+    constexpr int kW = NT / 32;  // warps
+    constexpr int kMaxSteps = MCSD_MAX_VOCAB / 32 / kStep;  // steps of a warp's run (the host picks NT so that they suffice)
+    __shared__ float s_wtot[32];
+    __shared__ float s_red[32];
+    __shared__ int s_redi[32];
     __shared__ int32_t s_rem_tok[MCSD_MAX_CHILDREN];
     __shared__ int s_pick;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1384,7 +1387,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
             for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
         }
     };
-    const int run = ((P.V + kWalkWarps - 1) / kWalkWarps + kStep - 1) / kStep * kStep;
+    const int run = ((P.V + kW - 1) / kW + kStep - 1) / kStep * kStep;
     const int x_lo = warp * run;
     int x_hi = x_lo + run;
     x_hi = x_hi > P.V ? P.V : x_hi;
@@ -1415,8 +1418,8 @@ sample_kernel(const __grid_constant__ SampleParams P)
             }
             if (lane == 0) { s_red[warp] = best; s_redi[warp] = best_i; }
             __syncthreads();
-            best = s_red[lane];
-            best_i = s_redi[lane];
+            best = lane < kW ? s_red[lane] : -INFINITY;
+            best_i = lane < kW ? s_redi[lane] : 0x7fffffff;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 const float ov = __shfl_xor_sync(0xffffffffu, best, o);
@@ -1442,7 +1445,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
     mx = warp_max(mx);
     if (lane == 0) s_red[warp] = mx;
     __syncthreads();
-    const float ref = int_ref(warp_max(s_red[lane]) * P.scale);
+    const float ref = int_ref(warp_max(lane < kW ? s_red[lane] : -INFINITY) * P.scale);
     const float ref0 = ref == -INFINITY ? 0.f : ref;
     auto weights = [&](int x0, float *w) {
         float v[GV];
@@ -1473,7 +1476,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
     for (int i = 0; i < k; ++i) {
         const float u = P.unif_draw[static_cast<long long>(b) * P.n_nodes + first + i];
         // the run that holds the quantile (every warp finds the same one)
-        const float m = s_wtot[lane];
+        const float m = lane < kW ? s_wtot[lane] : 0.f;
         const float total = warp_sum(m);
         const float target = u * total;
         const float inc = warp_scan_incl(m, lane);
