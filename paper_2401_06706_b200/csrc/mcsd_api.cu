@@ -428,10 +428,18 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
     for (int all = (T > 0.f && d->node_bonus && all_nodes_allowed) ? 1 : 0; all >= 0; --all) {
         p.all_nodes = all;
         const unsigned grid = static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch);
-        switch (d->dtype) {
-        case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
-        case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
-        default: walk_kernel<MCSD_DTYPE_F16><<<grid, kWalkThreads, 0, c.stream>>>(p); break;
+        if (d->vocab <= MCSD_MAX_VOCAB / 2) {
+            switch (d->dtype) {
+            case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32, 512><<<grid, 512, 0, c.stream>>>(p); break;
+            case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16, 512><<<grid, 512, 0, c.stream>>>(p); break;
+            default: walk_kernel<MCSD_DTYPE_F16, 512><<<grid, 512, 0, c.stream>>>(p); break;
+            }
+        } else {
+            switch (d->dtype) {
+            case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32, 1024><<<grid, 1024, 0, c.stream>>>(p); break;
+            case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16, 1024><<<grid, 1024, 0, c.stream>>>(p); break;
+            default: walk_kernel<MCSD_DTYPE_F16, 1024><<<grid, 1024, 0, c.stream>>>(p); break;
+            }
         }
         if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
         g_last_launches += 1;

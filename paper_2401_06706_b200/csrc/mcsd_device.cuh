@@ -1114,15 +1114,18 @@ constexpr int kWalkWarps = kWalkThreads / 32;
 // draws the token by inverse CDF in token order with that node's second uniform:
 // warp totals of contiguous runs -> the run holding the quantile -> that warp walks its
 // run again, 128 elements at a time.
-template <int DT>
-__global__ void __launch_bounds__(kWalkThreads)
+// NT threads per CTA: 512 (two CTAs per SM) when the vocabulary is at most half the maximum,
+// else 1024; a warp's run is at most MCSD_MAX_VOCAB / 32 elements either way.
+template <int DT, int NT>
+__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
 walk_kernel(const __grid_constant__ WalkParams P)
 {
     using E = Elem<DT>;
     constexpr int GV = E::kVec;
     __shared__ int s_term, s_len;
     __shared__ int32_t s_acc[MCSD_MAX_NODES], s_tok[MCSD_MAX_NODES];
-    __shared__ float s_wtot[kWalkWarps];
+    constexpr int kW = NT / 32;  // warps
+    __shared__ float s_wtot[32];
     __shared__ float s_leaf[2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int b, n;
@@ -1139,7 +1142,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
     if (!P.all_nodes) {
         // the tree's decisions and tokens come into shared memory with one parallel load, so
         // that the walk itself is not a chain of dependent global loads
-        for (int i = tid; i < P.n_nodes; i += kWalkThreads) {
+        for (int i = tid; i < P.n_nodes; i += NT) {
             s_acc[i] = P.node_accept[nb + i];
             s_tok[i] = P.cand[nb + i];
         }
@@ -1176,7 +1179,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
         const int a = P.node_bonus[nb + n];
         if (tid == 0 && !P.all_nodes) tok[len] = a;
         if (out)
-            for (int x = tid; x < P.V; x += kWalkThreads) out[x] = (x == a) ? 1.f : 0.f;
+            for (int x = tid; x < P.V; x += NT) out[x] = (x == a) ? 1.f : 0.f;
         return;
     }
 
@@ -1230,14 +1233,14 @@ walk_kernel(const __grid_constant__ WalkParams P)
 
     // contiguous runs: warp w owns [w * run, (w + 1) * run), walked 32 * GV elements at a time
     constexpr int kStep = 32 * GV;
-    const int run = ((P.V + kWalkWarps - 1) / kWalkWarps + kStep - 1) / kStep * kStep;
+    const int run = ((P.V + kW - 1) / kW + kStep - 1) / kStep * kStep;
     const int x_lo = warp * run;
     int x_hi = x_lo + run;
     x_hi = x_hi > P.V ? P.V : x_hi;
 
     // pass 1: the distribution itself, the mass of every run, and per lane the mass of its
     // group in every step of the run (kept for the search below)
-    constexpr int kMaxSteps = MCSD_MAX_VOCAB / kWalkWarps / kStep;
+    constexpr int kMaxSteps = MCSD_MAX_VOCAB / 32 / kStep;
     float g[kMaxSteps];
     float mass = 0.f;
 #pragma unroll
@@ -1261,7 +1264,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
 
     // the run that holds the quantile (every warp finds the same one)
     const float u_end = P.unif[2 * (nb + n) + 1];
-    const float m = s_wtot[lane];
+    const float m = lane < kW ? s_wtot[lane] : 0.f;
     const float total = warp_sum(m);
     const float target = u_end * total;
     const float inc = warp_scan_incl(m, lane);
