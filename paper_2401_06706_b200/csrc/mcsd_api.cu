@@ -117,21 +117,27 @@ bool rows_aligned16(const void *base, long long ld, int dtype)
 using NodeKernel = void (*)(const NodeParams);
 constexpr int kEptChoices[3] = {16, 32, 64};
 
-template <int DT, bool DIRECT>
+template <int DT, bool DIRECT, bool PATH>
 NodeKernel pick_ept(int ept)
 {
     switch (ept) {
-    case 16: return node_kernel<DT, 16, DIRECT>;
-    case 32: return node_kernel<DT, 32, DIRECT>;
-    default: return node_kernel<DT, 64, DIRECT>;
+    case 16: return node_kernel<DT, 16, DIRECT, PATH>;
+    case 32: return node_kernel<DT, 32, DIRECT, PATH>;
+    default: return node_kernel<DT, 64, DIRECT, PATH>;
     }
 }
-NodeKernel pick_node_kernel(int dtype, int ept, bool direct)
+template <int DT>
+NodeKernel pick_flags(int ept, bool direct, bool path)
+{
+    if (direct) return path ? pick_ept<DT, true, true>(ept) : pick_ept<DT, true, false>(ept);
+    return path ? pick_ept<DT, false, true>(ept) : pick_ept<DT, false, false>(ept);
+}
+NodeKernel pick_node_kernel(int dtype, int ept, bool direct, bool path)
 {
     switch (dtype) {
-    case MCSD_DTYPE_F32: return direct ? pick_ept<MCSD_DTYPE_F32, true>(ept) : pick_ept<MCSD_DTYPE_F32, false>(ept);
-    case MCSD_DTYPE_BF16: return direct ? pick_ept<MCSD_DTYPE_BF16, true>(ept) : pick_ept<MCSD_DTYPE_BF16, false>(ept);
-    default: return direct ? pick_ept<MCSD_DTYPE_F16, true>(ept) : pick_ept<MCSD_DTYPE_F16, false>(ept);
+    case MCSD_DTYPE_F32: return pick_flags<MCSD_DTYPE_F32>(ept, direct, path);
+    case MCSD_DTYPE_BF16: return pick_flags<MCSD_DTYPE_BF16>(ept, direct, path);
+    default: return pick_flags<MCSD_DTYPE_F16>(ept, direct, path);
     }
 }
 
@@ -323,7 +329,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     NodeConfig cfg;
     int rc = choose_config(d->vocab, d->dtype, aligned, &cfg);
     if (rc != MCSD_OK) return rc;
-    NodeKernel fn = pick_node_kernel(d->dtype, cfg.ept, cfg.direct);
+    NodeKernel fn = pick_node_kernel(d->dtype, cfg.ept, cfg.direct, path);
     const size_t smem = node_smem_bytes(elem_bytes(d->dtype), cfg.ept, cfg.direct);
     const int resident = resident_clusters(fn, cfg.cluster, smem, c.stream);
     if (resident < 1) return MCSD_ERR_CUDA;

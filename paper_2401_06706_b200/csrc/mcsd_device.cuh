@@ -410,7 +410,8 @@ constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
 }
 
 // DT: element type; EPT: vocabulary elements per thread per row; DIRECT: read the
-// rows with plain scalar loads (any alignment) instead of vector loads and bulk copies.
+// rows with plain scalar loads (any alignment) instead of vector loads and bulk copies;
+// PATH: the items are the sequences, each at the node its walk stands on (see NodeParams).
 //
 // Ownership inside a CTA: the slice is cut into 16-byte groups of GV elements; thread
 // (warp w, lane l) owns groups (w * NG + j) * 32 + l, j < NG, so that one warp-wide
@@ -420,7 +421,7 @@ constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
 // Every decision of the rejection loop is taken by every warp of the cluster from
 // bit-identical inputs, so all CTAs of a cluster execute the same number of exchange
 // rounds (the byte counts the exchange barriers are armed with rely on it).
-template <int DT, int EPT, bool DIRECT>
+template <int DT, int EPT, bool DIRECT, bool PATH>
 __global__ void __launch_bounds__(kNodeThreads, node_min_blocks(EPT))
 node_kernel(const __grid_constant__ NodeParams P)
 {
@@ -524,13 +525,13 @@ node_kernel(const __grid_constant__ NodeParams P)
         b += P.step_b;
         n += P.step_n;
         if (n >= P.n_nodes) { n -= P.n_nodes; ++b; }
-        if (P.path_cur) n = b < P.B ? __ldg(P.path_cur + b) : 0;
+        if (PATH) n = b < P.B ? __ldg(P.path_cur + b) : 0;
     };
 
     // ---- candidate pipeline (warp 0 only) -------------------------------------------
     auto fetch_tokens = [&](int b, int n, int slot3) {
         if (b < P.B) {
-            const int k = (n >= 0 && n < P.n_internal) ? P.child_count[n] : 0;
+            const int k = ((!PATH || n >= 0) && n < P.n_internal) ? P.child_count[n] : 0;
             if (lane < k) {
                 const long long ci = static_cast<long long>(b) * P.n_nodes + P.child_first[n] + lane;
                 cp_async4(&ring.tok[slot3][lane], P.cand + ci);
@@ -541,7 +542,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     // needs the item's tokens to have arrived (cp_async_wait_all by this thread)
     auto fetch_logits = [&](int b, int n, int slot3, int slot2) {
         if (b < P.B) {
-            const int k = (n >= 0 && n < P.n_internal) ? P.child_count[n] : 0;
+            const int k = ((!PATH || n >= 0) && n < P.n_internal) ? P.child_count[n] : 0;
             if (lane < k) {
                 const int xt = ring.tok[slot3][lane];
                 if (xt >= 0 && xt < P.V) {
@@ -562,7 +563,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     };
 
     int b = cluster_id / P.n_nodes, n = cluster_id - b * P.n_nodes;  // current item
-    if (P.path_cur) { b = cluster_id; n = b < P.B ? __ldg(P.path_cur + b) : 0; }
+    if (PATH) { b = cluster_id; n = b < P.B ? __ldg(P.path_cur + b) : 0; }
     int b1 = b, n1 = n;                                              // the next one
     advance(b1, n1);
     int b2 = b1, n2 = n1;                                            // the one after
@@ -582,7 +583,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     }
 
     for (; b < P.B; ++it) {
-        const bool internal = n >= 0 && n < P.n_internal;
+        const bool internal = (!PATH || n >= 0) && n < P.n_internal;
         const int k = internal ? P.child_count[n] : 0;
         const int first = internal ? P.child_first[n] : 0;
         const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
@@ -626,7 +627,7 @@ node_kernel(const __grid_constant__ NodeParams P)
             advance(b2, n2);
         };
 
-        if (n < 0) {  // path mode: this walk ended at an earlier level
+        if (PATH && n < 0) {  // this walk ended at an earlier level
             if (crank == 0 && tid == 0) P.path_next[b] = -1;
             look_ahead();
             next_item();
@@ -695,7 +696,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                             crank * NW + warp] = make_float2(rt, st);
             if (crank == 0 && tid == 0) {
                 P.node_accept[node_idx] = -1;
-                if (P.path_next) P.path_next[b] = -1;
+                if (PATH) P.path_next[b] = -1;
             }
             look_ahead();
             next_item();
@@ -950,7 +951,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (warp == 0) {
             if (crank == 0 && lane == 0) {
                 P.node_accept[node_idx] = accepted;
-                if (P.path_next) P.path_next[b] = accepted;
+                if (PATH) P.path_next[b] = accepted;
                 reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
                     make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
             }
