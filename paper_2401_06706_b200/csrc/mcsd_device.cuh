@@ -438,6 +438,9 @@ node_kernel(const __grid_constant__ NodeParams P)
     constexpr bool kPrefetch = !DIRECT && E::kBytes == 2;
     static_assert(EPT % GV == 0, "EPT must be a whole number of 16-byte groups");
     static_assert(NW == 4, "the exchange buffers hold four warps per CTA");
+    // warp 0 leads the exchange rounds and takes the decisions; the look-ahead requests for the
+    // next items are another warp's job so that they do not lengthen the leader's path
+    constexpr int kFetchWarp = 1;
 
     extern __shared__ __align__(128) unsigned char dyn[];
     float4 *qbuf = reinterpret_cast<float4 *>(dyn);  // exponentiated draft slice, thread-private slots
@@ -528,7 +531,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (PATH) n = b < P.B ? __ldg(P.path_cur + b) : 0;
     };
 
-    // ---- candidate pipeline (warp 0 only) -------------------------------------------
+    // ---- candidate pipeline (the fetch warp only) -------------------------------------------
     auto fetch_tokens = [&](int b, int n, int slot3) {
         if (b < P.B) {
             const int k = ((!PATH || n >= 0) && n < P.n_internal) ? P.child_count[n] : 0;
@@ -570,7 +573,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     advance(b2, n2);
     uint32_t it = 0;  // iteration count of this cluster
     bool prev_internal = false;
-    if (warp == 0) {
+    if (warp == kFetchWarp) {
         fetch_tokens(b, n, 0);
         cp_async_wait_all();
         __syncwarp();
@@ -591,7 +594,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         int status_bits = 0;
 
         // this item's candidate data has landed (it was requested one item ago) ...
-        if (warp == 0) cp_async_wait_all();
+        if (warp == kFetchWarp) cp_async_wait_all();
         // ... and, around an item with children, all warps meet: they are done with the
         // previous item (its draft buffer and ring entries may be overwritten) and they
         // see this item's ring entries.  A run of leaves needs no meeting at all.
@@ -609,10 +612,10 @@ node_kernel(const __grid_constant__ NodeParams P)
             bulk_load(smem_u32(kRawZone ? static_cast<const void *>(qraw) : static_cast<const void *>(qbuf)),
                       d_row, bulk_bytes, full_addr);
         }
-        // look-ahead duties of warp 0: L2 prefetch of the next item's slices, candidate
+        // look-ahead duties of the fetch warp: L2 prefetch of the next item's slices, candidate
         // data of the next two items
         auto look_ahead = [&]() {
-            if (warp == 0) {
+            if (warp == kFetchWarp) {
                 if (kPrefetch && lane == 0 && b1 < P.B && bulk_bytes) {
                     bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
                     if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
@@ -652,6 +655,9 @@ node_kernel(const __grid_constant__ NodeParams P)
                 float f[GV];
                 if (!DIRECT && g < n_full_groups) {
                     E::unpack(ld_stream_v4(t_row + static_cast<size_t>(g) * 16), f);
+                } else if (g * GV >= n_mine) {  // wholly past the data
+#pragma unroll
+                    for (int e = 0; e < GV; ++e) f[e] = -INFINITY;
                 } else {
 #pragma unroll
                     for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(t_row, g * GV + e) : -INFINITY;
@@ -732,7 +738,11 @@ node_kernel(const __grid_constant__ NodeParams P)
                         if (g >= n_full_groups) {
                             float f[GV];
 #pragma unroll
-                            for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(d_row, g * GV + e) : -INFINITY;
+                            for (int e = 0; e < GV; ++e) f[e] = -INFINITY;
+                            if (g * GV < n_mine) {  // the ragged last group of the slice
+#pragma unroll
+                                for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(d_row, g * GV + e) : -INFINITY;
+                            }
                             if constexpr (kRawZone) {
                                 uint4 r;
                                 r.x = E::to_bits(f[0]) | (E::to_bits(f[1]) << 16);
@@ -962,7 +972,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         next_item();
     }
 
-    if (warp == 0) cp_async_wait_all();
+    if (warp == kFetchWarp) cp_async_wait_all();
     // no CTA may leave while a peer can still write into its shared memory
     cluster_sync_all();
 }
