@@ -6,7 +6,7 @@
 //                    slice of the vocabulary.  Its slice of the target row goes straight
 //                    into registers with coalesced 128-bit loads; its slice of the draft
 //                    row (nodes that have children) is brought into shared memory with
-//                    one bulk async copy (TMA, no multicast) and stays there.  Both are
+//                    one bulk async copy (TMA, to this CTA alone) and stays there.  Both are
 //                    exponentiated once and then stay on chip while the k candidates of
 //                    the node are tested in order (Algorithm 1 / Algorithm 2), so every
 //                    logit row is read from HBM exactly once.  The rows of the cluster's
@@ -216,7 +216,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
-// One bulk async copy global -> this CTA's shared memory (TMA, no multicast);
+// One bulk async copy global -> this CTA's shared memory (TMA; the copy goes to this CTA alone);
 // completion is signalled on an mbarrier of this CTA as a byte count.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
