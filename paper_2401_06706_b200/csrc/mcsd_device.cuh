@@ -569,8 +569,6 @@ node_kernel(const __grid_constant__ NodeParams P)
     if (PATH) { b = cluster_id; n = b < P.B ? __ldg(P.path_cur + b) : 0; }
     int b1 = b, n1 = n;                                              // the next one
     advance(b1, n1);
-    int b2 = b1, n2 = n1;                                            // the one after
-    advance(b2, n2);
     uint32_t it = 0;  // iteration count of this cluster
     bool prev_internal = false;
     if (warp == kFetchWarp) {
@@ -588,7 +586,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     for (; b < P.B; ++it) {
         const bool internal = (!PATH || n >= 0) && n < P.n_internal;
         const int k = internal ? P.child_count[n] : 0;
-        const int first = internal ? P.child_first[n] : 0;
+        const int first = P.child_first[n];
         const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
         const int s3 = it % 3u, s2 = it & 1u;
         int status_bits = 0;
@@ -621,13 +619,14 @@ node_kernel(const __grid_constant__ NodeParams P)
                     if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
                 }
                 fetch_logits(b1, n1, (it + 1) % 3u, s2 ^ 1);
+                int b2 = b1, n2 = n1;
+                advance(b2, n2);
                 fetch_tokens(b2, n2, (it + 2) % 3u);
             }
         };
         auto next_item = [&]() {
             b = b1; n = n1;
-            b1 = b2; n1 = n2;
-            advance(b2, n2);
+            advance(b1, n1);
         };
 
         if (PATH && n < 0) {  // this walk ended at an earlier level
