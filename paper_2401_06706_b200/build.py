@@ -14,7 +14,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmcsd.so")
 SOURCES = [os.path.join(CSRC, "mcsd_api.cu")]
-HEADERS = [os.path.join(CSRC, "mcsd_device.cuh"), os.path.join(ROOT, "include", "mcsd.h")]
+HEADERS = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")) + [os.path.join(ROOT, "include", "mcsd.h")]
 
 
 def _nvcc() -> str:

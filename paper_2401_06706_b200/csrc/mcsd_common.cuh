@@ -1,0 +1,334 @@
+// Shared pieces of the MCSD device code (sm_100a): limits and bounded-wait constants, the
+// per-node record and the parameter block of the node kernel, the element types (fp32,
+// bf16, fp16) and the arithmetic, warp and PTX helpers that every kernel uses.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mcsd.h"
+
+namespace mcsd {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxCluster = 8;
+// Polls of a bounded wait before it gives up; with the back-off between polls the
+// bound is about two seconds, far beyond any legitimate wait.
+constexpr uint32_t kWaitPolls = 1u << 21;
+
+struct __align__(16) NodeStats {
+    float r_t, r_d;  // references of the sums: ceil(row maximum * scale), log2 units
+    float z_t, z_d;  // sum_x exp2(l * scale - r)
+    float c, s;      // final c_n and S_n of the node (0 and 1 for a leaf)
+    int32_t pad0, pad1;
+};
+
+struct NodeParams {
+    const void *target;
+    const void *draft;
+    const int32_t *cand;
+    const float *unif;
+    int32_t *node_accept;
+    float *node_ratio;  // may be null
+    NodeStats *stats;   // [B][n_nodes], written for nodes with children
+    float2 *leaf_part;  // [B][n_nodes - n_internal][32] per-warp (reference, sum) of every leaf row
+    int32_t *status;  // [B]
+    long long ld_t, ld_d;
+    int32_t B, n_nodes, n_internal, V;
+    int32_t slice;   // vocabulary elements owned by one CTA of the cluster
+    int32_t n_items; // B * n_nodes
+    int32_t step_b, step_n;  // quotient and remainder of (clusters in the grid) / n_nodes
+    // Path mode (one launch per tree level): the items are the sequences, item b works on node
+    // path_cur[b] (negative: that walk has ended, nothing to do) and leaves in path_next[b] the
+    // accepted child, or -1.  Null for the all-node form.  Then step_b = clusters, step_n = 0.
+    const int32_t *path_cur;
+    int32_t *path_next;
+    int32_t mode;
+    float scale;     // log2(e) / T rounded to float ...
+    float scale_lo;  // ... and what the rounding dropped (for the candidates' own probabilities)
+    uint16_t child_first[MCSD_MAX_NODES];
+    uint8_t child_count[MCSD_MAX_NODES];
+};
+
+// ------------------------------------------------------------------ element types
+// Three-input maximum (a NaN operand is ignored, as with fmaxf).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d;
+}
+
+// Per element type: unpacking of one 16-byte vector, scalar access, and a running maximum
+// over whole vectors that stays in the packed format for 2-byte types (two elements per
+// instruction) and is turned into a float once at the end.
+template <int DT> struct Elem;
+template <> struct Elem<MCSD_DTYPE_F32> {
+    static constexpr int kBytes = 4, kVec = 4;
+    static __device__ __forceinline__ void unpack(const uint4 &r, float *o) {
+        o[0] = __uint_as_float(r.x); o[1] = __uint_as_float(r.y);
+        o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
+    }
+    static __device__ __forceinline__ float load(const void *base, long long i) {
+        return __ldg(reinterpret_cast<const float *>(base) + i);
+    }
+    // value of element i given the aligned 32-bit word that contains it
+    static __device__ __forceinline__ float from_word(uint32_t w, long long) { return __uint_as_float(w); }
+    typedef float2 MaxAcc;
+    static __device__ __forceinline__ MaxAcc max_init() { return make_float2(-INFINITY, -INFINITY); }
+    static __device__ __forceinline__ void max_step(MaxAcc &a, const uint4 &r) {
+        a.x = max3(a.x, __uint_as_float(r.x), __uint_as_float(r.y));
+        a.y = max3(a.y, __uint_as_float(r.z), __uint_as_float(r.w));
+    }
+    static __device__ __forceinline__ float max_final(const MaxAcc &a) { return fmaxf(a.x, a.y); }
+};
+template <> struct Elem<MCSD_DTYPE_BF16> {
+    static constexpr int kBytes = 2, kVec = 8;
+    static __device__ __forceinline__ void unpack(const uint4 &r, float *o) {
+        o[0] = __uint_as_float(r.x << 16); o[1] = __uint_as_float(r.x & 0xffff0000u);
+        o[2] = __uint_as_float(r.y << 16); o[3] = __uint_as_float(r.y & 0xffff0000u);
+        o[4] = __uint_as_float(r.z << 16); o[5] = __uint_as_float(r.z & 0xffff0000u);
+        o[6] = __uint_as_float(r.w << 16); o[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ float load(const void *base, long long i) {
+        unsigned short h = __ldg(reinterpret_cast<const unsigned short *>(base) + i);
+        return __uint_as_float(static_cast<uint32_t>(h) << 16);
+    }
+    static __device__ __forceinline__ float from_word(uint32_t w, long long i) {
+        return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));
+    }
+    // 16-bit pattern of a value that this type represents exactly
+    static __device__ __forceinline__ uint32_t to_bits(float f) { return __float_as_uint(f) >> 16; }
+    typedef uint32_t MaxAcc;
+    static __device__ __forceinline__ uint32_t mx(uint32_t a, uint32_t b) {
+        const __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&a),
+                                         *reinterpret_cast<const __nv_bfloat162 *>(&b));
+        return *reinterpret_cast<const uint32_t *>(&r);
+    }
+    static __device__ __forceinline__ MaxAcc max_init() { return 0xff80ff80u; }  // (-inf, -inf)
+    static __device__ __forceinline__ void max_step(MaxAcc &a, const uint4 &r) {
+        a = mx(a, mx(mx(r.x, r.y), mx(r.z, r.w)));
+    }
+    static __device__ __forceinline__ float max_final(const MaxAcc &a) { return fmaxf(from_word(a, 0), from_word(a, 1)); }
+};
+template <> struct Elem<MCSD_DTYPE_F16> {
+    static constexpr int kBytes = 2, kVec = 8;
+    static __device__ __forceinline__ void unpack(const uint4 &r, float *o) {
+        const __half2 *h = reinterpret_cast<const __half2 *>(&r);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 f = __half22float2(h[i]);
+            o[2 * i] = f.x; o[2 * i + 1] = f.y;
+        }
+    }
+    static __device__ __forceinline__ float load(const void *base, long long i) {
+        return __half2float(__ldg(reinterpret_cast<const __half *>(base) + i));
+    }
+    static __device__ __forceinline__ float from_word(uint32_t w, long long i) {
+        const unsigned short h = static_cast<unsigned short>((i & 1) ? (w >> 16) : (w & 0xffffu));
+        return __half2float(__ushort_as_half(h));
+    }
+    static __device__ __forceinline__ uint32_t to_bits(float f) { return __half_as_ushort(__float2half_rn(f)); }
+    typedef uint32_t MaxAcc;
+    static __device__ __forceinline__ uint32_t mx(uint32_t a, uint32_t b) {
+        const __half2 r = __hmax2(*reinterpret_cast<const __half2 *>(&a), *reinterpret_cast<const __half2 *>(&b));
+        return *reinterpret_cast<const uint32_t *>(&r);
+    }
+    static __device__ __forceinline__ MaxAcc max_init() { return 0xfc00fc00u; }  // (-inf, -inf)
+    static __device__ __forceinline__ void max_step(MaxAcc &a, const uint4 &r) {
+        a = mx(a, mx(mx(r.x, r.y), mx(r.z, r.w)));
+    }
+    static __device__ __forceinline__ float max_final(const MaxAcc &a) { return fmaxf(from_word(a, 0), from_word(a, 1)); }
+};
+
+// ------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait with back-off (a waiting thread must not eat the issue slots of the
+// working ones): false when the poll budget ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitPolls; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(i < 64 ? 64 : 1000);
+    }
+    return false;
+}
+// One bulk async copy global -> this CTA's shared memory (TMA; the copy goes to this CTA alone);
+// completion is signalled on an mbarrier of this CTA as a byte count.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Asks L2 to fetch a 16-byte-aligned range (size a multiple of 16); nothing waits on it.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+// 4-byte asynchronous copy global -> shared (no register holds the value in flight).
+// Orders this thread's earlier ordinary shared-memory accesses before later bulk
+// (async-proxy) copies into the same locations.
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void cp_async4(void *smem_dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+// 128-bit streaming load (read once, do not keep in L1).
+__device__ __forceinline__ uint4 ld_stream_v4(const void *p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// Asynchronous 16-byte store into a CTA of the cluster that reports its bytes to an
+// mbarrier of that CTA: the data is visible to whoever sees the barrier's phase complete,
+// no fence on either side.
+__device__ __forceinline__ void st_async_f4(uint32_t addr, float4 v, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar) : "memory");
+}
+
+// Packed pairs of floats: sm_100 executes fma and add on both halves of an aligned
+// register pair with one instruction (each half rounds exactly like the scalar operation).
+typedef float2 f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { return __fadd2_rn(a, b); }
+// Warp-wide maximum in one instruction (NaN inputs are ignored).
+__device__ __forceinline__ float warp_max(float v) {
+    float d; asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(d) : "f"(v)); return d;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_scan_incl(float v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        float t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+// 2^d for an integer-valued d (a difference of two references): exact; 0 when
+// d < -126 (also for d = -inf), clamped to 2^127 above.
+__device__ __forceinline__ float exp2i(float d) {
+    d = fminf(fmaxf(d, -127.f), 127.f);
+    // adding 1.5 * 2^23 leaves the integer in the low mantissa bits (no conversion instruction)
+    const int i = __float_as_int(d + 12582912.f) - 0x4b400000;
+    return __int_as_float((i + 127) << 23);
+}
+// The same in double for an integer e: 0 below 2^-1000.
+__device__ __forceinline__ double exp2i_d(int e) {
+    if (e < -1000) return 0.0;
+    e = e > 1000 ? 1000 : e;
+    return __hiloint2double((e + 1023) << 20, 0);
+}
+// 2^(l * (scale + scale_lo)) as 2^ip * (return value), ip an integer and the return value
+// in [2^-0.51, 2^0.51], to about 1e-7 relative however large the exponent is: the
+// product is formed exactly as a sum of two floats, its integer part goes to ip and only
+// the fraction is exponentiated.  Infinite or NaN products give 0 (or +inf) with ip = 0.
+__device__ __forceinline__ float split_exp2(float l, float scale, float scale_lo, int &ip) {
+    const float ph = l * scale;
+    ip = 0;
+    if (!(fabsf(ph) < 1.0e9f)) return ph > 0.f ? INFINITY : 0.f;
+    const float pe = fmaf(l, scale, -ph);      // exact error of the rounded product
+    const float pl = fmaf(l, scale_lo, pe);    // plus the part of the scale that float drops
+    const float ipf = rintf(ph);
+    const float f = (ph - ipf) + pl;           // |f| <= 0.5 + tiny; the subtraction is exact
+    ip = static_cast<int>(ipf);
+    // Taylor series of exp(f ln 2), |f ln 2| <= 0.36: the degree-7 remainder is below 6e-9
+    float y = 1.5252733804059841e-05f;
+    y = fmaf(y, f, 1.5403530393381608e-04f);
+    y = fmaf(y, f, 1.3333558146428443e-03f);
+    y = fmaf(y, f, 9.6181291076284772e-03f);
+    y = fmaf(y, f, 5.5504108664821580e-02f);
+    y = fmaf(y, f, 2.4022650695910071e-01f);
+    y = fmaf(y, f, 6.9314718055994531e-01f);
+    return fmaf(y, f, 1.f);
+}
+// Integer reference of a set whose largest scaled logit is m (log2 units); -inf for
+// an empty set.  NaN-free inputs give ceil(m), so that every exponent is <= 0.
+__device__ __forceinline__ float int_ref(float m_scaled) {
+    return (m_scaled == -INFINITY) ? -INFINITY : ceilf(m_scaled);
+}
+
+// Warp totals of N values per lane in N-1 + (5 - log2 N) shuffles instead of 5 N: each
+// halving step pairs lanes and splits the value indices between them.  On return
+// every lane holds in `out` the warp total of value index `idx` (the return value),
+// idx = lane / (32 / N).
+template <int HALF>
+__device__ __forceinline__ void halve_step(float *w, int lane, int off, int &idx)
+{
+    const bool hi = (lane & off) != 0;
+#pragma unroll
+    for (int j = 0; j < HALF; ++j) {
+        const float send = hi ? w[j] : w[j + HALF];
+        const float keep = hi ? w[j + HALF] : w[j];
+        w[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+    idx += hi ? HALF : 0;
+}
+template <int N>
+__device__ __forceinline__ int warp_multi_sum(const float (&v)[N], int lane, float &out)
+{
+    static_assert(N == 1 || N == 2 || N == 4 || N == 8 || N == 16, "unsupported count");
+    float w[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) w[j] = v[j];
+    int idx = 0;
+    if constexpr (N >= 2) halve_step<N / 2>(w, lane, 16, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 16);
+    if constexpr (N >= 4) halve_step<N / 4>(w, lane, 8, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 8);
+    if constexpr (N >= 8) halve_step<N / 8>(w, lane, 4, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 4);
+    if constexpr (N >= 16) halve_step<N / 16>(w, lane, 2, idx);
+    else w[0] += __shfl_xor_sync(0xffffffffu, w[0], 2);
+    w[0] += __shfl_xor_sync(0xffffffffu, w[0], 1);
+    out = w[0];
+    return idx;
+}
+
+}  // namespace mcsd

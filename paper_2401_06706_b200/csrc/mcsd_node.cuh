@@ -1,0 +1,623 @@
+// node_kernel (T > 0): Algorithm 1 / Algorithm 2 at every node of every tree, one
+// thread-block cluster per (sequence, node) item with the two logit rows held on chip.
+#pragma once
+
+#include "mcsd_common.cuh"
+
+namespace mcsd {
+
+// Shared state of the cluster-wide exchange: two buffers of one float4 per (cluster
+// rank, warp) and one mbarrier per buffer.  In round r every warp of every CTA sends its
+// value into buffer r&1 of every CTA of the cluster (its own included) with asynchronous
+// stores that report their bytes to that CTA's barrier; the CTA armed the barrier with
+// the byte count of a whole round, so when its phase completes all values of the round
+// are there, in vocabulary order (rank-major, then warp).  One warp per CTA watches the
+// barrier (bounded, with back-off), the others wait for it at a CTA barrier, so nobody
+// spins on the issue slots the working CTAs need.  A buffer is rewritten two rounds
+// later, which a peer can only reach after all warps of this CTA have sent the round in
+// between, i.e. after they finished reading.
+struct Exchange {
+    float4 slot[2][kMaxCluster * 4];
+    unsigned long long bar[2];
+};
+
+// What the leader warp of a CTA tells the other warps at the end of an exchange round.
+struct Action {
+    float4 stats;  // (row reference of p, of q, 1 / Z_t, Z_t / Z_d); written in the statistics round only
+    float c_try;   // c of the residual sum to form next
+    int more;      // 1: form that sum and run another round; 0: the node is decided
+};
+
+// Candidate data of the next items, fetched ahead of use by warp 0 so that no DRAM
+// latency sits on the per-node critical path: lane i handles candidate i.
+//   token id and acceptance uniform   two items ahead  (ring of 3)
+//   the candidate's own two logits    one item ahead   (ring of 2; they need the token)
+struct CandRing {
+    int32_t tok[3][MCSD_MAX_CHILDREN];
+    float u[3][MCSD_MAX_CHILDREN];
+    uint32_t tl[2][MCSD_MAX_CHILDREN];  // aligned 32-bit word holding the target logit
+    uint32_t dl[2][MCSD_MAX_CHILDREN];  // same for the draft logit
+};
+
+// Threads of one node-kernel CTA.  Few threads with many elements each: the per-thread
+// bookkeeping (about 60 registers) is paid once per 64 elements, so that four CTAs
+// with a 64-element target slice per thread fit the register file without spilling.
+constexpr int kNodeThreads = 128;
+constexpr int kNodeWarps = kNodeThreads / 32;
+// Resident CTAs per SM the register budget is held to (128 / 96 / 80 registers).
+constexpr int node_min_blocks(int ept) { return ept >= 64 ? 4 : (ept >= 32 ? 5 : 6); }
+// Dynamic shared memory of one CTA: the exponentiated draft slice (float) and, for
+// 2-byte logits on the bulk-copy path, the zone the raw draft slice lands in.
+constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
+    return static_cast<size_t>(kNodeThreads) * ept * 4 +
+           ((!direct && elem_bytes == 2) ? static_cast<size_t>(kNodeThreads) * ept * 2 : 0);
+}
+
+// DT: element type; EPT: vocabulary elements per thread per row; DIRECT: read the
+// rows with plain scalar loads (any alignment) instead of vector loads and bulk copies;
+// PATH: the items are the sequences, each at the node its walk stands on (see NodeParams).
+//
+// Ownership inside a CTA: the slice is cut into 16-byte groups of GV elements; thread
+// (warp w, lane l) owns groups (w * NG + j) * 32 + l, j < NG, so that one warp-wide
+// access is contiguous and a warp's elements are one contiguous run of the vocabulary.
+// Groups past the end of the slice hold -inf (probability 0).
+//
+// Every decision of the rejection loop is taken by every warp of the cluster from
+// bit-identical inputs, so all CTAs of a cluster execute the same number of exchange
+// rounds (the byte counts the exchange barriers are armed with rely on it).
+template <int DT, int EPT, bool DIRECT, bool PATH>
+__global__ void __launch_bounds__(kNodeThreads, node_min_blocks(EPT))
+node_kernel(const __grid_constant__ NodeParams P)
+{
+    using E = Elem<DT>;
+    constexpr int NT = kNodeThreads, NW = kNodeWarps;
+    constexpr int GV = E::kVec;
+    constexpr int NG = EPT / GV;
+    constexpr int H = GV / 4;  // float4 per group once exponentiated
+    constexpr bool kRawZone = !DIRECT && E::kBytes == 2;
+    // L2 prefetch of the cluster's next item: with 2-byte logits the kernel is bound by the
+    // SMs and the prefetch takes DRAM latency off the per-node chain (measured +20 %); with
+    // 4-byte logits it is bound by HBM and the extra request stream only costs (-1 %, and
+    // -30 % on leaf-only trees), so it is left out there
+    constexpr bool kPrefetch = !DIRECT && E::kBytes == 2;
+    static_assert(EPT % GV == 0, "EPT must be a whole number of 16-byte groups");
+    static_assert(NW == 4, "the exchange buffers hold four warps per CTA");
+    // warp 0 leads the exchange rounds and takes the decisions; the look-ahead requests for the
+    // next items are another warp's job so that they do not lengthen the leader's path
+    constexpr int kFetchWarp = 1;
+
+    extern __shared__ __align__(128) unsigned char dyn[];
+    float4 *qbuf = reinterpret_cast<float4 *>(dyn);  // exponentiated draft slice, thread-private slots
+    uint4 *qraw = reinterpret_cast<uint4 *>(dyn + static_cast<size_t>(NT) * EPT * 4);
+    __shared__ Exchange xch;
+    __shared__ __align__(8) unsigned long long full_bar;
+    __shared__ CandRing ring;
+    __shared__ Action act[2];
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    // (broadcast from lane 0 so that the compiler knows the warp index is warp-uniform)
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+    const uint32_t crank = __clusterRelativeBlockRank(), csize = __clusterSizeInBlocks();
+    const int cluster_id = blockIdx.x / csize;
+    const int n_entries = static_cast<int>(csize) * NW;  // values per exchange round (<= 32)
+    const float scale = P.scale;
+    const uint32_t full_addr = smem_u32(&full_bar);
+    const uint32_t xbar_addr[2] = {smem_u32(&xch.bar[0]), smem_u32(&xch.bar[1])};
+
+    // this CTA's slice of the vocabulary and this warp's run of it
+    const int v_begin = static_cast<int>(crank) * P.slice;
+    int n_mine = P.V - v_begin;
+    n_mine = n_mine < 0 ? 0 : (n_mine > P.slice ? P.slice : n_mine);
+    const int n_full_groups = n_mine / GV;            // whole 16-byte groups
+    const int g0 = warp * (NG * 32) + lane;           // this thread's group of chunk 0
+    // every group of this warp is a whole group: the common case takes unpredicated loads
+    const bool warp_full = !DIRECT && (warp + 1) * (NG * 32) <= n_full_groups;
+    // bytes of the slice that are whole groups: what one bulk copy / prefetch moves
+    const uint32_t bulk_bytes = DIRECT ? 0u : static_cast<uint32_t>(n_full_groups) * 16u;
+
+    // slot of (chunk j, quarter h) in qbuf: for 4-byte logits it is the group's own place in
+    // the slice, so that the bulk copy lands the raw values where the exponentiated ones go
+    auto qslot = [&](int j, int h) -> int {
+        return E::kBytes == 4 ? g0 + j * 32 : (j * H + h) * NT + tid;
+    };
+
+    if (tid == 0) {
+        mbar_init(full_addr, 1);
+        mbar_init(xbar_addr[0], 1);
+        mbar_init(xbar_addr[1], 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    cluster_sync_all();  // every CTA's barriers exist before anyone stores into a peer
+
+    uint32_t full_parity = 0, round = 0;
+    int poisoned = 0;
+
+    auto t_slice = [&](long long item) -> const unsigned char * {
+        return reinterpret_cast<const unsigned char *>(P.target) + (item * P.ld_t + v_begin) * E::kBytes;
+    };
+    auto d_slice = [&](int b, int n) -> const unsigned char * {
+        return reinterpret_cast<const unsigned char *>(P.draft) +
+            ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + v_begin) * E::kBytes;
+    };
+
+    // One exchange round.  send: `mine` is this warp's value (the same in all lanes);
+    // whatever is placed between send and wait overlaps the round's latency.  wait:
+    // returns entry `lane` of the round (rank-major, then warp), the given identity for
+    // lanes beyond the entry count.
+    auto exchange_send = [&](float4 mine) {
+        const uint32_t s = round & 1u;
+        if (tid == 0) mbar_arrive_expect_tx(xbar_addr[s], static_cast<uint32_t>(n_entries) * 16u);
+        if (lane < static_cast<int>(csize)) {
+            const uint32_t dst = map_to_rank(smem_u32(&xch.slot[s][crank * NW + warp]), lane);
+            st_async_f4(dst, mine, map_to_rank(xbar_addr[s], lane));
+        }
+    };
+    // leader (warp 0) only: waits for the round and returns entry `lane`
+    auto exchange_leader_wait = [&](float4 identity) -> float4 {
+        const uint32_t s = round & 1u;
+        // once a wait has expired the results are void and later rounds do not wait again
+        if (!poisoned && !mbar_wait(xbar_addr[s], (round >> 1) & 1u)) poisoned = 1;
+        return lane < n_entries ? xch.slot[s][lane] : identity;
+    };
+    // all warps: ends the round (the other warps have been waiting here for the leader)
+    auto exchange_release = [&]() {
+        __syncthreads();
+        ++round;
+    };
+
+    // (sequence, node) of the items this cluster visits: the current one and the two after
+    // it, advanced by the precomputed quotient and remainder of the stride
+    auto advance = [&](int &b, int &n) {
+        b += P.step_b;
+        n += P.step_n;
+        if (n >= P.n_nodes) { n -= P.n_nodes; ++b; }
+        if (PATH) n = b < P.B ? __ldg(P.path_cur + b) : 0;
+    };
+
+    // ---- candidate pipeline (the fetch warp only) -------------------------------------------
+    auto fetch_tokens = [&](int b, int n, int slot3) {
+        if (b < P.B) {
+            const int k = ((!PATH || n >= 0) && n < P.n_internal) ? P.child_count[n] : 0;
+            if (lane < k) {
+                const long long ci = static_cast<long long>(b) * P.n_nodes + P.child_first[n] + lane;
+                cp_async4(&ring.tok[slot3][lane], P.cand + ci);
+                cp_async4(&ring.u[slot3][lane], P.unif + 2 * ci);
+            }
+        }
+    };
+    // needs the item's tokens to have arrived (cp_async_wait_all by this thread)
+    auto fetch_logits = [&](int b, int n, int slot3, int slot2) {
+        if (b < P.B) {
+            const int k = ((!PATH || n >= 0) && n < P.n_internal) ? P.child_count[n] : 0;
+            if (lane < k) {
+                const int xt = ring.tok[slot3][lane];
+                if (xt >= 0 && xt < P.V) {
+                    const unsigned char *t = reinterpret_cast<const unsigned char *>(P.target) +
+                        ((static_cast<long long>(b) * P.n_nodes + n) * P.ld_t + xt) * E::kBytes;
+                    const unsigned char *d = reinterpret_cast<const unsigned char *>(P.draft) +
+                        ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + xt) * E::kBytes;
+                    if (!DIRECT) {  // rows are 16-byte aligned: the enclosing word lies inside the row
+                        cp_async4(&ring.tl[slot2][lane], reinterpret_cast<const void *>(reinterpret_cast<uintptr_t>(t) & ~uintptr_t(3)));
+                        cp_async4(&ring.dl[slot2][lane], reinterpret_cast<const void *>(reinterpret_cast<uintptr_t>(d) & ~uintptr_t(3)));
+                    } else {        // any alignment: plain loads of exactly the element, kept as float
+                        ring.tl[slot2][lane] = __float_as_uint(E::load(t, 0));
+                        ring.dl[slot2][lane] = __float_as_uint(E::load(d, 0));
+                    }
+                }
+            }
+        }
+    };
+
+    int b = cluster_id / P.n_nodes, n = cluster_id - b * P.n_nodes;  // current item
+    if (PATH) { b = cluster_id; n = b < P.B ? __ldg(P.path_cur + b) : 0; }
+    int b1 = b, n1 = n;                                              // the next one
+    advance(b1, n1);
+    uint32_t it = 0;  // iteration count of this cluster
+    bool prev_internal = false;
+    if (warp == kFetchWarp) {
+        fetch_tokens(b, n, 0);
+        cp_async_wait_all();
+        __syncwarp();
+        fetch_logits(b, n, 0, 0);
+        fetch_tokens(b1, n1, 1);
+    }
+    if (kPrefetch && tid == 0 && b < P.B && bulk_bytes) {
+        bulk_prefetch_l2(t_slice(static_cast<long long>(b) * P.n_nodes + n), bulk_bytes);
+        if (n < P.n_internal) bulk_prefetch_l2(d_slice(b, n), bulk_bytes);
+    }
+
+    for (; b < P.B; ++it) {
+        const bool internal = (!PATH || n >= 0) && n < P.n_internal;
+        const int k = internal ? P.child_count[n] : 0;
+        const int first = P.child_first[n];
+        const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
+        const int s3 = it % 3u, s2 = it & 1u;
+        int status_bits = 0;
+
+        // this item's candidate data has landed (it was requested one item ago) ...
+        if (warp == kFetchWarp) cp_async_wait_all();
+        // ... and, around an item with children, all warps meet: they are done with the
+        // previous item (its draft buffer and ring entries may be overwritten) and they
+        // see this item's ring entries.  A run of leaves needs no meeting at all.
+        if (internal || prev_internal) {
+            if (!DIRECT) fence_proxy_async();
+            __syncthreads();
+        }
+        prev_internal = internal;
+
+        const unsigned char *t_row = t_slice(node_idx);
+        const unsigned char *d_row = d_slice(b, n);
+        const bool q_bulk = internal && bulk_bytes != 0;
+        if (tid == 0 && q_bulk && !poisoned) {  // (after an expired wait nothing more is copied)
+            mbar_arrive_expect_tx(full_addr, bulk_bytes);
+            bulk_load(smem_u32(kRawZone ? static_cast<const void *>(qraw) : static_cast<const void *>(qbuf)),
+                      d_row, bulk_bytes, full_addr);
+        }
+        // look-ahead duties of the fetch warp: L2 prefetch of the next item's slices, candidate
+        // data of the next two items
+        auto look_ahead = [&]() {
+            if (warp == kFetchWarp) {
+                if (kPrefetch && lane == 0 && b1 < P.B && bulk_bytes) {
+                    bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
+                    if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
+                }
+                fetch_logits(b1, n1, (it + 1) % 3u, s2 ^ 1);
+                int b2 = b1, n2 = n1;
+                advance(b2, n2);
+                fetch_tokens(b2, n2, (it + 2) % 3u);
+            }
+        };
+        auto next_item = [&]() {
+            b = b1; n = n1;
+            advance(b1, n1);
+        };
+
+        if (PATH && n < 0) {  // this walk ended at an earlier level
+            if (crank == 0 && tid == 0) P.path_next[b] = -1;
+            look_ahead();
+            next_item();
+            continue;
+        }
+
+        // ---- target slice -> registers, as packed pairs
+        f32x2 tv[EPT / 2];
+        if (warp_full) {
+            // every group of this warp is a whole group inside the slice
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                float f[GV];
+                E::unpack(ld_stream_v4(t_row + static_cast<size_t>(g0 + j * 32) * 16), f);
+#pragma unroll
+                for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                const int g = g0 + j * 32;
+                float f[GV];
+                if (!DIRECT && g < n_full_groups) {
+                    E::unpack(ld_stream_v4(t_row + static_cast<size_t>(g) * 16), f);
+                } else if (g * GV >= n_mine) {  // wholly past the data
+#pragma unroll
+                    for (int e = 0; e < GV; ++e) f[e] = -INFINITY;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(t_row, g * GV + e) : -INFINITY;
+                }
+#pragma unroll
+                for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
+            }
+        }
+        // Each warp exponentiates relative to its own integer reference; the factor to the
+        // row's reference and the normaliser are applied as per-warp scalars later.
+        float rt, zt;
+        {
+            float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+            for (int p = 0; p < EPT / 2; p += 2) {
+                m0 = max3(m0, tv[p].x, tv[p].y);
+                m1 = max3(m1, tv[p + 1].x, tv[p + 1].y);
+            }
+            rt = int_ref(warp_max(fmaxf(m0, m1)) * scale);  // one reference per warp
+            const float rt0 = (rt == -INFINITY) ? 0.f : rt;
+            const f32x2 scale2 = pack2(scale, scale), nref2 = pack2(-rt0, -rt0);
+            f32x2 z0 = pack2(0.f, 0.f), z1 = z0;
+#pragma unroll
+            for (int p = 0; p < EPT / 2; p += 2) {
+                const f32x2 x01 = fma2(tv[p], scale2, nref2), x23 = fma2(tv[p + 1], scale2, nref2);
+                tv[p] = pack2(ex2f(x01.x), ex2f(x01.y));
+                tv[p + 1] = pack2(ex2f(x23.x), ex2f(x23.y));
+                z0 = add2(z0, tv[p]);
+                z1 = add2(z1, tv[p + 1]);
+            }
+            const f32x2 z = add2(z0, z1);
+            zt = z.x + z.y;
+        }
+
+        if (!internal) {
+            // A leaf decides nothing.  Its softmax statistics are only needed if a walk ends
+            // here, so each warp leaves the partial statistics of its run in global memory
+            // (the walk kernel combines them) and goes on: no exchange, no barrier.
+            const float st = warp_sum(zt);
+            if (lane == 0)
+                P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * 32 +
+                            crank * NW + warp] = make_float2(rt, st);
+            if (crank == 0 && tid == 0) {
+                P.node_accept[node_idx] = -1;
+                if (PATH) P.path_next[b] = -1;
+            }
+            look_ahead();
+            next_item();
+            continue;
+        }
+
+        // ---- draft slice: exponentiated in shared memory, in the slots of its owner
+        float zd = 0.f, rd = -INFINITY;
+        {
+            if (DIRECT) {
+                // the owner copies its raw elements into its slots, as float
+#pragma unroll
+                for (int j = 0; j < NG; ++j) {
+                    const int g = g0 + j * 32;
+                    float f[GV];
+#pragma unroll
+                    for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(d_row, g * GV + e) : -INFINITY;
+#pragma unroll
+                    for (int h = 0; h < H; ++h)
+                        qbuf[qslot(j, h)] = make_float4(f[4 * h], f[4 * h + 1], f[4 * h + 2], f[4 * h + 3]);
+                }
+            } else {
+                if (q_bulk && !poisoned) {
+                    if (!mbar_wait(full_addr, full_parity)) poisoned = 1;
+                    full_parity ^= 1u;
+                }
+                if (!warp_full) {
+                    // groups the bulk copy did not bring: -inf past the data, and the ragged
+                    // last group of the slice element by element (the slots are this thread's own)
+#pragma unroll
+                    for (int j = 0; j < NG; ++j) {
+                        const int g = g0 + j * 32;
+                        if (g >= n_full_groups) {
+                            float f[GV];
+#pragma unroll
+                            for (int e = 0; e < GV; ++e) f[e] = -INFINITY;
+                            if (g * GV < n_mine) {  // the ragged last group of the slice
+#pragma unroll
+                                for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(d_row, g * GV + e) : -INFINITY;
+                            }
+                            if constexpr (kRawZone) {
+                                uint4 r;
+                                r.x = E::to_bits(f[0]) | (E::to_bits(f[1]) << 16);
+                                r.y = E::to_bits(f[2]) | (E::to_bits(f[3]) << 16);
+                                r.z = E::to_bits(f[4]) | (E::to_bits(f[5]) << 16);
+                                r.w = E::to_bits(f[6]) | (E::to_bits(f[7]) << 16);
+                                qraw[g] = r;
+                            } else {
+                                qbuf[g] = make_float4(f[0], f[1], f[2], f[3]);
+                            }
+                        }
+                    }
+                }
+            }
+            auto read_q_raw = [&](int j, float *r) {
+                if constexpr (kRawZone) {
+                    E::unpack(qraw[g0 + j * 32], r);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < H; ++h) {
+                        const float4 v = qbuf[qslot(j, h)];
+                        r[4 * h] = v.x; r[4 * h + 1] = v.y; r[4 * h + 2] = v.z; r[4 * h + 3] = v.w;
+                    }
+                }
+            };
+            float md;
+            if constexpr (kRawZone || E::kBytes == 4) {
+                // maximum over the raw vectors as they lie in shared memory (packed for 2-byte types)
+                typename E::MaxAcc acc = E::max_init();
+#pragma unroll
+                for (int j = 0; j < NG; ++j)
+                    E::max_step(acc, kRawZone ? qraw[g0 + j * 32] : *reinterpret_cast<const uint4 *>(&qbuf[qslot(j, 0)]));
+                md = E::max_final(acc);
+            } else {
+                float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < NG; ++j) {
+                    float r[GV];
+                    read_q_raw(j, r);
+#pragma unroll
+                    for (int e = 0; e < GV; e += 4) {
+                        m0 = max3(m0, r[e], r[e + 1]);
+                        m1 = max3(m1, r[e + 2], r[e + 3]);
+                    }
+                }
+                md = fmaxf(m0, m1);
+            }
+            rd = int_ref(warp_max(md) * scale);
+            const float rd0 = (rd == -INFINITY) ? 0.f : rd;
+            const f32x2 scale2 = pack2(scale, scale), nref2 = pack2(-rd0, -rd0);
+            f32x2 z0 = pack2(0.f, 0.f), z1 = z0;
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                float r[GV];
+                read_q_raw(j, r);
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    const f32x2 x01 = fma2(pack2(r[4 * h], r[4 * h + 1]), scale2, nref2);
+                    const f32x2 x23 = fma2(pack2(r[4 * h + 2], r[4 * h + 3]), scale2, nref2);
+                    const float4 ev = make_float4(ex2f(x01.x), ex2f(x01.y), ex2f(x23.x), ex2f(x23.y));
+                    qbuf[qslot(j, h)] = ev;
+                    z0 = add2(z0, pack2(ev.x, ev.y));
+                    z1 = add2(z1, pack2(ev.z, ev.w));
+                }
+            }
+            const f32x2 z = add2(z0, z1);
+            zd = z.x + z.y;
+        }
+
+        // ---- softmax statistics of both rows: one exchange round
+        exchange_send(make_float4(rt, warp_sum(zt), rd, warp_sum(zd)));  // per warp: (ref_t, z_t, ref_d, z_d)
+        look_ahead();  // in the shadow of the exchange
+
+        // From here on warp 0 of every CTA is the leader: it alone combines the exchanged
+        // values, evaluates the acceptance tests (Algorithm 1 / Algorithm 2) and tells the
+        // other warps through `act` what to do next; they only stream and reduce.  The
+        // leaders of a cluster work from bit-identical inputs and decide identically.
+        //
+        // leader state of the rejection loop, in units where W' = W * K, K = Z_t * Z_d:
+        double c = 0.0, S = 1.0, Wk = 0.0, K = 0.0, c_try = 0.0;
+        double px = 0.0, qx = 0.0;  // lane i of the leader: candidate i's p and q, times K
+        int cand_i = 0, attempt = 0, accepted = -1, my_tok = -1;
+        float u_acc = 2.f;
+        // tests candidates from cand_i on until one is accepted (returns 0), all are rejected
+        // (returns 0) or one is rejected and its residual sum is needed (returns 1, c_try set)
+        auto leader_decide = [&]() -> int {
+            while (cand_i < k) {
+                const int i = cand_i;
+                const int xi = __shfl_sync(0xffffffffu, my_tok, i);
+                const double ui = static_cast<double>(__shfl_sync(0xffffffffu, u_acc, i));
+                const double pxi = __shfl_sync(0xffffffffu, px, i), qxi = __shfl_sync(0xffffffffu, qx, i);
+                const bool valid = xi >= 0 && xi < P.V;
+                if (!valid) status_bits |= MCSD_STATUS_BAD_TOKEN;
+                // Algorithm 2: a token rejected earlier at this node has draft probability 0 now
+                const bool dup = P.mode == 1 &&
+                    (__ballot_sync(0xffffffffu, lane < i && my_tok == xi) != 0u);
+                const bool zero_q = !valid || dup || !(qxi > 0.0) || !(Wk > 0.0);
+                double Pn = pxi - c * qxi;
+                Pn = Pn > 0.0 ? Pn : 0.0;
+                // r <= [P_n(x~)/S_n] / [q(x~)/W_n] without divisions (all factors > 0)
+                const bool accept = !zero_q && ui * S * qxi * K <= Pn * Wk;
+                if (P.node_ratio && crank == 0 && lane == 0)
+                    P.node_ratio[static_cast<long long>(b) * P.n_nodes + first + i] =
+                        zero_q ? -1.f : static_cast<float>((Pn / S) / (qxi * K / Wk));
+                if (accept) { accepted = first + i; return 0; }
+                // rejected: p := norm(max(0, p - q)); Algorithm 2 also removes x~ from q
+                c_try = c;
+                if (Wk > 0.0) c_try = (P.mode == 1) ? c + S * K / Wk : c + S;
+                if (P.mode == 1 && !zero_q) { Wk -= qxi; if (!(Wk > 0.0)) Wk = 0.0; }
+                attempt = 0;
+                return 1;
+            }
+            return 0;
+        };
+
+        if (warp == 0) {
+            // while the round is in flight: 2^(scaled logit) of the candidates' own logits as
+            // 2^int * frac (lane i = candidate i)
+            float frac_t = 0.f, frac_d = 0.f;
+            int int_t = 0, int_d = 0;
+            bool cand_ok = false;
+            if (lane < k) {
+                my_tok = ring.tok[s3][lane];
+                u_acc = ring.u[s3][lane];
+                cand_ok = my_tok >= 0 && my_tok < P.V;
+                if (cand_ok) {
+                    const uint32_t wt = ring.tl[s2][lane], wd = ring.dl[s2][lane];
+                    frac_t = split_exp2(DIRECT ? __uint_as_float(wt) : E::from_word(wt, my_tok), scale, P.scale_lo, int_t);
+                    frac_d = split_exp2(DIRECT ? __uint_as_float(wd) : E::from_word(wd, my_tok), scale, P.scale_lo, int_d);
+                }
+            }
+            const float4 ent = exchange_leader_wait(make_float4(-INFINITY, 0.f, -INFINITY, 0.f));
+            // row references ceil(row maximum * scale) and normalisers
+            const float R_t = warp_max(ent.x), R_d = warp_max(ent.z);
+            const float Z_t = warp_sum(ent.y * exp2i(ent.x - R_t));
+            const float Z_d = warp_sum(ent.w * exp2i(ent.z - R_d));
+            const bool t_ok = Z_t > 0.f && Z_t < INFINITY;  // false for an all -inf or NaN row
+            const bool d_ok = Z_d > 0.f && Z_d < INFINITY;
+            if (!t_ok) status_bits |= MCSD_STATUS_NO_MASS;
+            // candidates' probabilities, both multiplied by K so that no division is needed:
+            // px' = 2^(l_t*scale - R_t) * Z_d, qx' = 2^(l_d*scale - R_d) * Z_t
+            K = static_cast<double>(Z_t) * static_cast<double>(Z_d);
+            Wk = K;
+            if (cand_ok && t_ok && d_ok) {
+                px = static_cast<double>(frac_t) * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
+                qx = static_cast<double>(frac_d) * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
+            }
+            const int more = leader_decide();
+            if (lane == 0) {
+                act[round & 1u].stats = make_float4(R_t, R_d, t_ok ? 1.f / Z_t : 0.f, (t_ok && d_ok) ? Z_t / Z_d : 0.f);
+                act[round & 1u].c_try = static_cast<float>(c_try);
+                act[round & 1u].more = more;
+                if (crank == 0) *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
+            }
+        }
+        exchange_release();  // CTA barrier: the leader's verdict is visible to all warps
+        const float4 st4 = act[(round - 1u) & 1u].stats;
+        int more = act[(round - 1u) & 1u].more;
+        float c_next = act[(round - 1u) & 1u].c_try;
+        // p(x) = tv * a, q(x) = dv * bq for this warp's elements
+        const float a = exp2i(rt - st4.x) * st4.z;
+        float b_over_a = 0.f;  // bq / a
+        if (a > 0.f && st4.w > 0.f && rd != -INFINITY) b_over_a = exp2i((rd - st4.y) - (rt - st4.x)) * st4.w;
+
+        // residual mass of this warp's run for a given c
+        auto residual_pass = [&](float c_f) -> float {
+            const float kappa = fminf(c_f * b_over_a, 3.0e38f);
+            const f32x2 nk2 = pack2(-kappa, -kappa);
+            f32x2 s0 = pack2(0.f, 0.f), s1 = s0;
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    const float4 d = qbuf[qslot(j, h)];
+                    const int o = (j * GV + 4 * h) / 2;
+                    const f32x2 x01 = fma2(pack2(d.x, d.y), nk2, tv[o]);
+                    const f32x2 x23 = fma2(pack2(d.z, d.w), nk2, tv[o + 1]);
+                    s0 = add2(s0, pack2(fmaxf(x01.x, 0.f), fmaxf(x01.y, 0.f)));
+                    s1 = add2(s1, pack2(fmaxf(x23.x, 0.f), fmaxf(x23.y, 0.f)));
+                }
+            }
+            const f32x2 t = add2(s0, s1);
+            return warp_sum((t.x + t.y) * a);
+        };
+
+        // ---- one round per rejection: all warps reduce, the leader decides what comes next
+#pragma unroll 1
+        while (more) {
+            exchange_send(make_float4(residual_pass(c_next), 0.f, 0.f, 0.f));
+            if (warp == 0) {
+                const float4 ent = exchange_leader_wait(make_float4(0.f, 0.f, 0.f, 0.f));
+                const float S_new = warp_sum(ent.x);
+                int next;
+                if (S_new > 0.f) {
+                    if (attempt == 0) { c = c_try; S = static_cast<double>(S_new); }
+                    ++cand_i;
+                    next = leader_decide();
+                } else {
+                    // zero residual mass: keep the previous residual (recompute its sums once)
+                    status_bits |= MCSD_STATUS_DEGENERATE;
+                    if (attempt == 0) { attempt = 1; c_try = c; next = 1; }
+                    else { ++cand_i; next = leader_decide(); }
+                }
+                if (lane == 0) {
+                    act[round & 1u].c_try = static_cast<float>(c_try);
+                    act[round & 1u].more = next;
+                }
+            }
+            exchange_release();
+            more = act[(round - 1u) & 1u].more;
+            c_next = act[(round - 1u) & 1u].c_try;
+        }
+
+        // ---- per-node results (the endpoint token is drawn by the walk kernel, and only
+        // for the node where a walk stops)
+        if (warp == 0) {
+            if (crank == 0 && lane == 0) {
+                P.node_accept[node_idx] = accepted;
+                if (PATH) P.path_next[b] = accepted;
+                reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
+                    make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
+            }
+        }
+        if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
+        status_bits = __reduce_or_sync(0xffffffffu, status_bits);
+        if (status_bits && lane == 0) atomicOr(P.status + b, status_bits);
+        next_item();
+    }
+
+    if (warp == kFetchWarp) cp_async_wait_all();
+    // no CTA may leave while a peer can still write into its shared memory
+    cluster_sync_all();
+}
+
+}  // namespace mcsd

@@ -1,0 +1,245 @@
+// sample_kernel: the k candidate draws of a node from the draft distribution, with
+// replacement or without (Eq. 1), top-k at temperature 0.
+#pragma once
+
+#include "mcsd_common.cuh"
+
+namespace mcsd {
+
+struct SampleParams {
+    const void *draft;
+    const float *unif_draw;  // [B][n_nodes] the uniform that draws the token of each draft node
+    int32_t *cand;           // [B][n_nodes]
+    int32_t *status;         // [B] or null
+    long long ld_d;
+    int32_t n_nodes, n_internal, V;
+    int32_t node_begin, n_range;  // nodes node_begin .. node_begin + n_range - 1 of every tree
+    int32_t mode;
+    int32_t vector_ok;
+    float scale;                  // log2(e)/T, or 0 for top-k
+    uint16_t child_first[MCSD_MAX_NODES];
+    uint8_t child_count[MCSD_MAX_NODES];
+};
+
+// One CTA per (sequence, node with children): draws the tokens of the node's k children from
+// softmax(draft row / T) by inverse CDF in token order with one supplied uniform each
+// (Section 3.2).  With replacement the k draws are independent; without (Eq. 1) every
+// drawn token is taken out of the distribution before the next draw, which here means
+// subtracting its weight from the partial sums of its lane, its warp's run and the
+// element scan.  The row is read once (twice for its maximum, the second time from L2);
+// temperature 0 takes the k largest logits instead (lowest index first on ties).
+// NT threads per CTA: 512 (two CTAs per SM, two independent chains) when the vocabulary fits
+// 16 steps per warp, else 1024.
+template <int DT, int NT>
+__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
+sample_kernel(const __grid_constant__ SampleParams P)
+{
+    using E = Elem<DT>;
+    constexpr int GV = E::kVec;
+    constexpr int kStep = 32 * GV;
+    constexpr int kW = NT / 32;  // warps
+    constexpr int kMaxSteps = MCSD_MAX_VOCAB / 32 / kStep;  // steps of a warp's run (the host picks NT so that they suffice)
+    __shared__ float s_wtot[32];
+    __shared__ float s_red[32];
+    __shared__ int s_redi[32];
+    __shared__ int32_t s_rem_tok[MCSD_MAX_CHILDREN];
+    __shared__ int s_pick;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x / P.n_range, n = P.node_begin + (blockIdx.x - b * P.n_range);
+    const int k = P.child_count[n], first = P.child_first[n];
+    if (k == 0) return;
+    int32_t *out = P.cand + static_cast<long long>(b) * P.n_nodes + first;
+    const unsigned char *row = reinterpret_cast<const unsigned char *>(P.draft) +
+        (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes;
+    auto load_group = [&](int x0, float *v) {   // GV logits from x0 on, -inf past the vocabulary
+        if (P.vector_ok && x0 + GV <= P.V) {
+            E::unpack(__ldg(reinterpret_cast<const uint4 *>(row + static_cast<size_t>(x0) * E::kBytes)), v);
+        } else {
+#pragma unroll
+            for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
+        }
+    };
+    const int run = ((P.V + kW - 1) / kW + kStep - 1) / kStep * kStep;
+    const int x_lo = warp * run;
+    int x_hi = x_lo + run;
+    x_hi = x_hi > P.V ? P.V : x_hi;
+
+    if (P.scale == 0.f) {
+        // ---- top-k: k block-wide maxima, each over the elements that come after the previous
+        // pick in the order (logit descending, index ascending)
+        float pv = INFINITY;
+        int pi = -1;
+        for (int i = 0; i < k; ++i) {
+            float best = -INFINITY;
+            int best_i = 0x7fffffff;
+            for (int x0 = x_lo + lane * GV; x0 < x_hi; x0 += kStep) {
+                float v[GV];
+                load_group(x0, v);
+#pragma unroll
+                for (int e = 0; e < GV; ++e) {
+                    const int x = x0 + e;
+                    const bool after = i == 0 || v[e] < pv || (v[e] == pv && x > pi);
+                    if (x < P.V && after && v[e] > best) { best = v[e]; best_i = x; }  // ascending x: ties keep the lowest
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+                if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+            }
+            if (lane == 0) { s_red[warp] = best; s_redi[warp] = best_i; }
+            __syncthreads();
+            best = lane < kW ? s_red[lane] : -INFINITY;
+            best_i = lane < kW ? s_redi[lane] : 0x7fffffff;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+                if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+            }
+            pv = best;
+            pi = best_i == 0x7fffffff ? -1 : best_i;
+            if (tid == 0) out[i] = pi;
+            __syncthreads();
+        }
+        return;
+    }
+
+    // ---- reference of the row: ceil(max * scale)
+    float mx = -INFINITY;
+    for (int x0 = x_lo + lane * GV; x0 < x_hi; x0 += kStep) {
+        float v[GV];
+        load_group(x0, v);
+#pragma unroll
+        for (int e = 0; e < GV; ++e) mx = fmaxf(mx, v[e]);
+    }
+    mx = warp_max(mx);
+    if (lane == 0) s_red[warp] = mx;
+    __syncthreads();
+    const float ref = int_ref(warp_max(lane < kW ? s_red[lane] : -INFINITY) * P.scale);
+    const float ref0 = ref == -INFINITY ? 0.f : ref;
+    auto weights = [&](int x0, float *w) {
+        float v[GV];
+        load_group(x0, v);
+#pragma unroll
+        for (int e = 0; e < GV; ++e) w[e] = ex2f(fmaf(v[e], P.scale, -ref0));
+    };
+    // ---- unnormalised weights: per lane the sum of its group in every step, per warp its run
+    float g[kMaxSteps];
+    float mass = 0.f;
+#pragma unroll
+    for (int st = 0; st < kMaxSteps; ++st) {
+        g[st] = 0.f;
+        const int x0 = x_lo + st * kStep + lane * GV;
+        if (x0 < x_hi) {
+            float w[GV];
+            weights(x0, w);
+#pragma unroll
+            for (int e = 0; e < GV; ++e) g[st] += w[e];
+            mass += g[st];
+        }
+    }
+    mass = warp_sum(mass);
+    if (lane == 0) s_wtot[warp] = mass;
+    __syncthreads();
+
+    int n_rem = 0;  // tokens taken out so far (Eq. 1); the same in every thread
+    for (int i = 0; i < k; ++i) {
+        const float u = P.unif_draw[static_cast<long long>(b) * P.n_nodes + first + i];
+        // the run that holds the quantile (every warp finds the same one)
+        const float m = lane < kW ? s_wtot[lane] : 0.f;
+        const float total = warp_sum(m);
+        const float target = u * total;
+        const float inc = warp_scan_incl(m, lane);
+        const unsigned hit = __ballot_sync(0xffffffffu, m > 0.f && inc > target);
+        const unsigned pos = __ballot_sync(0xffffffffu, m > 0.f);
+        const int pick = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
+        int found = -1;
+        if (pick >= 0 && total > 0.f && warp == pick) {
+            const float tgt = target - __shfl_sync(0xffffffffu, inc - m, pick);
+            float tj;
+            warp_multi_sum<kMaxSteps>(g, lane, tj);
+            int ps = -1, last_s = -1;
+            float runsum = 0.f, ps_before = 0.f;
+#pragma unroll
+            for (int st = 0; st < kMaxSteps; ++st) {
+                const float ms = __shfl_sync(0xffffffffu, tj, st * (32 / kMaxSteps));
+                if (ms > 0.f) {
+                    last_s = st;
+                    if (ps < 0 && runsum + ms > tgt) { ps = st; ps_before = runsum; }
+                }
+                runsum += ms;
+            }
+            float t2 = tgt - ps_before;
+            if (ps < 0) { ps = last_s; t2 = INFINITY; }   // rounding: take the run's last element with mass
+            if (ps >= 0) {
+                float gs = g[0];
+#pragma unroll
+                for (int st = 1; st < kMaxSteps; ++st) gs = (ps == st) ? g[st] : gs;
+                const float gi = warp_scan_incl(gs, lane);
+                const unsigned h2 = __ballot_sync(0xffffffffu, gs > 0.f && gi > t2);
+                const unsigned p2 = __ballot_sync(0xffffffffu, gs > 0.f);
+                if (p2) {
+                    const int l = h2 ? __ffs(h2) - 1 : 31 - __clz(p2);
+                    int pe = -1, last = -1;
+                    if (lane == l) {
+                        const int x0 = x_lo + ps * kStep + lane * GV;
+                        float w[GV];
+                        weights(x0, w);
+                        const float rem = t2 - (gi - gs);
+                        float acc = 0.f;
+#pragma unroll
+                        for (int e = 0; e < GV; ++e) {
+                            bool gone = false;
+                            for (int j = 0; j < n_rem; ++j) gone |= s_rem_tok[j] == x0 + e;
+                            if (!gone && w[e] > 0.f) {
+                                acc += w[e];
+                                last = e;
+                                if (pe < 0 && acc > rem) pe = e;
+                            }
+                        }
+                        if (pe < 0) pe = last;
+                        if (pe >= 0 && P.mode == 1) {
+                            // Eq. 1: the drawn token leaves the distribution.  The group's sum is
+                            // formed again from the tokens that remain (subtracting would lose
+                            // everything when the drawn token dominated the group)
+                            float rest = 0.f;
+#pragma unroll
+                            for (int e = 0; e < GV; ++e) {
+                                bool gone = e == pe;
+                                for (int j = 0; j < n_rem; ++j) gone |= s_rem_tok[j] == x0 + e;
+                                if (!gone) rest += w[e];
+                            }
+#pragma unroll
+                            for (int st = 0; st < kMaxSteps; ++st)
+                                if (st == ps) g[st] = rest;
+                        }
+                    }
+                    found = __shfl_sync(0xffffffffu, pe < 0 ? -1 : x_lo + ps * kStep + lane * GV + pe, l);
+                    if (P.mode == 1 && found >= 0) {
+                        // ... and so is the run's total, from the lanes' current group sums
+                        float rs = 0.f;
+#pragma unroll
+                        for (int st = 0; st < kMaxSteps; ++st) rs += g[st];
+                        rs = warp_sum(rs);
+                        if (lane == 0) s_wtot[warp] = rs;
+                    }
+                }
+            }
+            if (lane == 0) s_pick = found;
+        }
+        if (pick < 0 || !(total > 0.f)) { if (tid == 0) s_pick = -1; }
+        __syncthreads();
+        found = s_pick;
+        if (tid == 0) {
+            out[i] = found;
+            if (found < 0 && P.status) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
+            if (P.mode == 1) s_rem_tok[n_rem] = found;
+        }
+        if (P.mode == 1 && found >= 0) ++n_rem;
+        __syncthreads();
+    }
+}
+
+}  // namespace mcsd
