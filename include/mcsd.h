@@ -145,6 +145,9 @@ typedef struct mcsd_desc {
  *                  NULL to skip
  * Rows whose base address and stride are multiples of 16 bytes take the bulk-copy
  * (TMA) path; any other layout is accepted and takes a slower plain-load path.
+ * All ld elements of every row, the last one included, must be readable memory: on
+ * the bulk-copy path a row is loaded in 16-byte vectors, so up to 15 bytes of the
+ * padding behind element vocab-1 may be read (their values are ignored).
  */
 int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                 const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,

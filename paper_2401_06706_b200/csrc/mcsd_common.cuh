@@ -65,6 +65,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 template <int DT> struct Elem;
 template <> struct Elem<MCSD_DTYPE_F32> {
     static constexpr int kBytes = 4, kVec = 4;
+    static constexpr uint32_t kNegInfWord = 0xff800000u;  // 32 bits of -inf elements
     static __device__ __forceinline__ void unpack(const uint4 &r, float *o) {
         o[0] = __uint_as_float(r.x); o[1] = __uint_as_float(r.y);
         o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
@@ -84,6 +85,7 @@ template <> struct Elem<MCSD_DTYPE_F32> {
 };
 template <> struct Elem<MCSD_DTYPE_BF16> {
     static constexpr int kBytes = 2, kVec = 8;
+    static constexpr uint32_t kNegInfWord = 0xff80ff80u;
     static __device__ __forceinline__ void unpack(const uint4 &r, float *o) {
         o[0] = __uint_as_float(r.x << 16); o[1] = __uint_as_float(r.x & 0xffff0000u);
         o[2] = __uint_as_float(r.y << 16); o[3] = __uint_as_float(r.y & 0xffff0000u);
@@ -113,6 +115,7 @@ template <> struct Elem<MCSD_DTYPE_BF16> {
 };
 template <> struct Elem<MCSD_DTYPE_F16> {
     static constexpr int kBytes = 2, kVec = 8;
+    static constexpr uint32_t kNegInfWord = 0xfc00fc00u;
     static __device__ __forceinline__ void unpack(const uint4 &r, float *o) {
         const __half2 *h = reinterpret_cast<const __half2 *>(&r);
 #pragma unroll
@@ -213,6 +216,17 @@ __device__ __forceinline__ uint4 ld_stream_v4(const void *p) {
     uint4 r;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+// The same under a predicate: where it is false nothing is read and all four words are `fill`.
+// A run of these has no branch between the loads, so they are all in flight together.
+__device__ __forceinline__ uint4 ld_stream_v4_if(const void *p, bool pred, uint32_t fill) {
+    uint4 r;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\t"
+                 "mov.u32 %0, %6;\n\tmov.u32 %1, %6;\n\tmov.u32 %2, %6;\n\tmov.u32 %3, %6;\n\t"
+                 "@q ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];\n\t}"
+                 : "=&r"(r.x), "=&r"(r.y), "=&r"(r.z), "=&r"(r.w)
+                 : "l"(p), "r"(static_cast<uint32_t>(pred)), "r"(fill));
     return r;
 }
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {

@@ -291,22 +291,43 @@ node_kernel(const __grid_constant__ NodeParams P)
 #pragma unroll
                 for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
             }
-        } else {
+        } else if constexpr (DIRECT) {
 #pragma unroll
             for (int j = 0; j < NG; ++j) {
                 const int g = g0 + j * 32;
                 float f[GV];
-                if (!DIRECT && g < n_full_groups) {
-                    E::unpack(ld_stream_v4(t_row + static_cast<size_t>(g) * 16), f);
-                } else if (g * GV >= n_mine) {  // wholly past the data
 #pragma unroll
-                    for (int e = 0; e < GV; ++e) f[e] = -INFINITY;
-                } else {
-#pragma unroll
-                    for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(t_row, g * GV + e) : -INFINITY;
-                }
+                for (int e = 0; e < GV; ++e) f[e] = (g * GV + e < n_mine) ? E::load(t_row, g * GV + e) : -INFINITY;
 #pragma unroll
                 for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
+            }
+        } else {
+            // a warp at the ragged end of the vocabulary: predicated vector loads of the groups
+            // that hold data (no branch between them, so their latencies overlap as in the
+            // common case), -inf where there is none ...
+            const int n_groups = (n_mine + GV - 1) / GV;
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                const int g = g0 + j * 32;
+                float f[GV];
+                E::unpack(ld_stream_v4_if(t_row + static_cast<size_t>(g) * 16, g < n_groups, E::kNegInfWord), f);
+#pragma unroll
+                for (int e = 0; e < GV; e += 2) tv[(j * GV + e) / 2] = pack2(f[e], f[e + 1]);
+            }
+            // ... and where the vocabulary is no multiple of the vector width, the last group's
+            // elements past the end (padding of the 16-byte aligned row) are set to -inf
+            if (n_groups != n_full_groups) {
+#pragma unroll
+                for (int j = 0; j < NG; ++j) {
+                    if (g0 + j * 32 == n_full_groups) {
+#pragma unroll
+                        for (int e = 0; e < GV; e += 2) {
+                            const int x = n_full_groups * GV + e;
+                            f32x2 &v = tv[(j * GV + e) / 2];
+                            v = pack2(x < n_mine ? v.x : -INFINITY, x + 1 < n_mine ? v.y : -INFINITY);
+                        }
+                    }
+                }
             }
         }
         // Each warp exponentiates relative to its own integer reference; the factor to the
