@@ -119,7 +119,7 @@ def dist_env():
     return rank, world, local
 
 
-def pick_workload(name: str, batch: int = 0) -> synth.Workload:
+def pick_workload(name: str, batch: int = 0, logit_dtype: str = "") -> synth.Workload:
     from dataclasses import replace
     named = synth.named_workloads()
     found = named.get(name)
@@ -129,6 +129,8 @@ def pick_workload(name: str, batch: int = 0) -> synth.Workload:
                 found = w
     if found is None:
         raise SystemExit(f"unknown workload {name!r}; named: {sorted(named)}")
+    if logit_dtype:
+        found = replace(found, dtype=logit_dtype)
     return replace(found, batch=batch) if batch > 0 else found
 
 
@@ -176,7 +178,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    w = pick_workload(args.workload, args.batch)
+    w = pick_workload(args.workload, args.batch, args.logit_dtype)
     from dataclasses import replace
     # size the per-step sample so that the whole run takes about a minute of wall time
     probe = synth.make_inputs(replace(w, batch=min(w.batch, 8)), "cpu")
@@ -236,7 +238,7 @@ def run_cuda(args):
     dev = torch.device("cuda", torch.cuda.current_device())
     binding.load_library()       # raises if the CUDA library is missing: no fallback
 
-    w = shard_for_rank(pick_workload(args.workload, args.batch), rank, world)
+    w = shard_for_rank(pick_workload(args.workload, args.batch, args.logit_dtype), rank, world)
     inp = synth.make_inputs(w, dev)
     st = inp.stats
     ver = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[w.dtype], dev)
@@ -326,7 +328,7 @@ def run_cuda(args):
                 "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_avg": node_ms_avg,
                 "kernel_ms_min": min(node_ms), "step_share": node_ms_avg / ms_per_step,
                 "traffic": recorded_traffic(w.batch * st["n_nodes"])
-                if (w.name == "cfg5_largest" and args.form == "all_node") else None}
+                if (w.name == "cfg5_largest" and w.dtype == "fp32" and args.form == "all_node") else None}
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside
     e2e = None
@@ -478,6 +480,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch of the workload (profiling)")
+    ap.add_argument("--logit-dtype", default="", choices=["", "fp32", "bf16", "fp16"],
+                    help="override the logit type of the workload (profiling)")
     ap.add_argument("--form", default="all_node", choices=["all_node", "path"],
                     help="all_node: every node of every tree is evaluated (the measured configuration); "
                          "path: mcsd_verify_path, only the nodes the walks visit, one launch per level")

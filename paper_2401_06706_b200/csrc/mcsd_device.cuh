@@ -31,8 +31,8 @@
 // p_{n+1} ~ max(p_n - q_n, 0) by induction and holds for every rejection that can
 // occur with r in (0,1).  The test of candidate n+1 is r <= [P_n(x~)/S_n]/[q(x~)/W_n].
 // So one rejection costs one scalar-parameter reduction over the on-chip p and q,
-// and nothing is written back.  c_1 = 1 whatever the candidates are, so the first
-// reduction is started before the first test has been decided.
+// and nothing is written back; a node whose first candidate is accepted costs no
+// reduction at all.
 //
 // Softmax references are integers (ceil of the scaled row maximum, in log2 units), so
 // moving a partial sum from one reference to another is an exact multiplication by a
