@@ -210,7 +210,8 @@ int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const voi
  *   temperature 0                  the k largest draft logits in descending order, lowest
  *                                  index first among equals; uniforms_draw may be NULL
  * A draft model produces the rows of one tree level at a time, hence the node range.
- *   draft_logits   device [B][n_internal][ld_draft]
+ *   draft_logits   device [B][n_internal][ld_draft]; as in mcsd_verify, all ld_draft elements
+ *                  of the rows in range must be readable (16-byte vector loads)
  *   tree_parent    HOST   [n_nodes]
  *   uniforms_draw  device [B][n_nodes] float32 in (0, 1)
  *   cand_tokens    device [B][n_nodes], written for the children of the nodes in range

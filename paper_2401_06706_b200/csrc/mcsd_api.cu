@@ -621,6 +621,14 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
     // 16 warps cover the row within the per-warp step budget (half of MCSD_MAX_VOCAB / 32 elements
     // per warp at 1024 threads) when the vocabulary is at most half the maximum
     const bool small = desc->vocab <= MCSD_MAX_VOCAB / 2;
+    {
+        // CTAs resident at once (two of 512 threads or one of 1024 per SM): how far ahead the
+        // kernel asks rows into L2
+        int dev = 0, n_sm = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MCSD_ERR_CUDA;
+        p.prefetch_ahead = n_sm * (small ? 2 : 1);
+    }
     if (small) {
         switch (desc->dtype) {
         case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32, 512><<<grid, 512, 0, stream>>>(p); break;

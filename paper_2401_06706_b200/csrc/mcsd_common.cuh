@@ -229,6 +229,16 @@ __device__ __forceinline__ uint4 ld_stream_v4_if(const void *p, bool pred, uint3
                  : "l"(p), "r"(static_cast<uint32_t>(pred)), "r"(fill));
     return r;
 }
+// Predicated 128-bit load that may stay in the caches (for data that is read again soon).
+__device__ __forceinline__ uint4 ld_v4_if(const void *p, bool pred, uint32_t fill) {
+    uint4 r;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\t"
+                 "mov.u32 %0, %6;\n\tmov.u32 %1, %6;\n\tmov.u32 %2, %6;\n\tmov.u32 %3, %6;\n\t"
+                 "@q ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];\n\t}"
+                 : "=&r"(r.x), "=&r"(r.y), "=&r"(r.z), "=&r"(r.w)
+                 : "l"(p), "r"(static_cast<uint32_t>(pred)), "r"(fill));
+    return r;
+}
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));

@@ -16,6 +16,7 @@ struct SampleParams {
     int32_t node_begin, n_range;  // nodes node_begin .. node_begin + n_range - 1 of every tree
     int32_t mode;
     int32_t vector_ok;
+    int32_t prefetch_ahead;       // CTAs resident at once: the row of the CTA that far ahead is asked into L2
     float scale;                  // log2(e)/T, or 0 for top-k
     uint16_t child_first[MCSD_MAX_NODES];
     uint8_t child_count[MCSD_MAX_NODES];
@@ -26,7 +27,8 @@ struct SampleParams {
 // (Section 3.2).  With replacement the k draws are independent; without (Eq. 1) every
 // drawn token is taken out of the distribution before the next draw, which here means
 // subtracting its weight from the partial sums of its lane, its warp's run and the
-// element scan.  The row is read once (twice for its maximum, the second time from L2);
+// element scan.  The row is read twice, for its maximum and for the weights, both times from
+// L2: the CTA that held this CTA's place before asked for the row while it computed;
 // temperature 0 takes the k largest logits instead (lowest index first on ties).
 // NT threads per CTA: 512 (two CTAs per SM, two independent chains) when the vocabulary fits
 // 16 steps per warp, else 1024.
@@ -59,12 +61,43 @@ sample_kernel(const __grid_constant__ SampleParams P)
             for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
         }
     };
+    // The same where `on` holds and -inf where it does not, without a branch on 16-byte aligned
+    // rows (one predicated vector load; the padding an incomplete last group brings along is
+    // masked), so that the loads of an unrolled loop are in flight together.
+    const bool tail_mask = P.V % GV != 0;
+    auto load_group_if = [&](int x0, bool on, float *v) {
+        if (P.vector_ok) {
+            E::unpack(ld_v4_if(row + static_cast<size_t>(x0) * E::kBytes, on && x0 < P.V, E::kNegInfWord), v);
+            if (tail_mask) {
+#pragma unroll
+                for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? v[e] : -INFINITY;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < GV; ++e) v[e] = (on && x0 + e < P.V) ? E::load(row, x0 + e) : -INFINITY;
+        }
+    };
+    // The CTA that takes this one's place when it has finished is about `prefetch_ahead` blocks
+    // further on: its row is asked into L2 now, so that HBM streams while this CTA computes and
+    // that CTA's two passes both read from L2.
+    auto prefetch_later_row = [&]() {
+        if (P.vector_ok && tid == 0) {
+            const long long nb = static_cast<long long>(blockIdx.x) + P.prefetch_ahead;
+            if (nb < static_cast<long long>(gridDim.x)) {
+                const int b2 = static_cast<int>(nb / P.n_range), n2 = P.node_begin + static_cast<int>(nb - static_cast<long long>(b2) * P.n_range);
+                const unsigned char *r2 = reinterpret_cast<const unsigned char *>(P.draft) +
+                    (static_cast<long long>(b2) * P.n_internal + n2) * P.ld_d * E::kBytes;
+                bulk_prefetch_l2(r2, (static_cast<uint32_t>(P.V) * E::kBytes) & ~15u);
+            }
+        }
+    };
     const int run = ((P.V + kW - 1) / kW + kStep - 1) / kStep * kStep;
     const int x_lo = warp * run;
     int x_hi = x_lo + run;
     x_hi = x_hi > P.V ? P.V : x_hi;
 
     if (P.scale == 0.f) {
+        prefetch_later_row();
         // ---- top-k: k block-wide maxima, each over the elements that come after the previous
         // pick in the order (logit descending, index ascending)
         float pv = INFINITY;
@@ -108,17 +141,30 @@ sample_kernel(const __grid_constant__ SampleParams P)
 
     // ---- reference of the row: ceil(max * scale)
     float mx = -INFINITY;
-    for (int x0 = x_lo + lane * GV; x0 < x_hi; x0 += kStep) {
-        float v[GV];
-        load_group(x0, v);
+    {
+        // four loads in flight per thread (more cost registers the two resident CTAs do not have)
+        constexpr int U = 4 < kMaxSteps ? 4 : kMaxSteps;
+#pragma unroll 1
+        for (int s0 = 0; s0 < kMaxSteps; s0 += U) {
+            if (x_lo + s0 * kStep >= x_hi) break;
+            float v[U][GV];
 #pragma unroll
-        for (int e = 0; e < GV; ++e) mx = fmaxf(mx, v[e]);
+            for (int u = 0; u < U; ++u) {
+                const int x0 = x_lo + (s0 + u) * kStep + lane * GV;
+                load_group_if(x0, x0 < x_hi, v[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int e = 0; e < GV; e += 2) mx = max3(mx, v[u][e], v[u][e + 1]);
+        }
     }
     mx = warp_max(mx);
     if (lane == 0) s_red[warp] = mx;
     __syncthreads();
     const float ref = int_ref(warp_max(lane < kW ? s_red[lane] : -INFINITY) * P.scale);
     const float ref0 = ref == -INFINITY ? 0.f : ref;
+    prefetch_later_row();
     auto weights = [&](int x0, float *w) {
         float v[GV];
         load_group(x0, v);
@@ -130,15 +176,14 @@ sample_kernel(const __grid_constant__ SampleParams P)
     float mass = 0.f;
 #pragma unroll
     for (int st = 0; st < kMaxSteps; ++st) {
-        g[st] = 0.f;
         const int x0 = x_lo + st * kStep + lane * GV;
-        if (x0 < x_hi) {
-            float w[GV];
-            weights(x0, w);
+        float v[GV];
+        load_group_if(x0, x0 < x_hi, v);   // weight 0 where there is no element
+        float gs = 0.f;
 #pragma unroll
-            for (int e = 0; e < GV; ++e) g[st] += w[e];
-            mass += g[st];
-        }
+        for (int e = 0; e < GV; ++e) gs += ex2f(fmaf(v[e], P.scale, -ref0));
+        g[st] = gs;
+        mass += gs;
     }
     mass = warp_sum(mass);
     if (lane == 0) s_wtot[warp] = mass;
