@@ -48,26 +48,21 @@ argmax_kernel(const __grid_constant__ ArgmaxParams P)
         if (P.vector_ok) {
             const int n_vec = P.V / VEC;
             const uint4 *src = reinterpret_cast<const uint4 *>(t_row);
-            int v = tid;
-            for (; v + 3 * kThreads < n_vec; v += 4 * kThreads) {
-                uint4 r[4];
+            // eight predicated loads in flight per thread, the ragged end of the row included:
+            // where the predicate is off the vector is -inf, which never wins
+            for (int v = tid; v < n_vec; v += 8 * kThreads) {
+                uint4 r[8];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) r[u] = __ldg(src + v + u * kThreads);
+                for (int u = 0; u < 8; ++u)
+                    r[u] = ld_v4_if(src + v + u * kThreads, v + u * kThreads < n_vec, E::kNegInfWord);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < 8; ++u) {
                     float f[VEC];
                     E::unpack(r[u], f);
 #pragma unroll
                     for (int e = 0; e < VEC; ++e)
                         if (f[e] > best) { best = f[e]; best_i = (v + u * kThreads) * VEC + e; }
                 }
-            }
-            for (; v < n_vec; v += kThreads) {
-                float f[VEC];
-                E::unpack(__ldg(src + v), f);
-#pragma unroll
-                for (int e = 0; e < VEC; ++e)
-                    if (f[e] > best) { best = f[e]; best_i = v * VEC + e; }
             }
             for (int x = n_vec * VEC + tid; x < P.V; x += kThreads) {
                 const float f = E::load(t_row, x);
