@@ -74,6 +74,29 @@ def test_padded_row_stride():
     assert_parity(inp, out)
 
 
+@pytest.mark.parametrize("T", [1.0, 0.0])
+@pytest.mark.parametrize("dtype,vocab", [("fp32", 5003), ("bf16", 5003), ("fp16", 8197), ("fp32", 32002), ("bf16", 32001)])
+def test_aligned_rows_whose_vocabulary_ends_inside_a_vector(dtype, vocab, T):
+    """Rows padded to a 16-byte multiple take the vector path; the vector that holds the last
+    elements also holds padding, here larger than every logit, which must not count."""
+    w = synth.Workload("tail", 4, vocab, "3x2", dtype, "normal", 2.5, 1.0, 1.0, T, 1 if T > 0 else 0, 99 + vocab)
+    inp = synth.make_inputs(w, "cuda")
+    dt = synth.TORCH_DTYPES[dtype]
+    per16 = 16 // inp.target.element_size()
+    ld = (vocab + per16 - 1) // per16 * per16
+    assert ld > vocab
+    st = inp.stats
+    tpad = torch.full((4, st["n_nodes"], ld), 50.0, dtype=dt, device="cuda")
+    dpad = torch.full((4, st["n_internal"], ld), 50.0, dtype=dt, device="cuda")
+    tpad[:, :, :vocab] = inp.target
+    dpad[:, :, :vocab] = inp.draft
+    v = binding.Verifier(4, inp.parent, vocab, dt, "cuda", node_outputs=True)
+    out = v.mcsd_verify(tpad[:, :, :vocab], dpad[:, :, :vocab] if T > 0 else None, inp.cand, inp.unif, T, w.mode)
+    torch.cuda.synchronize()
+    assert v.desc.ld_target == ld and (ld * inp.target.element_size()) % 16 == 0
+    assert_parity(inp, out)
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("cluster,ept", [(1, 64), (2, 16), (4, 16), (8, 16), (8, 32), (2, 64), (4, 32)])
 def test_forced_cluster_shapes(cluster, ept, dtype, monkeypatch):

@@ -4,6 +4,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from oracle import compare as cmp
 from paper_2401_06706_b200 import binding, synth
 
@@ -51,6 +52,34 @@ def test_draws_match_the_oracle(vocab, kconfig, mode, dtype):
         for n in range(inp.stats["n_internal"]):
             ch = c[:, first[n]:first[n] + count[n]]
             assert all(len(set(row)) == len(row) for row in ch.tolist())
+
+
+@pytest.mark.parametrize("T,mode", [(1.0, 0), (1.0, 1), (0.0, 0)])
+@pytest.mark.parametrize("dtype,vocab", [("fp32", 5003), ("bf16", 5003), ("fp16", 32001)])
+def test_aligned_rows_whose_vocabulary_ends_inside_a_vector(dtype, vocab, T, mode):
+    """Padded, 16-byte aligned rows: the padding in the last vector is larger than every logit
+    and must neither be drawn nor carry weight."""
+    w = synth.Workload("sample_tail", 5, vocab, "4x2", dtype, "normal", 2.5, 1.0, 1.0, 1.0, mode, 300 + vocab)
+    inp, u = _inputs(w, 5 + vocab)
+    per16 = 16 // inp.draft.element_size()
+    ld = (vocab + per16 - 1) // per16 * per16
+    assert ld > vocab
+    dpad = torch.full((5, inp.stats["n_internal"], ld), 50.0, dtype=inp.draft.dtype, device="cuda")
+    dpad[:, :, :vocab] = inp.draft
+    cand = binding.mcsd_sample_candidates(dpad[:, :, :vocab], inp.parent, u, T, mode)
+    torch.cuda.synchronize()
+    c = cand.cpu().numpy()
+    assert (c[:, 1:] >= 0).all() and (c[:, 1:] < vocab).all()
+    if T > 0:
+        _check(inp, u, cand, T, mode)
+    else:
+        d = inp.draft.to(torch.float32).cpu().numpy()
+        first, count = synth.children_ranges(inp.parent)
+        for b in range(5):
+            for n in range(inp.stats["n_internal"]):
+                want = oracle.topk(d[b, n], int(count[n]))
+                got = c[b, first[n]:first[n] + count[n]]
+                assert (d[b, n][got] == d[b, n][want]).all()
 
 
 @pytest.mark.parametrize("T", [0.3, 0.7, 1.7])
