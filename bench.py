@@ -466,6 +466,78 @@ def run_sweep(args):
         out.close()
 
 
+def run_stage(args):
+    """--stage sample / greedy: one kernel of the wider path on the same workload, one GPU, device
+    timed.  sample: mcsd_sample_candidates over all internal nodes (the draft rows once); greedy:
+    the verification step at temperature 0 (argmax kernel; the target rows once).  One JSON line."""
+    from paper_2401_06706_b200 import binding
+    from dataclasses import replace
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback for the product path)"
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    binding.load_library()
+    w = pick_workload(args.workload, args.batch, args.logit_dtype)
+    if args.stage == "greedy":
+        w = replace(w, temperature=0.0)
+    inp = synth.make_inputs(w, dev)
+    st = inp.stats
+    esize = inp.target.element_size()
+    if args.stage == "sample":
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(w.seed)
+        u = synth.open_uniforms((w.batch, st["n_nodes"]), gen, dev)
+        cand = torch.full((w.batch, st["n_nodes"]), -1, dtype=torch.int32, device=dev)
+        call = lambda: binding.mcsd_sample_candidates(inp.draft, inp.parent, u, w.temperature, w.mode, cand=cand)
+        algo = w.batch * st["n_internal"] * w.vocab * esize + 8 * w.batch * st["n_draft"]
+        units, metric, unit, kernel = w.batch * st["n_draft"], "sampled_candidate_tokens_per_sec", "tokens/s", "sample_kernel"
+    else:
+        ver = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[w.dtype], dev, node_outputs=True)
+        call = lambda: ver.mcsd_verify_nodes(inp.target, None, inp.cand, None, 0.0, w.mode)
+        algo = w.batch * st["n_nodes"] * w.vocab * esize + 4 * w.batch * st["n_nodes"]
+        units, metric, unit, kernel = w.batch * st["n_draft"], METRIC, UNIT, "argmax_kernel"
+    for _ in range(max(args.warmup, 3)):
+        call()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.25)
+    torch.cuda.synchronize()
+    t_host0 = time.time()
+    for e0, e1 in ev:
+        e0.record()
+        call()
+        e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop(t_host0, time.time())
+    ms = [a.elapsed_time(b) for a, b in ev]
+    ms_avg = sum(ms) / len(ms)
+    peak, peak_kind = measured_peaks()
+    achieved = algo / (ms_avg * 1e-3) / 1e9
+    # parity of this stage on the first sequences, against the oracle
+    n_seq = min(w.batch, 8)
+    if args.stage == "sample":
+        from oracle import compare as cmp
+        rep = cmp.compare_samples(inp.draft[:n_seq].to(torch.float32).cpu().numpy(), inp.parent, u[:n_seq].cpu().numpy(),
+                                  w.temperature, w.mode, cand[:n_seq].cpu().numpy(), 0, None)
+        parity = {"sequences": n_seq, "draws": rep.n_draws, "tolerated": rep.n_tolerated, "ok": bool(rep.ok)}
+    else:
+        import oracle
+        t, _, c, uu = inp.host_f32(0, n_seq)
+        ref = oracle.verify(t, None, inp.parent, c, uu, 0.0, w.mode, want_residual=False)
+        got = ver.node_accept[:n_seq].cpu().numpy()
+        parity = {"sequences": n_seq, "nodes": int(got.size), "ok": bool((got == ref.node_accept).all())}
+    line = {"metric": metric, "value": units / (ms_avg * 1e-3), "unit": unit, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_avg, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "stage": args.stage,
+            "config": workload_config(w, st, l2="inputs far larger than the 126 MB L2" if algo > 4 * 126e6 else "inputs not much larger than L2"),
+            "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}",
+                         "unit": "GB/s", "frac": achieved / peak, "algorithmic_bytes_per_launch": algo,
+                         "kernel_ms_avg": ms_avg, "kernel_ms_min": min(ms), "traffic": None},
+            "gpu_launches": args.steps, "clocks": clocks, "parity_on_oracle_sample": parity}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -485,6 +557,9 @@ def main():
     ap.add_argument("--form", default="all_node", choices=["all_node", "path"],
                     help="all_node: every node of every tree is evaluated (the measured configuration); "
                          "path: mcsd_verify_path, only the nodes the walks visit, one launch per level")
+    ap.add_argument("--stage", default="verify", choices=["verify", "sample", "greedy"],
+                    help="verify: the bench line of the verification step (default); sample: time the candidate "
+                         "sampler on the workload's draft rows; greedy: the verification step at temperature 0")
     ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the bench line")
     ap.add_argument("--sweep-filter", default="", help="only sweep points whose name contains this text")
     ap.add_argument("--sweep-out", default="", help="file for one JSON line per sweep point")
@@ -495,6 +570,8 @@ def main():
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.stage != "verify":
+        run_stage(args)
     else:
         run_cuda(args)
 

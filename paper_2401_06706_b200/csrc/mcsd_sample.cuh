@@ -61,20 +61,24 @@ sample_kernel(const __grid_constant__ SampleParams P)
             for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
         }
     };
-    // The same where `on` holds and -inf where it does not, without a branch on 16-byte aligned
-    // rows (one predicated vector load; the padding an incomplete last group brings along is
-    // masked), so that the loads of an unrolled loop are in flight together.
+    // Branch-free variant for unrolled loops (their loads are then in flight together): on
+    // 16-byte aligned rows a group that starts past the vocabulary reads the row's last group
+    // instead, i.e. values that are in the row anyway.  That leaves a maximum unchanged; a sum
+    // must drop those groups (x0 >= V).  The padding an incomplete last group brings along is
+    // masked to -inf.
     const bool tail_mask = P.V % GV != 0;
-    auto load_group_if = [&](int x0, bool on, float *v) {
+    const int x_last = (P.V - 1) / GV * GV;
+    auto load_group_clamped = [&](int x0, float *v) {
         if (P.vector_ok) {
-            E::unpack(ld_v4_if(row + static_cast<size_t>(x0) * E::kBytes, on && x0 < P.V, E::kNegInfWord), v);
+            const int xc = x0 < x_last ? x0 : x_last;
+            E::unpack(__ldg(reinterpret_cast<const uint4 *>(row + static_cast<size_t>(xc) * E::kBytes)), v);
             if (tail_mask) {
 #pragma unroll
-                for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? v[e] : -INFINITY;
+                for (int e = 0; e < GV; ++e) v[e] = xc + e < P.V ? v[e] : -INFINITY;
             }
         } else {
 #pragma unroll
-            for (int e = 0; e < GV; ++e) v[e] = (on && x0 + e < P.V) ? E::load(row, x0 + e) : -INFINITY;
+            for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
         }
     };
     // The CTA that takes this one's place when it has finished is about `prefetch_ahead` blocks
@@ -150,8 +154,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
             float v[U][GV];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int x0 = x_lo + (s0 + u) * kStep + lane * GV;
-                load_group_if(x0, x0 < x_hi, v[u]);
+                load_group_clamped(x_lo + (s0 + u) * kStep + lane * GV, v[u]);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u)
@@ -178,10 +181,11 @@ sample_kernel(const __grid_constant__ SampleParams P)
     for (int st = 0; st < kMaxSteps; ++st) {
         const int x0 = x_lo + st * kStep + lane * GV;
         float v[GV];
-        load_group_if(x0, x0 < x_hi, v);   // weight 0 where there is no element
+        load_group_clamped(x0, v);
         float gs = 0.f;
 #pragma unroll
         for (int e = 0; e < GV; ++e) gs += ex2f(fmaf(v[e], P.scale, -ref0));
+        gs = x0 < x_hi ? gs : 0.f;   // a group past this warp's run (or the vocabulary) has no weight
         g[st] = gs;
         mass += gs;
     }
