@@ -27,8 +27,10 @@ struct SampleParams {
 // (Section 3.2).  With replacement the k draws are independent; without (Eq. 1) every
 // drawn token is taken out of the distribution before the next draw, which here means
 // subtracting its weight from the partial sums of its lane, its warp's run and the
-// element scan.  The row is read twice, for its maximum and for the weights, both times from
-// L2: the CTA that held this CTA's place before asked for the row while it computed;
+// element scan.  The row is read once, from L2: the CTA that held this CTA's place before asked
+// for the row while it computed.  There is no separate pass for the row's maximum: every
+// thread exponentiates its groups batch by batch against the batch's own integer reference and
+// moves the sums to the row's reference afterwards (an exact power of two);
 // temperature 0 takes the k largest logits instead (lowest index first on ties).
 // NT threads per CTA: 512 (two CTAs per SM, two independent chains) when the vocabulary fits
 // 16 steps per warp, else 1024.
@@ -143,52 +145,76 @@ sample_kernel(const __grid_constant__ SampleParams P)
         return;
     }
 
-    // ---- reference of the row: ceil(max * scale)
-    float mx = -INFINITY;
-    {
-        // four loads in flight per thread (more cost registers the two resident CTAs do not have)
-        constexpr int U = 4 < kMaxSteps ? 4 : kMaxSteps;
-#pragma unroll 1
-        for (int s0 = 0; s0 < kMaxSteps; s0 += U) {
-            if (x_lo + s0 * kStep >= x_hi) break;
-            float v[U][GV];
+    // ---- unnormalised weights in ONE pass over the row: per lane the sum of its group in every
+    // step, per warp its run.  A thread takes its groups in batches of U (that many 16-byte
+    // loads in flight; more cost registers the two resident CTAs do not have) and
+    // exponentiates each batch against the batch's own integer reference ceil(max * scale); once
+    // the row's reference is known every batch is moved to it by an exact power of two.
+    constexpr int U = 4 < kMaxSteps ? 4 : kMaxSteps;
+    constexpr int NB = kMaxSteps / U;
+    static_assert(kMaxSteps % U == 0, "whole batches");
+    float g[kMaxSteps];
+    float rb[NB];   // reference of each batch (-inf: nothing there)
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                load_group_clamped(x_lo + (s0 + u) * kStep + lane * GV, v[u]);
+    for (int bi = 0; bi < NB; ++bi) {
+        float v[U][GV];
+#pragma unroll
+        for (int u = 0; u < U; ++u) load_group_clamped(x_lo + (bi * U + u) * kStep + lane * GV, v[u]);
+        // (groups read in place of groups past the end are row elements too: they can only
+        // raise the batch's reference towards the row's, never beyond it)
+        float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int e = 0; e < GV; e += 4) {
+                m0 = max3(m0, v[u][e], v[u][e + 1]);
+                m1 = max3(m1, v[u][e + 2], v[u][e + 3]);
             }
+        rb[bi] = int_ref(fmaxf(m0, m1) * P.scale);
+        const float r0 = rb[bi] == -INFINITY ? 0.f : rb[bi];
 #pragma unroll
-            for (int u = 0; u < U; ++u)
+        for (int u = 0; u < U; ++u) {
+            const int x0 = x_lo + (bi * U + u) * kStep + lane * GV;
+            float gs = 0.f;
 #pragma unroll
-                for (int e = 0; e < GV; e += 2) mx = max3(mx, v[u][e], v[u][e + 1]);
+            for (int e = 0; e < GV; ++e) gs += ex2f(fmaf(v[u][e], P.scale, -r0));
+            g[bi * U + u] = x0 < x_hi ? gs : 0.f;   // a group past this warp's run (or the vocabulary) has no weight
         }
     }
-    mx = warp_max(mx);
-    if (lane == 0) s_red[warp] = mx;
-    __syncthreads();
-    const float ref = int_ref(warp_max(lane < kW ? s_red[lane] : -INFINITY) * P.scale);
-    const float ref0 = ref == -INFINITY ? 0.f : ref;
     prefetch_later_row();
-    auto weights = [&](int x0, float *w) {
-        float v[GV];
-        load_group(x0, v);
+    // reference of the row
+    float rmax = rb[0];
 #pragma unroll
-        for (int e = 0; e < GV; ++e) w[e] = ex2f(fmaf(v[e], P.scale, -ref0));
-    };
-    // ---- unnormalised weights: per lane the sum of its group in every step, per warp its run
-    float g[kMaxSteps];
+    for (int bi = 1; bi < NB; ++bi) rmax = fmaxf(rmax, rb[bi]);
+    rmax = warp_max(rmax);
+    if (lane == 0) s_red[warp] = rmax;
+    __syncthreads();
+    const float ref = warp_max(lane < kW ? s_red[lane] : -INFINITY);
+    float fb[NB];   // 2^(batch reference - row reference)
     float mass = 0.f;
 #pragma unroll
-    for (int st = 0; st < kMaxSteps; ++st) {
-        const int x0 = x_lo + st * kStep + lane * GV;
-        float v[GV];
-        load_group_clamped(x0, v);
-        float gs = 0.f;
+    for (int bi = 0; bi < NB; ++bi) {
+        fb[bi] = exp2i(rb[bi] - ref);
 #pragma unroll
-        for (int e = 0; e < GV; ++e) gs += ex2f(fmaf(v[e], P.scale, -ref0));
-        gs = x0 < x_hi ? gs : 0.f;   // a group past this warp's run (or the vocabulary) has no weight
-        g[st] = gs;
-        mass += gs;
+        for (int u = 0; u < U; ++u) {
+            g[bi * U + u] *= fb[bi];
+            mass += g[bi * U + u];
+        }
     }
+    // the weights of one group again, bit for bit as they went into g (st: the group's step)
+    auto weights = [&](int x0, int st, float *w) {
+        float v[GV];
+        load_group(x0, v);
+        float r = rb[0], f = fb[0];
+#pragma unroll
+        for (int bi = 1; bi < NB; ++bi) {
+            r = (st / U == bi) ? rb[bi] : r;
+            f = (st / U == bi) ? fb[bi] : f;
+        }
+        const float r0 = r == -INFINITY ? 0.f : r;
+#pragma unroll
+        for (int e = 0; e < GV; ++e) w[e] = ex2f(fmaf(v[e], P.scale, -r0)) * f;
+    };
     mass = warp_sum(mass);
     if (lane == 0) s_wtot[warp] = mass;
     __syncthreads();
@@ -235,7 +261,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
                     if (lane == l) {
                         const int x0 = x_lo + ps * kStep + lane * GV;
                         float w[GV];
-                        weights(x0, w);
+                        weights(x0, ps, w);
                         const float rem = t2 - (gi - gs);
                         float acc = 0.f;
 #pragma unroll
