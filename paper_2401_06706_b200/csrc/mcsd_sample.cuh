@@ -150,7 +150,8 @@ sample_kernel(const __grid_constant__ SampleParams P)
     // loads in flight; more cost registers the two resident CTAs do not have) and
     // exponentiates each batch against the batch's own integer reference ceil(max * scale); once
     // the row's reference is known every batch is moved to it by an exact power of two.
-    constexpr int U = 4 < kMaxSteps ? 4 : kMaxSteps;
+    constexpr int kBatch = E::kBytes == 4 ? 8 : 4;   // measured: 8 is 9 % faster than 4 with 4-byte logits, 5 % slower with 2-byte
+    constexpr int U = kBatch < kMaxSteps ? kBatch : kMaxSteps;
     constexpr int NB = kMaxSteps / U;
     static_assert(kMaxSteps % U == 0, "whole batches");
     float g[kMaxSteps];
