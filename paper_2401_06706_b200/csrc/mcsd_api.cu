@@ -618,28 +618,28 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
     std::memcpy(p.child_count, plan.child_count, sizeof(p.child_count));
     cudaStream_t stream = static_cast<cudaStream_t>(desc->stream);
     const unsigned grid = static_cast<unsigned>(n_ctas);
-    // 16 warps cover the row within the per-warp step budget (half of MCSD_MAX_VOCAB / 32 elements
-    // per warp at 1024 threads) when the vocabulary is at most half the maximum
+    // A vocabulary of at most half the maximum fits the per-warp step budget of smaller CTAs, of
+    // which several are resident per SM: 512 threads (two) with 4-byte logits, 256 (four) with 2-byte
     const bool small = desc->vocab <= MCSD_MAX_VOCAB / 2;
+    const int threads = !small ? 1024 : (desc->dtype == MCSD_DTYPE_F32 ? 512 : 256);
     {
-        // CTAs resident at once (two of 512 threads or one of 1024 per SM): how far ahead the
-        // kernel asks rows into L2
+        // CTAs resident at once: how far ahead in the grid the kernel asks rows into L2
         int dev = 0, n_sm = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MCSD_ERR_CUDA;
-        p.prefetch_ahead = n_sm * (small ? 2 : 1);
+        p.prefetch_ahead = n_sm * (1024 / threads);
     }
-    if (small) {
-        switch (desc->dtype) {
-        case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32, 512><<<grid, 512, 0, stream>>>(p); break;
-        case MCSD_DTYPE_BF16: sample_kernel<MCSD_DTYPE_BF16, 512><<<grid, 512, 0, stream>>>(p); break;
-        default: sample_kernel<MCSD_DTYPE_F16, 512><<<grid, 512, 0, stream>>>(p); break;
-        }
-    } else {
+    if (!small) {
         switch (desc->dtype) {
         case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32, 1024><<<grid, 1024, 0, stream>>>(p); break;
         case MCSD_DTYPE_BF16: sample_kernel<MCSD_DTYPE_BF16, 1024><<<grid, 1024, 0, stream>>>(p); break;
         default: sample_kernel<MCSD_DTYPE_F16, 1024><<<grid, 1024, 0, stream>>>(p); break;
+        }
+    } else {
+        switch (desc->dtype) {
+        case MCSD_DTYPE_F32: sample_kernel<MCSD_DTYPE_F32, 512><<<grid, 512, 0, stream>>>(p); break;
+        case MCSD_DTYPE_BF16: sample_kernel<MCSD_DTYPE_BF16, 256><<<grid, 256, 0, stream>>>(p); break;
+        default: sample_kernel<MCSD_DTYPE_F16, 256><<<grid, 256, 0, stream>>>(p); break;
         }
     }
     if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;

@@ -32,17 +32,20 @@ struct SampleParams {
 // thread exponentiates its groups batch by batch against the batch's own integer reference and
 // moves the sums to the row's reference afterwards (an exact power of two);
 // temperature 0 takes the k largest logits instead (lowest index first on ties).
-// NT threads per CTA: 512 (two CTAs per SM, two independent chains) when the vocabulary fits
-// 16 steps per warp, else 1024.
+// NT threads per CTA: 1024 when the vocabulary exceeds half the maximum, else as many independent
+// chains per SM as 16 steps per warp allow: 512 (two CTAs per SM) with 4-byte logits, 256 (four
+// CTAs per SM) with 2-byte logits.
 template <int DT, int NT>
-__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
+__global__ void __launch_bounds__(NT, NT == 512 ? 2 : (NT == 256 ? 4 : 1))
 sample_kernel(const __grid_constant__ SampleParams P)
 {
     using E = Elem<DT>;
     constexpr int GV = E::kVec;
     constexpr int kStep = 32 * GV;
     constexpr int kW = NT / 32;  // warps
-    constexpr int kMaxSteps = MCSD_MAX_VOCAB / 32 / kStep;  // steps of a warp's run (the host picks NT so that they suffice)
+    // steps of a warp's run: CTAs of 1024 threads cover the largest vocabulary, smaller ones half of it
+    constexpr int kMaxSteps = (NT == 1024 ? MCSD_MAX_VOCAB : MCSD_MAX_VOCAB / 2) / kW / kStep;
+    static_assert(kMaxSteps <= 16, "the per-lane group sums are kept in registers");
     __shared__ float s_wtot[32];
     __shared__ float s_red[32];
     __shared__ int s_redi[32];
