@@ -107,42 +107,80 @@ sample_kernel(const __grid_constant__ SampleParams P)
 
     if (P.scale == 0.f) {
         prefetch_later_row();
-        // ---- top-k: k block-wide maxima, each over the elements that come after the previous
-        // pick in the order (logit descending, index ascending)
-        float pv = INFINITY;
-        int pi = -1;
-        for (int i = 0; i < k; ++i) {
-            float best = -INFINITY;
-            int best_i = 0x7fffffff;
-            for (int x0 = x_lo + lane * GV; x0 < x_hi; x0 += kStep) {
-                float v[GV];
-                load_group(x0, v);
+        // ---- top-k.  One pass leaves in every thread the best of its own elements (largest
+        // logit, lowest index among equals).  Each pick is the block-wide best of those; then only
+        // the thread that held it needs a new best, which its warp finds together (lane j takes
+        // the thread's j-th group) among the elements after the pick in the order (logit
+        // descending, index ascending).
+        float best = -INFINITY;
+        int best_i = 0x7fffffff;
+        {
+            constexpr int UT = 4 < kMaxSteps ? 4 : kMaxSteps;
+#pragma unroll 1
+            for (int s0 = 0; s0 < kMaxSteps; s0 += UT) {
+                if (x_lo + s0 * kStep >= x_hi) break;
+                float v[UT][GV];
 #pragma unroll
-                for (int e = 0; e < GV; ++e) {
-                    const int x = x0 + e;
-                    const bool after = i == 0 || v[e] < pv || (v[e] == pv && x > pi);
-                    if (x < P.V && after && v[e] > best) { best = v[e]; best_i = x; }  // ascending x: ties keep the lowest
+                for (int u = 0; u < UT; ++u) load_group_clamped(x_lo + (s0 + u) * kStep + lane * GV, v[u]);
+#pragma unroll
+                for (int u = 0; u < UT; ++u) {
+                    const int x0 = x_lo + (s0 + u) * kStep + lane * GV;
+                    if (x0 < x_hi) {   // (a group read in place of one past the run is not this thread's)
+#pragma unroll
+                        for (int e = 0; e < GV; ++e)
+                            if (v[u][e] > best) { best = v[u][e]; best_i = x0 + e; }   // ascending index: ties keep the lowest
+                    }
                 }
             }
+        }
+        auto better = [](float av, int ai, float bv, int bi) { return av > bv || (av == bv && ai < bi); };
+        for (int i = 0; i < k; ++i) {
+            float wv = best;
+            int wi = best_i;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
-                if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+                const float ov = __shfl_xor_sync(0xffffffffu, wv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, wi, o);
+                if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
             }
-            if (lane == 0) { s_red[warp] = best; s_redi[warp] = best_i; }
+            if (lane == 0) { s_red[warp] = wv; s_redi[warp] = wi; }
             __syncthreads();
-            best = lane < kW ? s_red[lane] : -INFINITY;
-            best_i = lane < kW ? s_redi[lane] : 0x7fffffff;
+            wv = lane < kW ? s_red[lane] : -INFINITY;
+            wi = lane < kW ? s_redi[lane] : 0x7fffffff;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
-                if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+                const float ov = __shfl_xor_sync(0xffffffffu, wv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, wi, o);
+                if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
             }
-            pv = best;
-            pi = best_i == 0x7fffffff ? -1 : best_i;
+            const float pv = wv;
+            const int pi = wi == 0x7fffffff ? -1 : wi;
             if (tid == 0) out[i] = pi;
+            // the holder of the pick (one thread of one warp) gets its next best
+            const unsigned own = __ballot_sync(0xffffffffu, pi >= 0 && best_i == pi);
+            if (own && i + 1 < k) {
+                const int src = __ffs(own) - 1;
+                float nv = -INFINITY;
+                int ni = 0x7fffffff;
+                const int x0 = x_lo + lane * kStep + src * GV;   // lane = step of the holder's run
+                if (lane < kMaxSteps && x0 < x_hi) {
+                    float v[GV];
+                    load_group(x0, v);
+#pragma unroll
+                    for (int e = 0; e < GV; ++e) {
+                        const int x = x0 + e;
+                        const bool after = v[e] < pv || (v[e] == pv && x > pi);
+                        if (x < P.V && after && v[e] > nv) { nv = v[e]; ni = x; }
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ov = __shfl_xor_sync(0xffffffffu, nv, o);
+                    const int oi = __shfl_xor_sync(0xffffffffu, ni, o);
+                    if (better(ov, oi, nv, ni)) { nv = ov; ni = oi; }
+                }
+                if (lane == src) { best = nv; best_i = ni; }
+            }
             __syncthreads();
         }
         return;

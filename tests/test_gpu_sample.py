@@ -107,6 +107,30 @@ def test_top_k_at_temperature_zero_with_ties():
         assert torch.equal(mine, theirs)
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("vocab", [32000, 40000])
+def test_top_k_when_one_thread_holds_many_of_the_largest(dtype, vocab):
+    """The k largest logits sit, with ties, at indices a single thread of the kernel reads (the
+    same 16-byte group position in every step of one warp's run), so that thread has to renew
+    its best after every pick; others are spread out.  Exact indices against the oracle."""
+    w = synth.Workload("sample_t0_one_thread", 3, vocab, "32", dtype, "normal", 1.0, 1.0, 0.5, 0.0, 0, 11)
+    inp, u = _inputs(w, 13)
+    per_group = 16 // inp.draft.element_size()
+    draft = inp.draft.clone()
+    step = 32 * per_group
+    for b in range(3):
+        hot = [s * step + e for s in range(6) for e in range(per_group)][:24]      # one lane's groups
+        vals = torch.tensor([20.0 + (i // 3) for i in range(len(hot))], dtype=draft.dtype)   # runs of three equal values
+        draft[b, 0, torch.tensor(hot) + 1000 * b * 0] = vals.to(draft.device)
+        draft[b, 0, vocab - 1 - b] = 19.5
+    cand = binding.mcsd_sample_candidates(draft, inp.parent, None, 0.0, 0)
+    torch.cuda.synchronize()
+    d = draft.to(torch.float32).cpu().numpy()
+    c = cand.cpu().numpy()
+    for b in range(3):
+        assert (c[b, 1:33] == oracle.topk(d[b, 0], 32)).all(), b
+
+
 def test_node_range_touches_only_its_children_and_levels_compose():
     w = synth.Workload("sample_levels", 5, 4096, "3x2x2", "bf16", "normal", 2.5, 1.0, 1.0, 1.0, 1, 9)
     inp, u = _inputs(w, 21)
