@@ -628,6 +628,8 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MCSD_ERR_CUDA;
         p.prefetch_ahead = n_sm * (1024 / threads);
+        // (MCSD_SAMPLE_AHEAD: percent of that distance, for tuning)
+        p.prefetch_ahead = static_cast<int>(static_cast<long long>(p.prefetch_ahead) * env_int("MCSD_SAMPLE_AHEAD", 100) / 100);
     }
     if (!small) {
         switch (desc->dtype) {
