@@ -183,13 +183,15 @@ int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const voi
 
 /*
  * The same result computed the way Section 3 describes the procedure: only the nodes a
- * walk actually visits are evaluated.  Level by level (one kernel launch per level of the
- * tree, gamma + 1 in all), every sequence evaluates the node its walk stands on
- * (softmax of that node's two rows, Algorithm 1 / 2 on its candidates) and moves to the
- * accepted child; then the walk stage runs as in mcsd_verify.  At most 2 * gamma + 1 logit
- * rows per tree are read instead of all of them, at the price of gamma + 1 dependent
- * launches, so this is the form to use when the tree is large or latency matters more
- * than the node rate.  Outputs are identical to those of mcsd_verify (the same tests with
+ * walk actually visits are evaluated.  Every sequence starts at the root, evaluates the
+ * node its walk stands on (softmax of that node's two rows, Algorithm 1 / 2 on its
+ * candidates) and moves to the accepted child until a test sequence rejects all
+ * candidates or a leaf is reached; then the walk stage runs as in mcsd_verify.  At
+ * temperature > 0 one kernel launch does this for the whole batch (each sequence is
+ * walked by one thread-block cluster); at temperature 0 there is one launch per level
+ * of the tree.  At most 2 * gamma + 1 logit rows per tree are read instead of all of
+ * them, so this is the form to use when the tree is large or latency matters more than
+ * the node rate.  Outputs are identical to those of mcsd_verify (the same tests with
  * the same uniforms).  The optional per-node outputs of the descriptor are filled for
  * visited nodes only and node_bonus is not produced.  Arguments as in mcsd_verify.
  */

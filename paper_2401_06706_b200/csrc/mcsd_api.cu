@@ -280,8 +280,10 @@ int check_common(const mcsd_desc *d, const void *target, const void *draft, cons
 }
 
 // level < 0: the all-node form (every node of every tree is an item).  level >= 0: path
-// mode, the items are the sequences and each works on the node its walk stands on at
-// that level (path arrays in the workspace, swapped level by level).
+// mode, the items are the sequences.  At temperature > 0 ONE launch (level 0) walks every
+// sequence from the root to the node where its walk stops; at temperature 0 there is one
+// launch per level and each sequence works on the node its walk stands on at that level
+// (path arrays in the workspace, swapped level by level).
 int launch_nodes(const Call &c, const void *target, const void *draft, const int32_t *cand,
                  const float *unif, float T, int mode, int level = -1)
 {
@@ -345,7 +347,6 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     p.n_items = static_cast<int32_t>(n_items);
     p.step_b = static_cast<int32_t>(path ? n_clusters : n_clusters / d->n_nodes);
     p.step_n = static_cast<int32_t>(path ? 0 : n_clusters % d->n_nodes);
-    p.path_cur = path_cur; p.path_next = path_next;
     p.mode = mode;
     const double scale_d = 1.4426950408889634 / static_cast<double>(T);
     p.scale = static_cast<float>(scale_d);
@@ -577,9 +578,11 @@ int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const voi
                                 out_residual);
         replacement_mode = MCSD_MODE_WITH_REPLACEMENT;
     }
-    // one launch per level of the tree: level l evaluates, for every sequence, the node its
+    // temperature > 0: one launch, every cluster walks its sequences from the root.  Temperature
+    // 0: one launch per level of the tree; level l evaluates, for every sequence, the node its
     // walk stands on after l accepted tokens (nothing for walks that have ended)
-    for (int level = 0; level <= c.plan.gamma; ++level) {
+    const int n_levels = temperature > 0.f ? 1 : c.plan.gamma + 1;
+    for (int level = 0; level < n_levels; ++level) {
         rc = launch_nodes(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, replacement_mode, level);
         if (rc != MCSD_OK) return rc;
     }

@@ -41,11 +41,9 @@ struct NodeParams {
     int32_t slice;   // vocabulary elements owned by one CTA of the cluster
     int32_t n_items; // B * n_nodes
     int32_t step_b, step_n;  // quotient and remainder of (clusters in the grid) / n_nodes
-    // Path mode (one launch per tree level): the items are the sequences, item b works on node
-    // path_cur[b] (negative: that walk has ended, nothing to do) and leaves in path_next[b] the
-    // accepted child, or -1.  Null for the all-node form.  Then step_b = clusters, step_n = 0.
-    const int32_t *path_cur;
-    int32_t *path_next;
+    // Path mode: the items are the sequences (step_b = clusters in the grid, step_n = 0); a cluster
+    // follows each of its sequences from the root through the accepted children and evaluates
+    // only the nodes on that walk.
     int32_t mode;
     float scale;     // log2(e) / T rounded to float ...
     float scale_lo;  // ... and what the rounding dropped (for the candidates' own probabilities)

@@ -26,6 +26,7 @@ struct Action {
     float4 stats;  // (row reference of p, of q, 1 / Z_t, Z_t / Z_d); written in the statistics round only
     float c_try;   // c of the residual sum to form next
     int more;      // 1: form that sum and run another round; 0: the node is decided
+    int accepted;  // path mode, with more == 0: the accepted child of the node, or -1
 };
 
 // Candidate data of the next items, fetched ahead of use by warp 0 so that no DRAM
@@ -55,7 +56,8 @@ constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
 
 // DT: element type; EPT: vocabulary elements per thread per row; DIRECT: read the
 // rows with plain scalar loads (any alignment) instead of vector loads and bulk copies;
-// PATH: the items are the sequences, each at the node its walk stands on (see NodeParams).
+// PATH: the items are the sequences; a cluster walks each of its sequences from the root,
+// evaluating only the nodes the walk visits (see NodeParams).
 //
 // Ownership inside a CTA: the slice is cut into 16-byte groups of GV elements; thread
 // (warp w, lane l) owns groups (w * NG + j) * 32 + l, j < NG, so that one warp-wide
@@ -79,7 +81,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     // SMs and the prefetch takes DRAM latency off the per-node chain (measured +20 %); with
     // 4-byte logits it is bound by HBM and the extra request stream only costs (-1 %, and
     // -30 % on leaf-only trees), so it is left out there
-    constexpr bool kPrefetch = !DIRECT && E::kBytes == 2;
+    constexpr bool kPrefetch = !DIRECT && !PATH && E::kBytes == 2;
     static_assert(EPT % GV == 0, "EPT must be a whole number of 16-byte groups");
     static_assert(NW == 4, "the exchange buffers hold four warps per CTA");
     // warp 0 leads the exchange rounds and takes the decisions; the look-ahead requests for the
@@ -172,13 +174,12 @@ node_kernel(const __grid_constant__ NodeParams P)
         b += P.step_b;
         n += P.step_n;
         if (n >= P.n_nodes) { n -= P.n_nodes; ++b; }
-        if (PATH) n = b < P.B ? __ldg(P.path_cur + b) : 0;
     };
 
     // ---- candidate pipeline (the fetch warp only) -------------------------------------------
     auto fetch_tokens = [&](int b, int n, int slot3) {
         if (b < P.B) {
-            const int k = ((!PATH || n >= 0) && n < P.n_internal) ? P.child_count[n] : 0;
+            const int k = n < P.n_internal ? P.child_count[n] : 0;
             if (lane < k) {
                 const long long ci = static_cast<long long>(b) * P.n_nodes + P.child_first[n] + lane;
                 cp_async4(&ring.tok[slot3][lane], P.cand + ci);
@@ -189,7 +190,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     // needs the item's tokens to have arrived (cp_async_wait_all by this thread)
     auto fetch_logits = [&](int b, int n, int slot3, int slot2) {
         if (b < P.B) {
-            const int k = ((!PATH || n >= 0) && n < P.n_internal) ? P.child_count[n] : 0;
+            const int k = n < P.n_internal ? P.child_count[n] : 0;
             if (lane < k) {
                 const int xt = ring.tok[slot3][lane];
                 if (xt >= 0 && xt < P.V) {
@@ -210,12 +211,12 @@ node_kernel(const __grid_constant__ NodeParams P)
     };
 
     int b = cluster_id / P.n_nodes, n = cluster_id - b * P.n_nodes;  // current item
-    if (PATH) { b = cluster_id; n = b < P.B ? __ldg(P.path_cur + b) : 0; }
+    if (PATH) { b = cluster_id; n = 0; }  // every walk starts at the root
     int b1 = b, n1 = n;                                              // the next one
     advance(b1, n1);
     uint32_t it = 0;  // iteration count of this cluster
     bool prev_internal = false;
-    if (warp == kFetchWarp) {
+    if (!PATH && warp == kFetchWarp) {
         fetch_tokens(b, n, 0);
         cp_async_wait_all();
         __syncwarp();
@@ -228,7 +229,7 @@ node_kernel(const __grid_constant__ NodeParams P)
     }
 
     for (; b < P.B; ++it) {
-        const bool internal = (!PATH || n >= 0) && n < P.n_internal;
+        const bool internal = n < P.n_internal;
         const int k = internal ? P.child_count[n] : 0;
         const int first = P.child_first[n];
         const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
@@ -236,7 +237,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         int status_bits = 0;
 
         // this item's candidate data has landed (it was requested one item ago) ...
-        if (warp == kFetchWarp) cp_async_wait_all();
+        if (!PATH && warp == kFetchWarp) cp_async_wait_all();
         // ... and, around an item with children, all warps meet: they are done with the
         // previous item (its draft buffer and ring entries may be overwritten) and they
         // see this item's ring entries.  A run of leaves needs no meeting at all.
@@ -245,6 +246,10 @@ node_kernel(const __grid_constant__ NodeParams P)
             __syncthreads();
         }
         prev_internal = internal;
+        // path mode: the next node is only known once this one is decided, so nothing is fetched
+        // ahead; the leader warp asks for this node's candidate data now and picks it up when it
+        // needs it, behind the row work and the exchange
+        if (PATH && warp == 0 && internal) fetch_tokens(b, n, s3);
 
         const unsigned char *t_row = t_slice(node_idx);
         const unsigned char *d_row = d_slice(b, n);
@@ -257,7 +262,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         // look-ahead duties of the fetch warp: L2 prefetch of the next item's slices, candidate
         // data of the next two items
         auto look_ahead = [&]() {
-            if (warp == kFetchWarp) {
+            if (!PATH && warp == kFetchWarp) {
                 if (kPrefetch && lane == 0 && b1 < P.B && bulk_bytes) {
                     bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
                     if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
@@ -272,13 +277,6 @@ node_kernel(const __grid_constant__ NodeParams P)
             b = b1; n = n1;
             advance(b1, n1);
         };
-
-        if (PATH && n < 0) {  // this walk ended at an earlier level
-            if (crank == 0 && tid == 0) P.path_next[b] = -1;
-            look_ahead();
-            next_item();
-            continue;
-        }
 
         // ---- target slice -> registers, as packed pairs
         f32x2 tv[EPT / 2];
@@ -364,12 +362,14 @@ node_kernel(const __grid_constant__ NodeParams P)
             if (lane == 0)
                 P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * 32 +
                             crank * NW + warp] = make_float2(rt, st);
-            if (crank == 0 && tid == 0) {
-                P.node_accept[node_idx] = -1;
-                if (PATH) P.path_next[b] = -1;
+            if (crank == 0 && tid == 0) P.node_accept[node_idx] = -1;
+            if (PATH) {  // the walk ends at this leaf: on to the cluster's next sequence
+                b += P.step_b;
+                n = 0;
+            } else {
+                look_ahead();
+                next_item();
             }
-            look_ahead();
-            next_item();
             continue;
         }
 
@@ -523,6 +523,13 @@ node_kernel(const __grid_constant__ NodeParams P)
         };
 
         if (warp == 0) {
+            if (PATH) {  // tokens and uniforms have landed by now; then the candidates' own logits
+                cp_async_wait_all();
+                __syncwarp();
+                fetch_logits(b, n, s3, s2);
+                cp_async_wait_all();
+                __syncwarp();
+            }
             // while the round is in flight: 2^(scaled logit) of the candidates' own logits as
             // 2^int * frac (lane i = candidate i)
             float frac_t = 0.f, frac_d = 0.f;
@@ -559,6 +566,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                 act[round & 1u].stats = make_float4(R_t, R_d, t_ok ? 1.f / Z_t : 0.f, (t_ok && d_ok) ? Z_t / Z_d : 0.f);
                 act[round & 1u].c_try = static_cast<float>(c_try);
                 act[round & 1u].more = more;
+                if (PATH) act[round & 1u].accepted = accepted;
                 if (crank == 0) *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
             }
         }
@@ -613,6 +621,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                 if (lane == 0) {
                     act[round & 1u].c_try = static_cast<float>(c_try);
                     act[round & 1u].more = next;
+                    if (PATH) act[round & 1u].accepted = accepted;
                 }
             }
             exchange_release();
@@ -625,7 +634,6 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (warp == 0) {
             if (crank == 0 && lane == 0) {
                 P.node_accept[node_idx] = accepted;
-                if (PATH) P.path_next[b] = accepted;
                 reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
                     make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
             }
@@ -633,7 +641,14 @@ node_kernel(const __grid_constant__ NodeParams P)
         if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
         status_bits = __reduce_or_sync(0xffffffffu, status_bits);
         if (status_bits && lane == 0) atomicOr(P.status + b, status_bits);
-        next_item();
+        if (PATH) {
+            // the walk goes on at the accepted child, or ends here
+            const int acc = act[(round - 1u) & 1u].accepted;
+            if (acc >= 0) n = acc;
+            else { b += P.step_b; n = 0; }
+        } else {
+            next_item();
+        }
     }
 
     if (warp == kFetchWarp) cp_async_wait_all();

@@ -66,8 +66,13 @@ def test_low_acceptance_stops_early_and_launch_count():
     w = synth.Workload("path_low", 64, 32000, "2x2x2x1", "fp32", "normal", 2.5, 1.0, 3.0, 1.0, 1, 99)
     inp, v, out = _run(w, "mcsd_verify_path")
     _check(inp, out)
-    assert binding.mcsd_last_launch_count() == inp.stats["gamma"] + 1 + 1   # one per level, then the walk
+    assert binding.mcsd_last_launch_count() == 2   # one kernel walks every sequence, then the walk kernel
     assert float(out.accept_len.float().mean()) < 1.0
+    # temperature 0: one argmax launch per level, then the walk
+    w0 = synth.Workload("path_low_t0", 64, 32000, "2x2x2x1", "fp32", "normal", 2.5, 1.0, 3.0, 0.0, 0, 99)
+    inp0, _, out0 = _run(w0, "mcsd_verify_path")
+    _check(inp0, out0)
+    assert binding.mcsd_last_launch_count() == inp0.stats["gamma"] + 1 + 1
 
 
 def test_empty_batch_and_root_only():
