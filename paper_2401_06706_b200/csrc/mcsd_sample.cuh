@@ -96,7 +96,8 @@ sample_kernel(const __grid_constant__ SampleParams P)
                 const int b2 = static_cast<int>(nb / P.n_range), n2 = P.node_begin + static_cast<int>(nb - static_cast<long long>(b2) * P.n_range);
                 const unsigned char *r2 = reinterpret_cast<const unsigned char *>(P.draft) +
                     (static_cast<long long>(b2) * P.n_internal + n2) * P.ld_d * E::kBytes;
-                bulk_prefetch_l2(r2, (static_cast<uint32_t>(P.V) * E::kBytes) & ~15u);
+                const uint32_t bytes = (static_cast<uint32_t>(P.V) * E::kBytes) & ~15u;
+                if (bytes) bulk_prefetch_l2(r2, bytes);
             }
         }
     };
