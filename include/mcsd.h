@@ -119,6 +119,14 @@ typedef struct mcsd_desc {
                              -1.  With the flattened-tree layout of Section 3.3 (node n
                              at sequence position prefix_len + n) these are the key/value
                              cache rows that stay after verification.                */
+    float *node_residual; /* [B][n_nodes][V] float32 (device), NULL to skip: for every node
+                             that can end a walk (as for node_bonus) the distribution its
+                             endpoint token is drawn from, i.e. the residual p left by
+                             Algorithm 1 / 2 after all k rejections, the target distribution
+                             at a leaf, one-hot at temperature 0; rows of other nodes are
+                             not written.  A debugging output: B * n_nodes * V * 4 bytes
+                             and a pass over every such node; not produced by
+                             mcsd_verify_path.                                        */
 } mcsd_desc;
 
 /*

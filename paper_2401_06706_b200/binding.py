@@ -35,7 +35,7 @@ class McsdDesc(ctypes.Structure):
                 ("workspace_bytes", ctypes.c_size_t),
                 ("node_accept", ctypes.c_void_p), ("node_bonus", ctypes.c_void_p),
                 ("node_ratio", ctypes.c_void_p), ("out_status", ctypes.c_void_p),
-                ("out_path_nodes", ctypes.c_void_p)]
+                ("out_path_nodes", ctypes.c_void_p), ("node_residual", ctypes.c_void_p)]
 
 
 class McsdError(RuntimeError):
@@ -149,6 +149,7 @@ class VerifyOutput:
     node_bonus: Optional[torch.Tensor] = None
     node_ratio: Optional[torch.Tensor] = None
     path_nodes: Optional[torch.Tensor] = None  # [B, gamma+1] tree nodes of the accepted tokens, -1 padded
+    node_residual: Optional[torch.Tensor] = None  # [B, n_nodes, V] float32; rows of nodes that cannot end a walk are NaN
 
 
 class Verifier:
@@ -157,7 +158,7 @@ class Verifier:
 
     def __init__(self, batch: int, parent, vocab: int, dtype: torch.dtype, device="cuda", *,
                  want_residual: bool = True, node_outputs: bool = False, ld_target: Optional[int] = None,
-                 ld_draft: Optional[int] = None):
+                 ld_draft: Optional[int] = None, node_residual: bool = False):
         self.lib = load_library()
         self.parent = np.ascontiguousarray(parent, dtype=np.int32)
         self.device = torch.device(device)
@@ -198,6 +199,11 @@ class Verifier:
             d.node_accept = self.node_accept.data_ptr()
             d.node_bonus = self.node_bonus.data_ptr()
             d.node_ratio = self.node_ratio.data_ptr()
+        self.node_residual = None
+        if node_residual:   # a debugging output: B * n_nodes * V floats
+            self.node_residual = torch.full((self.batch, self.n_nodes, self.vocab), float("nan"), dtype=torch.float32,
+                                            device=self.device)
+            d.node_residual = self.node_residual.data_ptr()
 
     def _bind(self, target, draft):
         assert target.dtype == self.dtype and target.shape == (self.batch, self.n_nodes, self.vocab)
@@ -209,7 +215,7 @@ class Verifier:
 
     def _out(self) -> VerifyOutput:
         return VerifyOutput(self.accept_len, self.tokens, self.residual, self.status, self.node_accept,
-                            self.node_bonus, self.node_ratio, self.path_nodes)
+                            self.node_bonus, self.node_ratio, self.path_nodes, self.node_residual)
 
     def mcsd_verify(self, target, draft, cand, unif, temperature: float, mode: int) -> VerifyOutput:
         self._bind(target, draft)

@@ -416,6 +416,7 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
     p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part; p.status = c.status;
     p.out_accept_len = out_accept_len; p.out_tokens = out_tokens; p.out_residual = out_residual;
     p.out_path_nodes = d->out_path_nodes;
+    p.node_residual = d->node_residual;
     p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
     p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab; p.gamma = c.plan.gamma;
     p.scale = T > 0.f ? static_cast<float>(1.4426950408889634 / static_cast<double>(T)) : 0.f;
@@ -431,8 +432,10 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
         if (rc != MCSD_OK) return rc;
         p.n_entries = cfg.cluster * kNodeWarps;
     }
-    // all-nodes pass first (only when per-node endpoint tokens were asked for), then the walks
-    for (int all = (T > 0.f && d->node_bonus && all_nodes_allowed) ? 1 : 0; all >= 0; --all) {
+    // all-nodes pass first (only when per-node endpoint tokens or distributions were asked for;
+    // at temperature 0 the tokens are there already), then the walks
+    const bool want_all = all_nodes_allowed && ((T > 0.f && d->node_bonus) || d->node_residual);
+    for (int all = want_all ? 1 : 0; all >= 0; --all) {
         p.all_nodes = all;
         const unsigned grid = static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch);
         if (d->vocab <= MCSD_MAX_VOCAB / 2) {
@@ -756,6 +759,7 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
     mcsd_desc cd = *desc;
     cd.batch = chunk;
     cd.node_accept = nullptr; cd.node_bonus = nullptr; cd.node_ratio = nullptr; cd.out_path_nodes = nullptr;
+    cd.node_residual = nullptr;
     const size_t ws_bytes = mcsd_workspace_bytes(&cd);
     bool ok = true;
     auto chk = [&](cudaError_t e) { if (e != cudaSuccess) ok = false; return e == cudaSuccess; };

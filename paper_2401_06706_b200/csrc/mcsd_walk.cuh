@@ -18,6 +18,7 @@ struct WalkParams {
     int32_t *out_accept_len;
     int32_t *out_tokens;
     float *out_residual;  // may be null
+    float *node_residual; // [B][n_nodes][V], may be null: where the all-nodes pass leaves each node's distribution
     int32_t *out_path_nodes;  // may be null
     int32_t *status;      // [B]
     long long ld_t, ld_d;
@@ -96,7 +97,8 @@ walk_kernel(const __grid_constant__ WalkParams P)
         if (tid == 0) P.node_bonus[nb + n] = -1;  // a walk never stops here
         return;
     }
-    float *out = P.out_residual ? P.out_residual + static_cast<long long>(b) * P.V : nullptr;
+    float *out = P.all_nodes ? (P.node_residual ? P.node_residual + (nb + n) * P.V : nullptr)
+                             : (P.out_residual ? P.out_residual + static_cast<long long>(b) * P.V : nullptr);
 
     if (P.scale == 0.f) {
         // argmax rule: the endpoint is the target argmax of the stopping node, the

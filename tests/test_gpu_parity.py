@@ -271,3 +271,44 @@ def test_largest_configuration_sampled_parity_and_properties():
     end = torch.from_numpy(tok[np.arange(w.batch), ln]).to(res.device).long()
     assert bool((res.gather(1, end[:, None]) > 0).all())       # the endpoint token has positive mass
     assert 0.5 < ln.mean() < 4.5
+
+
+@pytest.mark.parametrize("dtype,T,mode", [("fp32", 1.0, 0), ("fp32", 0.7, 1), ("bf16", 1.0, 1), ("fp16", 0.0, 0)])
+def test_per_node_residual_output(dtype, T, mode):
+    """node_residual: for every node that can end a walk, the distribution its endpoint token is
+    drawn from (Algorithm 1 / 2 residual after k rejections, target distribution at a leaf,
+    one-hot at temperature 0), against the oracle node by node; other rows stay untouched."""
+    import oracle
+    w = synth.Workload("node_res", 3, 3000, "3x2x1", dtype, "normal", 2.5, 1.0, 1.5, T, mode, 808)
+    inp = synth.make_inputs(w, "cuda")
+    v = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[dtype], "cuda", node_outputs=True,
+                         node_residual=True)
+    out = v.mcsd_verify(inp.target, inp.draft if T > 0 else None, inp.cand, inp.unif, T, mode)
+    torch.cuda.synchronize()
+    assert_parity(inp, out)
+    t, d, c, u = inp.host_f32()
+    acc = to_np(out.node_accept)
+    res = to_np(out.node_residual)
+    first, count = synth.children_ranges(inp.parent)
+    tol = 1e-5 if dtype == "fp32" else 2e-3
+    seen_stop = seen_skip = 0
+    for b in range(w.batch):
+        for n in range(inp.stats["n_nodes"]):
+            if acc[b, n] >= 0:
+                assert np.isnan(res[b, n]).all()      # a walk never stops here: row not written
+                seen_skip += 1
+                continue
+            seen_stop += 1
+            if T == 0:
+                want = np.zeros(w.vocab)
+                want[oracle.argmax(t[b, n])] = 1.0
+            else:
+                want = oracle.softmax(t[b, n], T)
+                k = int(count[n])
+                if k:
+                    ch = np.arange(first[n], first[n] + k)
+                    r = oracle.mcss(want, oracle.softmax(d[b, n], T), c[b, ch], u[b, ch, 0].astype(np.float64), mode)
+                    assert r.accepted == -1
+                    want = r.p
+            assert np.abs(res[b, n] - want).max() <= tol, (b, n)
+    assert seen_stop > 0 and seen_skip > 0
