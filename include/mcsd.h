@@ -48,7 +48,8 @@
 extern "C" {
 #endif
 
-#define MCSD_VERSION 100
+/* 101: mcsd_desc gained node_residual at its end (a caller built against 100 must be rebuilt) */
+#define MCSD_VERSION 101
 
 /* logit element types (both logit tensors share one) */
 #define MCSD_DTYPE_F32 0

@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(lib):
     assert set(names) == set(binding.EXPORTS)
     for name in names:
         assert getattr(lib, name) is not None
-    assert lib.mcsd_version() == 100
+    assert lib.mcsd_version() == 101
 
 
 def test_header_constants_match_binding():
