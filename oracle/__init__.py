@@ -240,3 +240,20 @@ def path_nodes(result: "VerifyResult", gamma: int) -> np.ndarray:
             out[b, i] = n
             i += 1
     return out
+
+
+def gather_accepted_kv(cache, prefix_len, path_nodes, accept_len) -> np.ndarray:
+    """What stays of the target model's key/value cache after verification (Sections 3 and 3.3).
+    The tree was fed as one flattened sequence, node n at position prefix_len[b] + n, so the cache
+    holds one row per tree node; the i-th accepted token (node path_nodes[b][i], depth i + 1) belongs
+    at position prefix_len[b] + 1 + i of the committed sequence.  cache: [S][B][L][R] (S independent
+    slabs: layers, keys and values, heads).  Returns a copy with those rows moved there; every other
+    row is as it was."""
+    cache = np.asarray(cache)
+    out = cache.copy()
+    S, B = cache.shape[0], cache.shape[1]
+    for s in range(S):
+        for b in range(B):
+            for i in range(int(accept_len[b])):
+                out[s, b, int(prefix_len[b]) + 1 + i] = cache[s, b, int(prefix_len[b]) + int(path_nodes[b][i])]
+    return out
