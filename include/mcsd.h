@@ -296,6 +296,29 @@ int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const v
 int mcsd_tree_attention_layout(const int32_t *tree_parent, int32_t n_nodes, int32_t prefix_len,
                                uint8_t *mask, int32_t *position_ids, void *stream);
 
+/*
+ * After verification (Sections 3 and 3.3): the target model ran over the flattened tree, so
+ * its key/value cache holds one row per tree node, node n of sequence b at position
+ * prefix_len[b] + n.  Only the rows of the accepted path stay.  This call moves, in place,
+ * the row of the i-th accepted token's node (path_nodes[b][i], as mcsd_verify writes them to
+ * desc->out_path_nodes) to position prefix_len[b] + 1 + i, for i < accept_len[b]; no other
+ * row is written (rows behind the committed part keep stale tree rows).
+ *   cache       device; row (slab s, sequence b, position t) starts at byte
+ *               s * slab_stride + b * seq_stride + t * pos_stride and has row_bytes bytes.
+ *               A slab is whatever shares this layout: a layer's keys, its values, one head.
+ *               Rows are moved in the widest unit (16, 8, 4, 2 or 1 bytes) that divides the
+ *               base address, the three strides and row_bytes.
+ *   prefix_len  device [batch] int32: position of the root (the last committed token)
+ *   path_nodes  device [batch][gamma + 1], accept_len device [batch]: outputs of mcsd_verify
+ *   n_positions positions per sequence the cache holds
+ * Entries of path_nodes below i + 1 (impossible for a walk) or at a position beyond the cache
+ * are skipped; prefix_len must not be negative.
+ */
+int mcsd_gather_accepted_kv(void *cache, int64_t n_slabs, int64_t slab_stride, int32_t batch,
+                            int64_t seq_stride, int64_t pos_stride, int64_t row_bytes,
+                            int64_t n_positions, const int32_t *prefix_len, const int32_t *path_nodes,
+                            const int32_t *accept_len, int32_t gamma, void *stream);
+
 /* Bytes of device workspace mcsd_verify needs for this descriptor (batch and
  * n_nodes are read); 0 if the descriptor is NULL or its shape is invalid. */
 size_t mcsd_workspace_bytes(const mcsd_desc *desc);

@@ -23,6 +23,7 @@ STATUS_DEGENERATE, STATUS_BAD_TOKEN, STATUS_NO_MASS, STATUS_TIMEOUT = 1, 2, 4, 8
 MAX_NODES, MAX_CHILDREN, MAX_VOCAB = 512, 32, 65536
 
 EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path", "mcsd_sample_candidates", "mcsd_tree_attention_layout",
+           "mcsd_gather_accepted_kv",
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
            "mcsd_version")
 
@@ -67,6 +68,9 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_sample_candidates.restype = ctypes.c_int
     lib.mcsd_tree_attention_layout.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.mcsd_tree_attention_layout.restype = ctypes.c_int
+    i64 = ctypes.c_int64
+    lib.mcsd_gather_accepted_kv.argtypes = [vp, i64, i64, i32, i64, i64, i64, i64, vp, vp, vp, i32, vp]
+    lib.mcsd_gather_accepted_kv.restype = ctypes.c_int
     lib.mcsd_verify_static.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int, vp, vp, vp]
     lib.mcsd_verify_static.restype = ctypes.c_int
     lib.mcsd_verify_nodes.argtypes = [dp, vp, vp, vp, vp, vp, f32, ctypes.c_int]
@@ -281,6 +285,27 @@ def mcsd_tree_attention_layout(parent, prefix_len: int, device="cuda"):
     _check(lib.mcsd_tree_attention_layout(parent.ctypes.data, n, int(prefix_len), _ptr(mask), _ptr(pos),
                                           torch.cuda.current_stream(torch.device(device)).cuda_stream))
     return mask, pos
+
+
+def mcsd_gather_accepted_kv(cache: torch.Tensor, prefix_len: torch.Tensor, path_nodes: torch.Tensor,
+                            accept_len: torch.Tensor) -> torch.Tensor:
+    """Moves, in place, the cache rows of the accepted path to their committed positions (see mcsd.h).
+    cache: device tensor [slabs, batch, positions, ...] whose trailing dimensions form one contiguous row;
+    prefix_len, accept_len: int32 [batch]; path_nodes: int32 [batch, gamma + 1].  Returns cache."""
+    lib = load_library()
+    assert cache.dim() >= 4 and cache.is_cuda
+    S, B, L = cache.shape[:3]
+    row = cache[0, 0, 0]
+    assert row.is_contiguous(), "the trailing dimensions must form one contiguous row"
+    es = cache.element_size()
+    assert path_nodes.dtype == torch.int32 and path_nodes.is_contiguous() and path_nodes.shape[0] == B
+    assert prefix_len.dtype == torch.int32 and accept_len.dtype == torch.int32
+    gamma = int(path_nodes.shape[1]) - 1
+    _check(lib.mcsd_gather_accepted_kv(cache.data_ptr(), S, cache.stride(0) * es, B, cache.stride(1) * es,
+                                       cache.stride(2) * es, row.numel() * es, L, _ptr(prefix_len),
+                                       _ptr(path_nodes), _ptr(accept_len), gamma,
+                                       torch.cuda.current_stream(cache.device).cuda_stream))
+    return cache
 
 
 def mcsd_sample_candidates(draft, parent, unif_draw, temperature: float, mode: int, *, node_begin: int = 0,

@@ -672,6 +672,49 @@ int mcsd_tree_attention_layout(const int32_t *tree_parent, int32_t n_nodes, int3
     return MCSD_OK;
 }
 
+int mcsd_gather_accepted_kv(void *cache, int64_t n_slabs, int64_t slab_stride, int32_t batch,
+                            int64_t seq_stride, int64_t pos_stride, int64_t row_bytes,
+                            int64_t n_positions, const int32_t *prefix_len, const int32_t *path_nodes,
+                            const int32_t *accept_len, int32_t gamma, void *stream)
+{
+    if (n_slabs < 0 || batch < 0 || row_bytes < 0 || gamma < 0 || slab_stride < 0 || seq_stride < 0 || n_positions < 0)
+        return MCSD_ERR_SHAPE;
+    if (pos_stride < row_bytes) return MCSD_ERR_STRIDE;
+    g_last_launches = 0;
+    const long long n_items = static_cast<long long>(n_slabs) * batch;
+    if (n_items == 0 || row_bytes == 0 || gamma == 0) return MCSD_OK;
+    if (!cache || !prefix_len || !path_nodes || !accept_len) return MCSD_ERR_NULL;
+    // widest unit that divides the base address, the strides and the row length
+    const unsigned long long all = reinterpret_cast<uintptr_t>(cache) | static_cast<unsigned long long>(slab_stride) |
+        static_cast<unsigned long long>(seq_stride) | static_cast<unsigned long long>(pos_stride) |
+        static_cast<unsigned long long>(row_bytes);
+    int unit = 16;
+    while (unit > 1 && (all & static_cast<unsigned long long>(unit - 1))) unit >>= 1;
+    if (row_bytes / unit > 0x7fffffffLL) return MCSD_ERR_UNSUPPORTED;
+    GatherParams p = {};
+    p.cache = static_cast<unsigned char *>(cache);
+    p.slab_stride = slab_stride; p.seq_stride = seq_stride; p.pos_stride = pos_stride;
+    p.n_items = n_items; p.n_positions = n_positions; p.batch = batch; p.gamma = gamma;
+    p.row_units = static_cast<int32_t>(row_bytes / unit);
+    p.prefix_len = prefix_len; p.path_nodes = path_nodes; p.accept_len = accept_len;
+    int dev = 0, n_sm = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    const long long cap = static_cast<long long>(n_sm) * 8;
+    const unsigned grid = static_cast<unsigned>(n_items < cap ? n_items : cap);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (unit) {
+    case 16: gather_kernel<uint4><<<grid, kThreads, 0, st>>>(p); break;
+    case 8: gather_kernel<uint2><<<grid, kThreads, 0, st>>>(p); break;
+    case 4: gather_kernel<uint32_t><<<grid, kThreads, 0, st>>>(p); break;
+    case 2: gather_kernel<uint16_t><<<grid, kThreads, 0, st>>>(p); break;
+    default: gather_kernel<uint8_t><<<grid, kThreads, 0, st>>>(p); break;
+    }
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches = 1;
+    return MCSD_OK;
+}
+
 // ---- mcsd_verify_static: the scratch memory is an array built into the library --------
 // In host code the name below is only a handle for the runtime; the address kernels can
 // use comes from cudaGetSymbolAddress, looked up once per device.

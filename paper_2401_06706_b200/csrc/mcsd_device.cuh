@@ -21,6 +21,8 @@
 //   naive_kernel     (mcsd_naive.cuh)  The sample-and-match baseline of Section 4.3.
 //   layout_kernel    (mcsd_layout.cuh)  Mask and position ids of the tree attention
 //                    (Section 3.3).
+//   gather_kernel    (mcsd_gather.cuh)  Key/value cache rows of the accepted path to their
+//                    committed positions.
 // mcsd_common.cuh holds what they share.
 //
 // How the rejection loop avoids rewriting the residual.  After n rejections the
@@ -46,3 +48,4 @@
 #include "mcsd_sample.cuh"
 #include "mcsd_naive.cuh"
 #include "mcsd_layout.cuh"
+#include "mcsd_gather.cuh"
