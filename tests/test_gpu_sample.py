@@ -41,7 +41,7 @@ def _check(inp, u, cand, T, mode, node_begin=0, node_end=None):
 @pytest.mark.parametrize("dtype", ["fp32", "bf16", "fp16"])
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("vocab,kconfig", [(7, "3x2"), (1000, "4x2"), (8200, "8x1"), (32000, "4x2x2x1"),
-                                           (32001, "2x2"), (50272, "2x2x2x2"), (65536, "32")])
+                                           (32001, "2x2"), (50272, "2x2x2x2"), (65536, "32"), (32000, "32"), (20000, "16x2")])
 def test_draws_match_the_oracle(vocab, kconfig, mode, dtype):
     if mode == 1 and vocab < 16:
         kconfig = "3x2"
