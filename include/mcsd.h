@@ -152,6 +152,9 @@ typedef struct mcsd_desc {
  *                  was drawn from (final residual p of the stopping node, its
  *                  target distribution for a leaf, one-hot at temperature 0);
  *                  NULL to skip
+ * The call allocates nothing and does not synchronise: it enqueues its kernels on
+ * desc->stream and returns.  After one ordinary call on a device (which looks up launch
+ * attributes once per kernel) it can be captured in a CUDA graph and replayed.
  * Rows whose base address and stride are multiples of 16 bytes take the bulk-copy
  * (TMA) path; any other layout is accepted and takes a slower plain-load path.
  * All ld elements of every row, the last one included, must be readable memory: on
