@@ -125,3 +125,10 @@ def test_host_validation_codes(lib):
 def test_binding_fails_loudly_without_library(tmp_path):
     with pytest.raises(RuntimeError, match="missing"):
         binding.load_library(str(tmp_path / "libmcsd.so"))
+
+
+def test_the_build_entry_point_runs():
+    """build() of the repository's entry file compiles the CUDA library and the oracle and checks
+    the library against the header; it needs nvcc and gcc but no GPU."""
+    import __graft_entry__
+    __graft_entry__.build()
