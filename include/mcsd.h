@@ -154,7 +154,8 @@ typedef struct mcsd_desc {
  *                  NULL to skip
  * The call allocates nothing and does not synchronise: it enqueues its kernels on
  * desc->stream and returns.  After one ordinary call on a device (which looks up launch
- * attributes once per kernel) it can be captured in a CUDA graph and replayed.
+ * attributes once per kernel) it can be captured in a CUDA graph and replayed (tested for
+ * mcsd_verify and mcsd_verify_path).
  * Rows whose base address and stride are multiples of 16 bytes take the bulk-copy
  * (TMA) path; any other layout is accepted and takes a slower plain-load path.
  * All ld elements of every row, the last one included, must be readable memory: on
@@ -264,7 +265,8 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
  * MCSD_STATIC_WORKSPACE_BYTES bytes compiled into the library; every GPU that
  * loads the library carries that array until the process exits.  Inputs and
  * outputs are still the caller's buffers; desc->workspace and
- * desc->workspace_bytes are ignored.  Everything else is as in mcsd_verify.
+ * desc->workspace_bytes are ignored.  Arguments, outputs and return codes are those of
+ * mcsd_verify.
  *
  * Limits and rules
  *   - If mcsd_workspace_bytes(desc) exceeds MCSD_STATIC_WORKSPACE_BYTES the call
