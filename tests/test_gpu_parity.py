@@ -312,3 +312,44 @@ def test_per_node_residual_output(dtype, T, mode):
                     want = r.p
             assert np.abs(res[b, n] - want).max() <= tol, (b, n)
     assert seen_stop > 0 and seen_skip > 0
+
+
+@pytest.mark.skipif(os.environ.get("MCSD_SKIP_LARGE") == "1", reason="large case disabled")
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_largest_configuration_path_form_and_sampler(dtype):
+    """The same full-size inputs through the other entry points, in the launch shapes the bench
+    times: the path form must reproduce the all-node form bit for bit on all 512 sequences (and the
+    oracle on sampled ones); the sampler is compared with the oracle on sampled sequences and must
+    draw valid, and without replacement distinct, tokens everywhere."""
+    from dataclasses import replace
+    from oracle import compare as cmp
+    w = replace(NAMED["cfg5_largest"], dtype=dtype, mode=1)
+    inp = synth.make_inputs(w, "cuda")
+    v = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[dtype], "cuda")
+    a = v.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+    torch.cuda.synchronize()
+    a_len, a_tok, a_res, a_st = (x.clone() for x in (a.accept_len, a.tokens, a.residual, a.status))
+    b = v.mcsd_verify_path(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+    torch.cuda.synchronize()
+    assert torch.equal(a_len, b.accept_len) and torch.equal(a_tok, b.tokens) and torch.equal(a_st, b.status)
+    assert torch.equal(a_res, b.residual)
+    for b0 in (0, 300, 506):
+        assert_parity(inp, b, b0, b0 + 6)
+    # sampler
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(99)
+    u = synth.open_uniforms((w.batch, inp.stats["n_nodes"]), gen, "cuda")
+    cand = binding.mcsd_sample_candidates(inp.draft, inp.parent, u, 1.0, 1)
+    torch.cuda.synchronize()
+    c = cand.cpu().numpy()
+    assert (c[:, 0] == -1).all() and (c[:, 1:] >= 0).all() and (c[:, 1:] < w.vocab).all()
+    first, count = synth.children_ranges(inp.parent)
+    for n in range(inp.stats["n_internal"]):
+        ch = np.sort(c[:, first[n]:first[n] + count[n]], axis=1)
+        assert (np.diff(ch, axis=1) > 0).all()          # Eq. 1: the children of a node carry distinct tokens
+    for b0 in (0, 400, 508):
+        sl = slice(b0, b0 + 4)
+        rep = cmp.compare_samples(inp.draft[sl].to(torch.float32).cpu().numpy(), inp.parent, u[sl].cpu().numpy(), 1.0, 1,
+                                  c[sl], 0, None)
+        assert rep.ok, rep.failures[:5]
+        assert rep.n_tolerated <= max(3, 1e-6 * w.vocab * rep.n_draws)
