@@ -514,19 +514,30 @@ def run_stage(args):
     ms_avg = sum(ms) / len(ms)
     peak, peak_kind = measured_peaks()
     achieved = algo / (ms_avg * 1e-3) / 1e9
-    # parity of this stage on the first sequences, against the oracle
-    n_seq = min(w.batch, 8)
-    if args.stage == "sample":
-        from oracle import compare as cmp
-        rep = cmp.compare_samples(inp.draft[:n_seq].to(torch.float32).cpu().numpy(), inp.parent, u[:n_seq].cpu().numpy(),
-                                  w.temperature, w.mode, cand[:n_seq].cpu().numpy(), 0, None)
-        parity = {"sequences": n_seq, "draws": rep.n_draws, "tolerated": rep.n_tolerated, "ok": bool(rep.ok)}
-    else:
+    # CPU baseline leg: the oracle of this stage, as it stands, timed on a bounded sample of the same
+    # inputs; what it computed also serves to check the kernel's output on those sequences
+    cpu_baseline, parity = None, None
+    if not args.no_cpu_baseline:
         import oracle
-        t, _, c, uu = inp.host_f32(0, n_seq)
-        ref = oracle.verify(t, None, inp.parent, c, uu, 0.0, w.mode, want_residual=False)
-        got = ver.node_accept[:n_seq].cpu().numpy()
-        parity = {"sequences": n_seq, "nodes": int(got.size), "ok": bool((got == ref.node_accept).all())}
+        n_seq = min(w.batch, args.oracle_seqs if args.stage == "greedy" else max(8, args.oracle_seqs // 8))
+        if args.stage == "sample":
+            from oracle import compare as cmp
+            d_h, u_h = inp.draft[:n_seq].to(torch.float32).cpu().numpy(), u[:n_seq].cpu().numpy()
+            t0 = time.time()
+            oracle.sample(d_h, inp.parent, u_h, w.temperature, w.mode)
+            t1 = time.time()
+            rep = cmp.compare_samples(d_h, inp.parent, u_h, w.temperature, w.mode, cand[:n_seq].cpu().numpy(), 0, None)
+            parity = {"sequences": n_seq, "draws": rep.n_draws, "tolerated": rep.n_tolerated, "ok": bool(rep.ok)}
+        else:
+            t, _, c, uu = inp.host_f32(0, n_seq)
+            t0 = time.time()
+            ref = oracle.verify(t, None, inp.parent, c, uu, 0.0, w.mode, want_residual=False)
+            t1 = time.time()
+            got = ver.node_accept[:n_seq].cpu().numpy()
+            parity = {"sequences": n_seq, "nodes": int(got.size), "ok": bool((got == ref.node_accept).all())}
+        cpu_baseline = {"value": n_seq * st["n_draft"] / max(t1 - t0, 1e-9), "unit": unit, "cores": oracle.num_threads(),
+                        "kind": "oracle", "sample": f"first {n_seq} of {w.batch} sequences of the same inputs, "
+                                                      f"{t1 - t0:.2f} s wall"}
     line = {"metric": metric, "value": units / (ms_avg * 1e-3), "unit": unit, "n_gpus": 1, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_avg, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "stage": args.stage,
@@ -534,7 +545,8 @@ def run_stage(args):
             "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}",
                          "unit": "GB/s", "frac": achieved / peak, "algorithmic_bytes_per_launch": algo,
                          "kernel_ms_avg": ms_avg, "kernel_ms_min": min(ms), "traffic": None},
-            "gpu_launches": args.steps, "clocks": clocks, "parity_on_oracle_sample": parity}
+            "cpu_baseline": cpu_baseline, "gpu_launches": args.steps, "clocks": clocks,
+            "parity_on_oracle_sample": parity}
     print(json.dumps(line), flush=True)
 
 
