@@ -443,8 +443,13 @@ def run_sweep(args):
             times.append(e0.elapsed_time(e1))
         med, best = statistics.median(times), min(times)
         n_par = min(w.batch, args.sweep_parity_seqs)
+        # cpu_baseline leg of the point: the oracle on its first sequences, timed; its output is
+        # what the kernels' output is compared with
         t, d, c, u = inp.host_f32(0, n_par)
-        rep = compare.compare(t, d, inp.parent, c, u, w.temperature, w.mode, w.dtype,
+        t_cpu0 = time.time()
+        ref = oracle.verify(t, d, inp.parent, c, u, w.temperature, w.mode)
+        t_cpu = time.time() - t_cpu0
+        rep = compare.compare(t, d, inp.parent, c, u, w.temperature, w.mode, w.dtype, oracle_result=ref,
                               accept_len=ver.accept_len[:n_par].cpu().numpy(), tokens=ver.tokens[:n_par].cpu().numpy(),
                               residual=ver.residual[:n_par].cpu().numpy(), status=ver.status[:n_par].cpu().numpy())
         algo = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
@@ -454,7 +459,9 @@ def run_sweep(args):
                "frac_of_peak": algo / (med * 1e-3) / 1e9 / peak, "peak_kind": peak_kind,
                "regime": "hbm" if algo > 4 * 126e6 else "latency/L2-bound point (inputs < 4x L2)",
                "accept_len_mean": float(ver.accept_len.float().mean().item()), "parity_ok": rep.ok,
-               "parity": rep.summary()}
+               "parity": rep.summary(),
+               "cpu_baseline": {"value": n_par * st["n_draft"] / max(t_cpu, 1e-9), "unit": UNIT, "cores": oracle.num_threads(),
+                                "kind": "oracle", "sample": f"first {n_par} sequences, {t_cpu:.3f} s wall"}}
         if out:
             out.write(json.dumps(rec) + "\n")
             out.flush()
