@@ -34,7 +34,14 @@
  *   - the candidates of a node are its children, tested in ascending node index;
  *   - every test owns a pre-drawn uniform, indexed by the child node it tests;
  *   - if the residual mass is exactly 0 the residual is left unchanged and a
- *     status bit is set.
+ *     status bit is set;
+ *   - a draft row from which no distribution can be formed (its softmax is NaN)
+ *     rejects every candidate of its node, leaves p as it is and sets the same
+ *     status bit;
+ *   - "r ~ U(0,1)" is an input of the verification step; a supplied r that is
+ *     not below 1 (NaN included) counts as 1 there, so that every value a caller can pass has a defined
+ *     outcome: such an r accepts exactly when p(x~) >= q(x~).  (An r <= 0 needs no
+ *     rule: the ratio is never negative, so it accepts whenever q(x~) > 0.)
  *
  * All sums run left to right in double.  Inputs are float32 arrays holding the
  * exact (dtype-rounded) logits; every element is widened to double first.
@@ -333,6 +340,21 @@ static int32_t verify_node(int32_t n, int32_t n_nodes, int32_t n_internal, int32
     for (int32_t i = 0; i < k; ++i) {
         cands[i] = cand_b[first + i];
         r[i] = (double)unif_b[2 * (first + i)];
+        if (!(r[i] < 1.0)) r[i] = 1.0; /* supplied in place of r ~ U(0,1): not below 1 counts as 1 */
+    }
+    if (qbuf[0] != qbuf[0]) {
+        /* No draft distribution can be formed from this row (all -inf, or a NaN or +inf logit:
+         * the normaliser is not a positive number and every entry is NaN).  There is no q to
+         * test against: every candidate is rejected without a ratio, p stays as it is, and
+         * the failed residual update is reported as a zero-mass one. */
+        for (int32_t i = 0; i < k; ++i) {
+            if (cands[i] < 0 || cands[i] >= V) *status |= ORACLE_STATUS_BAD_TOKEN;
+            if (ratio_b) ratio_b[first + i] = -1.0;
+        }
+        *status |= ORACLE_STATUS_DEGENERATE;
+        *bonus = mcsd_oracle_invcdf(residual, V, (double)unif_b[2 * n + 1]);
+        if (*bonus < 0) *status |= ORACLE_STATUS_NO_MASS;
+        return -1;
     }
     int32_t acc = mcsd_oracle_mcss(residual, qbuf, V, cands, r, k, mode, ratio, S, status);
     if (ratio_b)

@@ -104,7 +104,10 @@ node_kernel(const __grid_constant__ NodeParams P)
     const int n_entries = static_cast<int>(csize) * NW;  // values per exchange round (<= 32)
     const float scale = P.scale;
     const uint32_t full_addr = smem_u32(&full_bar);
-    const uint32_t xbar_addr[2] = {smem_u32(&xch.bar[0]), smem_u32(&xch.bar[1])};
+    // barrier of exchange buffer s (computed, not looked up: an array indexed at run time would
+    // live in local memory)
+    const uint32_t xbar_base = smem_u32(&xch.bar[0]);
+    auto xbar_addr = [&](uint32_t s) -> uint32_t { return xbar_base + s * 8u; };
 
     // this CTA's slice of the vocabulary and this warp's run of it
     const int v_begin = static_cast<int>(crank) * P.slice;
@@ -125,8 +128,8 @@ node_kernel(const __grid_constant__ NodeParams P)
 
     if (tid == 0) {
         mbar_init(full_addr, 1);
-        mbar_init(xbar_addr[0], 1);
-        mbar_init(xbar_addr[1], 1);
+        mbar_init(xbar_addr(0), 1);
+        mbar_init(xbar_addr(1), 1);
         fence_mbar_init();
     }
     __syncthreads();
@@ -149,17 +152,17 @@ node_kernel(const __grid_constant__ NodeParams P)
     // lanes beyond the entry count.
     auto exchange_send = [&](float4 mine) {
         const uint32_t s = round & 1u;
-        if (tid == 0) mbar_arrive_expect_tx(xbar_addr[s], static_cast<uint32_t>(n_entries) * 16u);
+        if (tid == 0) mbar_arrive_expect_tx(xbar_addr(s), static_cast<uint32_t>(n_entries) * 16u);
         if (lane < static_cast<int>(csize)) {
             const uint32_t dst = map_to_rank(smem_u32(&xch.slot[s][crank * NW + warp]), lane);
-            st_async_f4(dst, mine, map_to_rank(xbar_addr[s], lane));
+            st_async_f4(dst, mine, map_to_rank(xbar_addr(s), lane));
         }
     };
     // leader (warp 0) only: waits for the round and returns entry `lane`
     auto exchange_leader_wait = [&](float4 identity) -> float4 {
         const uint32_t s = round & 1u;
         // once a wait has expired the results are void and later rounds do not wait again
-        if (!poisoned && !mbar_wait(xbar_addr[s], (round >> 1) & 1u)) poisoned = 1;
+        if (!poisoned && !mbar_wait(xbar_addr(s), (round >> 1) & 1u)) poisoned = 1;
         return lane < n_entries ? xch.slot[s][lane] : identity;
     };
     // all warps: ends the round (the other warps have been waiting here for the leader)

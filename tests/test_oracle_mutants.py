@@ -10,6 +10,7 @@ import oracle
 import test_oracle_pins as pins
 import test_oracle_sample_pins as spins
 import test_oracle_mcns_pins as npins
+import test_oracle_edge_pins as epins
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "mcsd_oracle.c")
 
@@ -74,6 +75,24 @@ MUTANTS = [
      [npins.test_walk_over_levels_and_leaf_endpoint]),
     ("sample_children_of_wrong_node", "const float *d = draft + ((size_t)b * n_internal + n) * V;", "const float *d = draft + ((size_t)b * n_internal) * V;",
      [lambda: spins.test_tree_level_routine_is_the_node_routine_in_child_order(1, 0.7)]),
+    ("zero_mass_residual_overwritten", "} else {\n            *status |= ORACLE_STATUS_DEGENERATE;",
+     "} else {\n            for (int32_t x = 0; x < V; ++x) p[x] = 0.0;\n            *status |= ORACLE_STATUS_DEGENERATE;",
+     [lambda: epins.test_zero_residual_mass_keeps_p_and_later_candidates_see_it(0)]),
+    ("zero_mass_not_reported", "} else {\n            *status |= ORACLE_STATUS_DEGENERATE;\n        }", "}",
+     [lambda: epins.test_zero_residual_mass_after_a_candidate_of_probability_zero(1)]),
+    ("zero_mass_divided_anyway", "if (s > 0.0) {", "if (s >= 0.0) {",
+     [lambda: epins.test_all_candidates_rejected_on_zero_mass_draws_from_the_kept_p(0)]),
+    ("no_mass_not_reported", "if (*bonus < 0) *status |= ORACLE_STATUS_NO_MASS;", ";",
+     [lambda: epins.test_target_row_without_mass_at_the_root("nan", 0), epins.test_leaf_without_mass_ends_the_walk_with_no_token]),
+    ("no_mass_returns_a_token", "    return last;\n}", "    return last < 0 ? 0 : last;\n}",
+     [lambda: epins.test_target_row_without_mass_at_the_root("all_minus_inf", 1)]),
+    ("naive_no_mass_not_reported", "if (x < 0) { *status |= ORACLE_STATUS_NO_MASS; *bonus = -1; return -1; }",
+     "if (x < 0) { *bonus = -1; return -1; }",
+     [lambda: epins.test_target_row_without_mass_at_the_root("plus_inf", 2)]),
+    ("uniform_cap_missing", "if (!(r[i] < 1.0)) r[i] = 1.0;", ";",
+     [epins.test_uniform_not_below_one_counts_as_one]),
+    ("draft_without_mass_falls_through", "if (qbuf[0] != qbuf[0]) {", "if (0) {",
+     [lambda: epins.test_draft_row_without_mass_rejects_everything_and_draws_from_p(1)]),
 ]
 
 
