@@ -26,10 +26,14 @@
  *   - Randomness is supplied by the caller: uniforms[b][n][0] is the r of the
  *     acceptance test of node n as a candidate of its parent, uniforms[b][n][1]
  *     is the uniform used to draw the endpoint token if the walk stops at n.
- *     Uniforms are expected in the open interval (0, 1).
+ *     Uniforms are expected in the open interval (0, 1).  Other values have a
+ *     defined outcome: an acceptance uniform that is not below 1 (NaN included)
+ *     counts as 1, i.e. it accepts exactly when p(x) >= q(x); one that is <= 0
+ *     accepts whenever q(x) > 0; an endpoint uniform >= 1 or NaN draws the last
+ *     token of positive probability, one <= 0 the first.
  *   - Endpoint draw: inverse CDF in token order, the smallest x with
  *     sum_{y<=x} P(y) > u * sum_y P(y); tokens of probability 0 are never drawn.
- *   - Temperature 0 selects the argmax rule (Section 4.4): a candidate is
+ *   - Temperature 0 selects the argmax rule (Section 4.5): a candidate is
  *     accepted iff it equals the target argmax (lowest index on ties) and the
  *     endpoint token is the target argmax of the node where the walk stops;
  *     draft logits are not read.
@@ -37,6 +41,17 @@
  *     nothing has been enqueued.  Faults that only the device can see (token out
  *     of range, zero mass, expired bounded wait) set MCSD_STATUS_* bits in
  *     out_status[b]; kernels never trap and every wait in them is bounded.
+ *     out_status[b] describes the walk of sequence b: it is the OR of what was
+ *     met at the nodes the walk visited (the nodes the sequential procedure of
+ *     Section 3 evaluates), the node where it stopped included; a fault at a node
+ *     the walk never reached does not show.  The words are written, not
+ *     accumulated: they need no clearing by the caller.
+ *   - Logits: -inf is legal (probability 0).  A row from which no distribution
+ *     can be formed (all -inf, a NaN or a +inf logit) is handled as follows: a
+ *     target row without mass accepts nothing, a walk that stops there returns
+ *     token -1 (MCSD_STATUS_NO_MASS | MCSD_STATUS_DEGENERATE); a draft row without
+ *     mass rejects every candidate of its node and the endpoint is drawn from the
+ *     untouched target distribution (MCSD_STATUS_DEGENERATE).
  */
 #ifndef MCSD_H_
 #define MCSD_H_
@@ -48,8 +63,10 @@
 extern "C" {
 #endif
 
-/* 101: mcsd_desc gained node_residual at its end (a caller built against 100 must be rebuilt) */
-#define MCSD_VERSION 101
+/* 101: mcsd_desc gained node_residual at its end (a caller built against 100 must be rebuilt)
+ * 102: out_status describes the walk only and is written, not accumulated; mcsd_set_option,
+ *      mcsd_get_option, mcsd_release_host_staging; desc->reserved is checked */
+#define MCSD_VERSION 102
 
 /* logit element types (both logit tensors share one) */
 #define MCSD_DTYPE_F32 0
@@ -59,7 +76,7 @@ extern "C" {
 /* replacement_mode */
 #define MCSD_MODE_WITH_REPLACEMENT 0    /* Algorithm 1 */
 #define MCSD_MODE_WITHOUT_REPLACEMENT 1 /* Algorithm 2 */
-#define MCSD_MODE_NAIVE 2 /* multi-candidate naive sampling, the ablation baseline of Section 4.4:
+#define MCSD_MODE_NAIVE 2 /* multi-candidate naive sampling, the ablation baseline of Section 4.5:
                              draw x from the target distribution (second uniform of the node);
                              accept the first child that carries x, else x is the endpoint token.
                              mcsd_verify, mcsd_verify_path and mcsd_verify_host only; draft_logits
@@ -94,13 +111,29 @@ extern "C" {
 #define MCSD_STATUS_NO_MASS 4    /* endpoint draw from a distribution of mass 0 / NaN    */
 #define MCSD_STATUS_TIMEOUT 8    /* a bounded on-chip wait expired; results invalid      */
 
+/* Options of mcsd_set_option: process-wide tuning and test overrides, 0 = library default.
+ * The first four also take their initial value from the environment variable of the same
+ * name (MCSD_CLUSTER, MCSD_EPT, MCSD_DIRECT, MCSD_SAMPLE_AHEAD, MCSD_PDL), read once when
+ * the library is loaded. */
+#define MCSD_OPT_CLUSTER 0       /* CTAs per thread-block cluster of the node kernel (1..8)          */
+#define MCSD_OPT_EPT 1           /* vocabulary elements per thread and row of the node kernel         */
+#define MCSD_OPT_DIRECT 2        /* 1: plain element loads even where rows are 16-byte aligned        */
+#define MCSD_OPT_SAMPLE_AHEAD 3  /* L2 look-ahead of the sampling kernel, percent of its default (100) */
+#define MCSD_OPT_WAIT_POLLS 4    /* poll budget of the node kernel's exchange wait (0: about 2 s)     */
+#define MCSD_OPT_TEST_EXTRA_TX 5 /* test of the expiry path only: the exchange barrier of every round
+                                    expects this many bytes (a multiple of 16) that nobody sends, so
+                                    the bounded wait runs out and MCSD_STATUS_TIMEOUT is reported      */
+#define MCSD_OPT_PDL 6           /* 1 (default): the walk stage is launched as a programmatic dependent
+                                    of the node stage; 0: plain stream order                         */
+#define MCSD_OPT_COUNT 7
+
 typedef struct mcsd_desc {
     int32_t batch;      /* B: number of trees                                         */
     int32_t n_nodes;    /* N+1: nodes per tree, root included                         */
     int32_t n_internal; /* nodes that have children (= rows of draft_logits per tree) */
     int32_t vocab;      /* V                                                          */
     int32_t dtype;      /* MCSD_DTYPE_*                                               */
-    int32_t reserved;   /* must be 0                                                  */
+    int32_t reserved;   /* must be 0 (MCSD_ERR_SHAPE otherwise)                       */
     int64_t ld_target;  /* elements between consecutive rows of target_logits, >= V   */
     int64_t ld_draft;   /* same for draft_logits                                      */
     void *stream;       /* cudaStream_t the work is enqueued on (0 = default stream)  */
@@ -114,7 +147,8 @@ typedef struct mcsd_desc {
                              asking for it adds a pass over every such node       */
     float *node_ratio;    /* [B][n_nodes] p/q seen by the test of each draft node; -1
                              for a forced rejection; untouched if never tested      */
-    int32_t *out_status;  /* [B] MCSD_STATUS_* bits (device), NULL to skip            */
+    int32_t *out_status;  /* [B] MCSD_STATUS_* bits of each walk (device), NULL to skip;
+                             written by every call, no clearing needed              */
     int32_t *out_path_nodes; /* [B][gamma+1] (device), NULL to skip: entry i < accept_len
                              is the tree node whose token is out_tokens[i], the rest is
                              -1.  With the flattened-tree layout of Section 3.3 (node n
@@ -172,7 +206,8 @@ int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *dr
  * the rejection loop of Algorithm 1 / 2 at every node that has children).  Fills
  * node_accept (in the workspace when the descriptor leaves it NULL) and the
  * per-node statistics kept in the workspace; at temperature 0 also node_bonus
- * (the target argmax of every node).  Arguments as in mcsd_verify.
+ * (the target argmax of every node that accepted nothing, else -1).  out_status is
+ * written by stage 2.  Arguments as in mcsd_verify.
  */
 int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                       const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
@@ -242,10 +277,14 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
  * is a host pointer.  The library allocates device buffers for a slice of the
  * batch, copies the slice in, verifies it and copies the results back, slice
  * after slice on two internal streams so that copies overlap the kernels; it
- * frees everything and synchronises before it returns.  Only batch, n_nodes,
- * n_internal, vocab, dtype, ld_target and ld_draft of the descriptor are read;
- * node_* outputs are not produced.  out_status (host, [B]) may be NULL.
- * Host buffers in page-locked memory make the copies asynchronous.
+ * synchronises before it returns.  The device staging buffers (two slices' worth:
+ * about 2 x 256 MiB plus outputs) and the two streams are kept for the next call on
+ * the same device and grown on demand; mcsd_release_host_staging frees them.  Calls
+ * on one device are serialised.  Only batch, n_nodes, n_internal, vocab, dtype,
+ * ld_target and ld_draft of the descriptor are read; node_* outputs are not produced.
+ * out_status (host, [B]) may be NULL.  Host buffers in page-locked memory make the
+ * copies asynchronous.  If a CUDA call fails part way (MCSD_ERR_CUDA) the outputs of
+ * the slices not yet finished are undefined.
  */
 int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
@@ -324,8 +363,20 @@ int mcsd_gather_accepted_kv(void *cache, int64_t n_slabs, int64_t slab_stride, i
                             int64_t n_positions, const int32_t *prefix_len, const int32_t *path_nodes,
                             const int32_t *accept_len, int32_t gamma, void *stream);
 
-/* Bytes of device workspace mcsd_verify needs for this descriptor (batch and
- * n_nodes are read); 0 if the descriptor is NULL or its shape is invalid. */
+/* Frees the device staging buffers and streams mcsd_verify_host keeps on the current
+ * device (allocating again on its next call).  Returns MCSD_OK or MCSD_ERR_CUDA. */
+int mcsd_release_host_staging(void);
+
+/* Sets one of the MCSD_OPT_* overrides for the whole process (not synchronised with calls
+ * running on other host threads).  value >= 0; 0 restores the default.  Returns MCSD_OK, or
+ * MCSD_ERR_SHAPE for an unknown option or a negative value.  mcsd_get_option returns the
+ * current value (or MCSD_ERR_SHAPE). */
+int mcsd_set_option(int option, int value);
+int mcsd_get_option(int option);
+
+/* Bytes of device workspace mcsd_verify needs for this descriptor (batch, n_nodes and
+ * n_internal are read: the need depends on the node counts only, not on the shape of the
+ * tree); 0 if the descriptor is NULL or its shape is invalid. */
 size_t mcsd_workspace_bytes(const mcsd_desc *desc);
 
 /* Depth (gamma) of a tree given as a host parent array, or a negative MCSD_ERR_*

@@ -16,7 +16,13 @@ Rules
   * Endpoint tokens are draws by inverse CDF; a different token is tolerated only
     if it has positive oracle probability and u lies within NEAR_TIE (in CDF
     units) of that token's oracle CDF interval.  Such cases are counted.
-  * Residual distributions agree within `residual_tol` max abs error.
+  * Residual distributions agree within `residual_tol` max abs error (not compared where the
+    oracle reports NO_MASS: there is no distribution then, its entries are NaN).
+  * Status words describe the walk: they are compared with those of the oracle's sequential
+    form (the nodes the procedure of Section 3 evaluates), bit for bit.
+  * Tolerated endpoint draws are bounded: their count may not exceed BOUNDARY_DRAW_LIMIT(V, draws)
+    (three times the expected number of draws whose uniform falls within float rounding of one of
+    the V interval boundaries, at least 3 events).
   * Naive sampling (mode 2): every emitted token is such a draw; the first differing token of a
     sequence is judged by the endpoint rule and the rest of that sequence is skipped.
 """
@@ -36,6 +42,15 @@ NEAR_TIE_SHARE = 1e-4
 # tests inside the band by chance alone).  Up to this many events are always allowed.
 NEAR_TIE_MIN_EVENTS = 3
 RESIDUAL_TOL = {"fp32": 1e-5, "bf16": 2e-3, "fp16": 2e-3}
+STATUS_NO_MASS = 4
+
+
+def boundary_draw_limit(vocab: int, draws: int) -> float:
+    """Most inverse-CDF draws that may land on the other side of an interval boundary.  A float32
+    evaluation places each of the V boundaries within about 1e-7 (CDF units) of its exact position,
+    so a draw differs with probability about 2e-7 * V; three times that expectation is allowed,
+    and never fewer than 3 events."""
+    return max(3.0, 3 * 2e-7 * vocab * draws)
 
 
 @dataclass
@@ -46,7 +61,9 @@ class ParityReport:
     n_flipped: int = 0               # nodes whose decision differs inside the near-tie band
     n_excluded_sequences: int = 0    # sequences whose oracle path crosses a flipped node
     n_bonus_tolerated: int = 0       # endpoint tokens that differ within the CDF tolerance
+    n_bonus_draws: int = 0           # endpoint draws that were compared
     n_nodes_compared: int = 0
+    excluded: List[int] = field(default_factory=list)   # sequences left out of the path comparison
     max_residual_err: float = 0.0
     failures: List[str] = field(default_factory=list)
 
@@ -57,7 +74,8 @@ class ParityReport:
     def summary(self) -> dict:
         return {"sequences": self.n_sequences, "tests": self.n_tests, "near_ties": self.n_near_tie,
                 "flipped": self.n_flipped, "excluded_sequences": self.n_excluded_sequences,
-                "bonus_tolerated": self.n_bonus_tolerated, "max_residual_err": self.max_residual_err,
+                "bonus_tolerated": self.n_bonus_tolerated, "bonus_draws": self.n_bonus_draws,
+                "max_residual_err": self.max_residual_err,
                 "failures": len(self.failures)}
 
 
@@ -95,15 +113,22 @@ def _node_residual(target_b, draft_b, parent, cand_b, unif_b, n, first, count, T
 
 def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: str, *,
             accept_len, tokens, residual=None, node_accept=None, node_bonus=None, status=None,
-            oracle_result=None, max_failures: int = 20) -> ParityReport:
+            path_nodes=None, oracle_result=None, max_failures: int = 20) -> ParityReport:
     """target/draft: float32 numpy (exact widening of the rounded logits); the keyword arrays are
-    the outputs under test (numpy)."""
+    the outputs under test (numpy).  path_nodes (tree nodes of the accepted tokens, -1 padded), when
+    given, is compared too and lets a diverging walk be traced to the test where it diverged."""
     parent = np.asarray(parent, dtype=np.int32)
     ref = oracle_result if oracle_result is not None else oracle_verify(
         target, draft if T > 0 else None, parent, cand, unif, T, mode)
     B, n_nodes = cand.shape
+    V = target.shape[-1]
     first, count = _children(parent)
     rep = ParityReport(n_sequences=B)
+    # the status words describe the walk: the oracle's sequential form evaluates exactly those nodes
+    ref_status = None
+    if status is not None:
+        ref_status = oracle_verify(target, draft if T > 0 else None, parent, cand, unif, T, mode,
+                                   sequential=True, want_residual=False).status
     tol = RESIDUAL_TOL[dtype_name]
 
     def fail(msg):
@@ -142,6 +167,7 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
         both_stop = (ref.node_accept < 0) & ~flipped
         if node_accept is not None:
             both_stop &= node_accept < 0
+        rep.n_bonus_draws += int(both_stop.sum()) if T > 0 else 0
         diff = np.argwhere(both_stop & (node_bonus != ref.node_bonus))
         for b, n in diff:
             g = int(node_bonus[b, n])
@@ -169,8 +195,31 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
             path_flipped |= bool(flipped[b, n])
         if path_flipped:
             rep.n_excluded_sequences += 1
+            rep.excluded.append(b)
             continue
         L = int(ref.accept_len[b])
+        if path_nodes is not None and T > 0 and mode != 2:
+            # where does the walk under test leave the oracle's?  At that node both evaluated the same
+            # tests in the same order; the first test whose outcome differs decides
+            po, nn = [], 0
+            while ref.node_accept[b, nn] >= 0:
+                nn = int(ref.node_accept[b, nn])
+                po.append(nn)
+            pg = [int(x) for x in path_nodes[b] if x >= 0]
+            if po != pg:
+                i = 0
+                while i < min(len(po), len(pg)) and po[i] == pg[i]:
+                    i += 1
+                ends = [c for c in ((po[i] if i < len(po) else -1), (pg[i] if i < len(pg) else -1)) if c >= 0]
+                i_star = min(ends)
+                rho, u = ref.node_ratio[b, i_star], float(unif[b, i_star, 0])
+                if rho >= 0 and abs(u - rho) < NEAR_TIE:
+                    rep.n_flipped += 1
+                    rep.n_excluded_sequences += 1
+                    rep.excluded.append(b)
+                else:
+                    fail(f"seq {b}: path {pg}, oracle {po} (u={u}, rho={rho} at node {i_star})")
+                continue
         if mode == 2 and T > 0 and not np.array_equal(tokens[b], ref.tokens[b]):
             # naive sampling: every emitted token is itself a draw by inverse CDF.  At the first
             # position where the token sequences differ, the other token passes under the same
@@ -183,6 +232,7 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
                                               float(unif[b, node, 1])):
                 rep.n_bonus_tolerated += 1
                 rep.n_excluded_sequences += 1
+                rep.excluded.append(b)
             else:
                 fail(f"seq {b}: tokens {tokens[b].tolist()}, oracle {ref.tokens[b].tolist()}")
             continue
@@ -195,19 +245,24 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
         if not (tokens[b, L + 1:] == -1).all():
             fail(f"seq {b}: padding after the endpoint token is not -1")
         g, o = int(tokens[b, L]), int(ref.tokens[b, L])
+        if T > 0 and node_bonus is None:
+            rep.n_bonus_draws += (L + 1) if mode == 2 else 1
         if g != o:
             if T > 0 and _bonus_tolerated(ref.residual[b], g, float(unif[b, n, 1])):
                 if node_bonus is None:
                     rep.n_bonus_tolerated += 1
             else:
                 fail(f"seq {b}: endpoint token {g}, oracle {o}")
-        if residual is not None:
+        if residual is not None and not (int(ref.status[b]) & STATUS_NO_MASS):
             err = float(np.abs(residual[b].astype(np.float64) - ref.residual[b]).max())
             rep.max_residual_err = max(rep.max_residual_err, err)
             if not err <= tol:
                 fail(f"seq {b}: residual max abs error {err:.3e} > {tol:.1e}")
-        if status is not None and int(status[b]) != int(ref.status[b]):
-            fail(f"seq {b}: status {int(status[b])}, oracle {int(ref.status[b])}")
+        if status is not None and int(status[b]) != int(ref_status[b]):
+            fail(f"seq {b}: status {int(status[b])}, oracle (sequential form) {int(ref_status[b])}")
+    if rep.n_bonus_tolerated > boundary_draw_limit(V, max(rep.n_bonus_draws, 1)):
+        fail(f"{rep.n_bonus_tolerated} of {rep.n_bonus_draws} endpoint draws differ inside the tolerance: "
+             f"more than the {boundary_draw_limit(V, max(rep.n_bonus_draws, 1)):.1f} float rounding explains")
     return rep
 
 
@@ -253,4 +308,7 @@ def compare_samples(draft, parent, unif_draw, T: float, mode: int, cand, node_be
                 rep.n_tolerated += 1
             elif len(rep.failures) < max_failures:
                 rep.failures.append(f"seq {b} node {n} draw {i}: token {g}, oracle {int(ref[b, ch[i]])}")
+    if T > 0 and rep.n_tolerated > boundary_draw_limit(V, max(rep.n_draws, 1)):
+        rep.failures.append(f"{rep.n_tolerated} of {rep.n_draws} draws differ inside the tolerance: more than the "
+                            f"{boundary_draw_limit(V, max(rep.n_draws, 1)):.1f} float rounding explains")
     return rep

@@ -19,7 +19,7 @@
  *   - Section 3.2, Eq. 1 (how the k candidates of a node are drawn without replacement);
  *     the draws themselves are made deterministic by supplied uniforms.
  *   - Section 4.1 (sampling setups): temperature 1 is plain softmax sampling,
- *     temperature 0 is argmax.  Section 4.4 states that at temperature 0 the
+ *     temperature 0 is argmax.  Section 4.5 states that at temperature 0 the
  *     with-replacement algorithm degenerates to standard speculative decoding and
  *     the without-replacement one to naive sampling; both reduce to "accept a
  *     candidate iff it equals the target argmax".
@@ -35,9 +35,10 @@
  *   - every test owns a pre-drawn uniform, indexed by the child node it tests;
  *   - if the residual mass is exactly 0 the residual is left unchanged and a
  *     status bit is set;
- *   - a draft row from which no distribution can be formed (its softmax is NaN)
- *     rejects every candidate of its node, leaves p as it is and sets the same
- *     status bit;
+ *   - Algorithm 2's "q(x~) := 0; q := q / sum q" is the identity, and is skipped, where
+ *     x~ is not a token or has draft probability 0 already (nothing is removed);
+ *     as a consequence a draft row from which no distribution can be formed (its
+ *     softmax is NaN) rejects every candidate of its node and leaves p as it is;
  *   - "r ~ U(0,1)" is an input of the verification step; a supplied r that is
  *     not below 1 (NaN included) counts as 1 there, so that every value a caller can pass has a defined
  *     outcome: such an r accepts exactly when p(x~) >= q(x~).  (An r <= 0 needs no
@@ -167,9 +168,12 @@ int32_t mcsd_oracle_mcss(double *p, double *q, int32_t V, const int32_t *cand,
         } else {
             *status |= ORACLE_STATUS_DEGENERATE;
         }
-        if (mode == 1) {
-            /* Algorithm 2 only: q(x~) <- 0, q := q / sum q */
-            if (valid) q[xt] = 0.0;
+        if (mode == 1 && valid && q[xt] > 0.0) {
+            /* Algorithm 2 only: q(x~) <- 0, q := q / sum q.  Where x~ is not a token, or has
+             * draft probability 0 already, nothing is removed and the step is the identity:
+             * q is left as it is (dividing it by its own sum, 1 up to rounding, would only
+             * disturb the last bits, which matters when p and q are equal). */
+            q[xt] = 0.0;
             double w = 0.0;
             for (int32_t x = 0; x < V; ++x) w += q[x];
             if (w > 0.0)
@@ -314,7 +318,7 @@ static int32_t verify_node(int32_t n, int32_t n_nodes, int32_t n_internal, int32
     }
     mcsd_oracle_softmax(t, V, T, residual); /* p */
     if (mode == 2 && k > 0) {
-        /* Naive sampling (the baseline of Section 2 that Section 4.4 and Appendix C compare
+        /* Naive sampling (the baseline of Section 2 that Section 4.5 and Appendix C compare
          * with): draw x from the target distribution itself; if one of the candidates
          * carries x the walk moves to (the first) such child, otherwise x is the endpoint
          * token.  The draft distribution plays no part. */
@@ -341,20 +345,6 @@ static int32_t verify_node(int32_t n, int32_t n_nodes, int32_t n_internal, int32
         cands[i] = cand_b[first + i];
         r[i] = (double)unif_b[2 * (first + i)];
         if (!(r[i] < 1.0)) r[i] = 1.0; /* supplied in place of r ~ U(0,1): not below 1 counts as 1 */
-    }
-    if (qbuf[0] != qbuf[0]) {
-        /* No draft distribution can be formed from this row (all -inf, or a NaN or +inf logit:
-         * the normaliser is not a positive number and every entry is NaN).  There is no q to
-         * test against: every candidate is rejected without a ratio, p stays as it is, and
-         * the failed residual update is reported as a zero-mass one. */
-        for (int32_t i = 0; i < k; ++i) {
-            if (cands[i] < 0 || cands[i] >= V) *status |= ORACLE_STATUS_BAD_TOKEN;
-            if (ratio_b) ratio_b[first + i] = -1.0;
-        }
-        *status |= ORACLE_STATUS_DEGENERATE;
-        *bonus = mcsd_oracle_invcdf(residual, V, (double)unif_b[2 * n + 1]);
-        if (*bonus < 0) *status |= ORACLE_STATUS_NO_MASS;
-        return -1;
     }
     int32_t acc = mcsd_oracle_mcss(residual, qbuf, V, cands, r, k, mode, ratio, S, status);
     if (ratio_b)

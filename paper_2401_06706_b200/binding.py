@@ -25,7 +25,8 @@ MAX_NODES, MAX_CHILDREN, MAX_VOCAB = 512, 32, 65536
 EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path", "mcsd_sample_candidates", "mcsd_tree_attention_layout",
            "mcsd_gather_accepted_kv",
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
-           "mcsd_version")
+           "mcsd_version", "mcsd_set_option", "mcsd_get_option", "mcsd_release_host_staging")
+OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL = range(7)
 
 
 class McsdDesc(ctypes.Structure):
@@ -89,6 +90,12 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_status_string.restype = ctypes.c_char_p
     lib.mcsd_version.argtypes = []
     lib.mcsd_version.restype = ctypes.c_int
+    lib.mcsd_set_option.argtypes = [ctypes.c_int, ctypes.c_int]
+    lib.mcsd_set_option.restype = ctypes.c_int
+    lib.mcsd_get_option.argtypes = [ctypes.c_int]
+    lib.mcsd_get_option.restype = ctypes.c_int
+    lib.mcsd_release_host_staging.argtypes = []
+    lib.mcsd_release_host_staging.restype = ctypes.c_int
     if path is None:
         _lib = lib
     return lib
@@ -116,6 +123,20 @@ def mcsd_tree_depth(parent) -> int:
 
 def mcsd_last_launch_count() -> int:
     return int(load_library().mcsd_last_launch_count())
+
+
+def mcsd_set_option(option: int, value: int) -> None:
+    _check(load_library().mcsd_set_option(int(option), int(value)))
+
+
+def mcsd_get_option(option: int) -> int:
+    rc = load_library().mcsd_get_option(int(option))
+    _check(rc if rc < 0 else 0)
+    return rc
+
+
+def mcsd_release_host_staging() -> None:
+    _check(load_library().mcsd_release_host_staging())
 
 
 def _n_internal(parent: np.ndarray) -> int:

@@ -14,6 +14,29 @@ namespace {
 
 thread_local int g_last_launches = 0;
 
+// Tuning and test overrides (mcsd_set_option).  Initial values come from the environment
+// variables of the same names, read once when the library is loaded.
+int env_int(const char *name, int fallback)
+{
+    const char *v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : fallback;
+}
+struct Options {
+    int v[MCSD_OPT_COUNT];
+    Options()
+    {
+        for (int &x : v) x = 0;
+        v[MCSD_OPT_CLUSTER] = env_int("MCSD_CLUSTER", 0);
+        v[MCSD_OPT_EPT] = env_int("MCSD_EPT", 0);
+        v[MCSD_OPT_DIRECT] = env_int("MCSD_DIRECT", 0);
+        v[MCSD_OPT_SAMPLE_AHEAD] = env_int("MCSD_SAMPLE_AHEAD", 100);
+        v[MCSD_OPT_WAIT_POLLS] = 0;
+        v[MCSD_OPT_TEST_EXTRA_TX] = 0;
+        v[MCSD_OPT_PDL] = env_int("MCSD_PDL", 1);
+    }
+};
+Options g_opt;
+
 struct TreePlan {
     int gamma = 0;
     uint16_t child_first[MCSD_MAX_NODES];
@@ -50,6 +73,34 @@ int plan_tree(const int32_t *parent, int n_nodes, int n_internal, TreePlan *plan
     return MCSD_OK;
 }
 
+// The tree a host thread verified last is almost always the tree it verifies next: its plan is
+// kept and found again by comparing the parent array (at most 2 KB).
+struct CachedPlan {
+    int n_nodes = 0, n_internal = -2;
+    int32_t parent[MCSD_MAX_NODES];
+    TreePlan plan;
+};
+thread_local CachedPlan g_plan_cache;
+
+int plan_tree_cached(const int32_t *parent, int n_nodes, int n_internal, TreePlan *plan)
+{
+    if (!parent) return MCSD_ERR_NULL;
+    CachedPlan &cp = g_plan_cache;
+    if (n_nodes >= 1 && n_nodes <= MCSD_MAX_NODES && cp.n_nodes == n_nodes && cp.n_internal == n_internal &&
+        std::memcmp(cp.parent, parent, sizeof(int32_t) * n_nodes) == 0) {
+        *plan = cp.plan;
+        return MCSD_OK;
+    }
+    const int rc = plan_tree(parent, n_nodes, n_internal, plan);
+    if (rc == MCSD_OK) {
+        cp.n_nodes = n_nodes;
+        cp.n_internal = n_internal;
+        std::memcpy(cp.parent, parent, sizeof(int32_t) * n_nodes);
+        cp.plan = *plan;
+    }
+    return rc;
+}
+
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Workspace {
@@ -74,7 +125,7 @@ Workspace carve(void *base, long long n_items, long long n_leaf_items, int batch
     w.node_accept = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
     w.node_bonus = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
     w.stats = reinterpret_cast<NodeStats *>(take(sizeof(NodeStats) * n_items));
-    w.leaf_part = reinterpret_cast<float2 *>(take(sizeof(float2) * 32 * n_leaf_items));
+    w.leaf_part = reinterpret_cast<float2 *>(take(sizeof(float2) * kLeafEntries * n_leaf_items));
     w.status = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
     w.path[0] = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
     w.path[1] = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
@@ -85,6 +136,7 @@ Workspace carve(void *base, long long n_items, long long n_leaf_items, int batch
 int check_desc(const mcsd_desc *d)
 {
     if (!d) return MCSD_ERR_NULL;
+    if (d->reserved != 0) return MCSD_ERR_SHAPE;
     if (d->batch < 0 || d->n_nodes < 1 || d->vocab < 1 || d->n_internal < 0 ||
         d->n_internal > d->n_nodes)
         return MCSD_ERR_SHAPE;
@@ -141,26 +193,20 @@ NodeKernel pick_node_kernel(int dtype, int ept, bool direct, bool path)
     }
 }
 
-int env_int(const char *name, int fallback)
-{
-    const char *v = std::getenv(name);
-    return (v && *v) ? std::atoi(v) : fallback;
-}
-
 struct NodeConfig {
-    int cluster, ept, slice;
+    int cluster, ept, slice, threads;
     bool direct;
 };
 
 // Smallest (cluster size x elements per thread) that holds one vocabulary row,
 // larger per-thread share first so that fewer CTAs have to agree per node.
-// MCSD_CLUSTER / MCSD_EPT / MCSD_DIRECT override the choice (tuning and tests).
+// The options MCSD_OPT_CLUSTER / MCSD_OPT_EPT / MCSD_OPT_DIRECT override the choice (tuning and tests).
 int choose_config(int vocab, int dtype, bool aligned, NodeConfig *cfg)
 {
     const int vec = 16 / elem_bytes(dtype);
     int best_c = 0, best_e = 0;
     long long best_cap = -1;
-    const int force_c = env_int("MCSD_CLUSTER", 0), force_e = env_int("MCSD_EPT", 0);
+    const int force_c = g_opt.v[MCSD_OPT_CLUSTER], force_e = g_opt.v[MCSD_OPT_EPT];
     for (int c = 1; c <= kMaxCluster; ++c) {
         if (force_c && c != force_c) continue;
         for (int ei = 2; ei >= 0; --ei) {
@@ -176,8 +222,9 @@ int choose_config(int vocab, int dtype, bool aligned, NodeConfig *cfg)
     cfg->ept = best_e;
     // every CTA but the last owns a full slice, so that only the last one has ragged warps
     cfg->slice = kNodeThreads * best_e;
+    cfg->threads = kNodeThreads;
     (void)vec;
-    cfg->direct = !aligned || env_int("MCSD_DIRECT", 0) != 0;
+    cfg->direct = !aligned || g_opt.v[MCSD_OPT_DIRECT] != 0;
     return MCSD_OK;
 }
 
@@ -186,7 +233,7 @@ struct OccKey { int dev; NodeKernel fn; int cluster; int clusters; };
 std::mutex g_occ_mutex;
 std::vector<OccKey> g_occ;
 
-int resident_clusters(NodeKernel fn, int cluster, size_t smem, cudaStream_t stream)
+int resident_clusters(NodeKernel fn, int cluster, size_t smem, cudaStream_t stream, int threads = kNodeThreads)
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return -1;
@@ -204,7 +251,7 @@ int resident_clusters(NodeKernel fn, int cluster, size_t smem, cudaStream_t stre
     cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
     cudaFuncAttributes fa = {};
     if (cudaFuncGetAttributes(&fa, fn) == cudaSuccess && smem_sm > 0 && fa.numRegs > 0) {
-        int by_regs = 65536 / (fa.numRegs * kNodeThreads);
+        int by_regs = 65536 / (fa.numRegs * threads);
         if (by_regs < 1) by_regs = 1;
         const size_t per_cta = smem + fa.sharedSizeBytes + 1024;
         size_t want = per_cta * static_cast<size_t>(by_regs);
@@ -215,7 +262,7 @@ int resident_clusters(NodeKernel fn, int cluster, size_t smem, cudaStream_t stre
     }
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(static_cast<unsigned>(cluster * n_sm * 8));
-    lc.blockDim = dim3(kNodeThreads);
+    lc.blockDim = dim3(static_cast<unsigned>(threads));
     lc.dynamicSmemBytes = smem;
     lc.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -247,7 +294,7 @@ int prepare(const mcsd_desc *d, const int32_t *parent, Call *c)
 {
     int rc = check_desc(d);
     if (rc != MCSD_OK) return rc;
-    rc = plan_tree(parent, d->n_nodes, d->n_internal, &c->plan);
+    rc = plan_tree_cached(parent, d->n_nodes, d->n_internal, &c->plan);
     if (rc != MCSD_OK) return rc;
     rc = check_workspace(d);
     if (rc != MCSD_OK) return rc;
@@ -293,12 +340,10 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     if (n_items == 0) return MCSD_OK;
     const int32_t *path_cur = path ? c.ws.path[level & 1] : nullptr;
     int32_t *path_next = path ? c.ws.path[(level + 1) & 1] : nullptr;
-    if (level <= 0) {
-        if (cudaMemsetAsync(c.status, 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
-            return MCSD_ERR_CUDA;
-        if (path && cudaMemsetAsync(c.ws.path[0], 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
-            return MCSD_ERR_CUDA;  // every walk starts at the root
-    }
+    // (the status words need no clearing: the walk stage writes them)
+    if (level == 0 && T == 0.f &&
+        cudaMemsetAsync(c.ws.path[0], 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
+        return MCSD_ERR_CUDA;  // every walk starts at the root
 
     if (T == 0.f) {
         ArgmaxParams p = {};
@@ -333,15 +378,17 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     if (rc != MCSD_OK) return rc;
     NodeKernel fn = pick_node_kernel(d->dtype, cfg.ept, cfg.direct, path);
     const size_t smem = node_smem_bytes(elem_bytes(d->dtype), cfg.ept, cfg.direct);
-    const int resident = resident_clusters(fn, cfg.cluster, smem, c.stream);
+    const int resident = resident_clusters(fn, cfg.cluster, smem, c.stream, cfg.threads);
     if (resident < 1) return MCSD_ERR_CUDA;
     const long long n_clusters = n_items < resident ? n_items : resident;
 
     NodeParams p = {};
     p.target = target; p.draft = draft; p.cand = cand; p.unif = unif;
     p.node_accept = c.node_accept; p.node_ratio = d->node_ratio;
-    p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part; p.status = c.status;
+    p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part;
     p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
+    p.wait_polls = g_opt.v[MCSD_OPT_WAIT_POLLS] > 0 ? static_cast<uint32_t>(g_opt.v[MCSD_OPT_WAIT_POLLS]) : kWaitPolls;
+    p.test_extra_tx = static_cast<uint32_t>(g_opt.v[MCSD_OPT_TEST_EXTRA_TX]) & ~15u;
     p.B = d->batch; p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
     p.slice = cfg.slice;
     p.n_items = static_cast<int32_t>(n_items);
@@ -356,7 +403,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
 
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(static_cast<unsigned>(n_clusters * cfg.cluster));
-    lc.blockDim = dim3(kNodeThreads);
+    lc.blockDim = dim3(static_cast<unsigned>(cfg.threads));
     lc.dynamicSmemBytes = smem;
     lc.stream = c.stream;
     cudaLaunchAttribute attr[1];
@@ -380,7 +427,6 @@ int launch_naive(const Call &c, const void *target, const int32_t *cand, const f
 {
     const mcsd_desc *d = c.d;
     if (d->batch == 0) return MCSD_OK;
-    if (cudaMemsetAsync(c.status, 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess) return MCSD_ERR_CUDA;
     NaiveParams p = {};
     p.target = target; p.cand = cand; p.unif = unif;
     p.node_accept = c.node_accept;
@@ -430,28 +476,41 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
         NodeConfig cfg;
         const int rc = choose_config(d->vocab, d->dtype, node_aligned, &cfg);
         if (rc != MCSD_OK) return rc;
-        p.n_entries = cfg.cluster * kNodeWarps;
+        p.n_entries = cfg.cluster * (cfg.threads / 32);
+    }
+    // The walk stage may be set up on the GPU while the node stage still runs (programmatic
+    // dependent launch): its CTAs wait for the node stage's results at their first instruction.
+    p.pdl = g_opt.v[MCSD_OPT_PDL] ? 1 : 0;
+    using WalkKernel = void (*)(const WalkParams);
+    WalkKernel fn;
+    int threads;
+    if (d->vocab <= MCSD_MAX_VOCAB / 2) {
+        threads = 512;
+        fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 512>
+           : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 512> : walk_kernel<MCSD_DTYPE_F16, 512>;
+    } else {
+        threads = 1024;
+        fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 1024>
+           : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 1024> : walk_kernel<MCSD_DTYPE_F16, 1024>;
     }
     // all-nodes pass first (only when per-node endpoint tokens or distributions were asked for;
     // at temperature 0 the tokens are there already), then the walks
     const bool want_all = all_nodes_allowed && ((T > 0.f && d->node_bonus) || d->node_residual);
     for (int all = want_all ? 1 : 0; all >= 0; --all) {
         p.all_nodes = all;
-        const unsigned grid = static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch);
-        if (d->vocab <= MCSD_MAX_VOCAB / 2) {
-            switch (d->dtype) {
-            case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32, 512><<<grid, 512, 0, c.stream>>>(p); break;
-            case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16, 512><<<grid, 512, 0, c.stream>>>(p); break;
-            default: walk_kernel<MCSD_DTYPE_F16, 512><<<grid, 512, 0, c.stream>>>(p); break;
-            }
-        } else {
-            switch (d->dtype) {
-            case MCSD_DTYPE_F32: walk_kernel<MCSD_DTYPE_F32, 1024><<<grid, 1024, 0, c.stream>>>(p); break;
-            case MCSD_DTYPE_BF16: walk_kernel<MCSD_DTYPE_BF16, 1024><<<grid, 1024, 0, c.stream>>>(p); break;
-            default: walk_kernel<MCSD_DTYPE_F16, 1024><<<grid, 1024, 0, c.stream>>>(p); break;
-            }
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3(static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch));
+        lc.blockDim = dim3(static_cast<unsigned>(threads));
+        lc.stream = c.stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = p.pdl ? 1 : 0;
+        if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
+            cudaGetLastError();
+            return MCSD_ERR_CUDA;
         }
-        if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
         g_last_launches += 1;
     }
     return MCSD_OK;
@@ -500,6 +559,20 @@ int mcsd_tree_depth(const int32_t *tree_parent, int32_t n_nodes)
 }
 
 int mcsd_last_launch_count(void) { return g_last_launches; }
+
+int mcsd_set_option(int option, int value)
+{
+    if (option < 0 || option >= MCSD_OPT_COUNT) return MCSD_ERR_SHAPE;
+    if (value < 0) return MCSD_ERR_SHAPE;
+    g_opt.v[option] = value;
+    return MCSD_OK;
+}
+
+int mcsd_get_option(int option)
+{
+    if (option < 0 || option >= MCSD_OPT_COUNT) return MCSD_ERR_SHAPE;
+    return g_opt.v[option];
+}
 
 int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                       const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
@@ -634,8 +707,8 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MCSD_ERR_CUDA;
         p.prefetch_ahead = n_sm * (1024 / threads);
-        // (MCSD_SAMPLE_AHEAD: percent of that distance, for tuning)
-        p.prefetch_ahead = static_cast<int>(static_cast<long long>(p.prefetch_ahead) * env_int("MCSD_SAMPLE_AHEAD", 100) / 100);
+        // (MCSD_OPT_SAMPLE_AHEAD: percent of that distance, for tuning)
+        p.prefetch_ahead = static_cast<int>(static_cast<long long>(p.prefetch_ahead) * g_opt.v[MCSD_OPT_SAMPLE_AHEAD] / 100);
     }
     if (!small) {
         switch (desc->dtype) {
@@ -762,6 +835,38 @@ int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const v
                        temperature, replacement_mode, out_accept_len, out_tokens, out_residual);
 }
 
+// ---- mcsd_verify_host: device staging buffers kept between calls ------------------------
+namespace {
+struct HostSlot {
+    cudaStream_t stream = nullptr;
+    unsigned char *buf = nullptr;   // one allocation, carved per call
+    size_t bytes = 0;
+};
+struct HostStaging {
+    HostSlot slot[2];
+};
+std::mutex g_host_mutex;
+HostStaging g_host[kMaxDevices];
+
+void release_staging(HostStaging &hs)
+{
+    for (HostSlot &sl : hs.slot) {
+        if (sl.buf) cudaFree(sl.buf);
+        if (sl.stream) cudaStreamDestroy(sl.stream);
+        sl = HostSlot();
+    }
+}
+}  // namespace
+
+int mcsd_release_host_staging(void)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MCSD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_host_mutex);
+    release_staging(g_host[dev]);
+    return MCSD_OK;
+}
+
 int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                      float temperature, int replacement_mode, int32_t *out_accept_len,
@@ -770,7 +875,7 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
     int rc = check_desc(desc);
     if (rc != MCSD_OK) return rc;
     TreePlan plan;
-    rc = plan_tree(tree_parent, desc->n_nodes, desc->n_internal, &plan);
+    rc = plan_tree_cached(tree_parent, desc->n_nodes, desc->n_internal, &plan);
     if (rc != MCSD_OK) return rc;
     rc = check_common(desc, target_logits, draft_logits, cand_tokens, uniforms, temperature,
                       replacement_mode, true, true);
@@ -778,6 +883,8 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
     if (!out_accept_len || !out_tokens) return MCSD_ERR_NULL;
     const int B = desc->batch;
     if (B == 0) return MCSD_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MCSD_ERR_CUDA;
 
     const size_t es = elem_bytes(desc->dtype);
     const bool use_draft = temperature > 0.f && desc->n_internal > 0 && replacement_mode != MCSD_MODE_NAIVE;
@@ -792,76 +899,75 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
     if (per > static_cast<size_t>((B + 1) / 2)) per = static_cast<size_t>((B + 1) / 2);
     const int chunk = static_cast<int>(per);
 
-    struct Slot {
-        cudaStream_t stream = nullptr;
-        unsigned char *t = nullptr, *d = nullptr;
-        int32_t *cand = nullptr, *len = nullptr, *tok = nullptr, *status = nullptr;
-        float *unif = nullptr, *res = nullptr;
-        void *ws = nullptr;
-    } slot[2];
     mcsd_desc cd = *desc;
     cd.batch = chunk;
     cd.node_accept = nullptr; cd.node_bonus = nullptr; cd.node_ratio = nullptr; cd.out_path_nodes = nullptr;
     cd.node_residual = nullptr;
     const size_t ws_bytes = mcsd_workspace_bytes(&cd);
+    // layout of one slot's staging buffer
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes, 256); return o; };
+    const size_t o_t = take(t_seq * chunk), o_d = take(d_seq * chunk), o_c = take(c_seq * chunk),
+                 o_u = take(u_seq * chunk), o_len = take(sizeof(int32_t) * chunk), o_tok = take(tok_seq * chunk),
+                 o_st = take(sizeof(int32_t) * chunk), o_res = take(out_residual ? res_seq * chunk : 0),
+                 o_ws = take(ws_bytes);
+    const size_t need = off;
+
+    // one call at a time per device uses the staging buffers
+    std::lock_guard<std::mutex> lock(g_host_mutex);
+    HostStaging &hs = g_host[dev];
     bool ok = true;
     auto chk = [&](cudaError_t e) { if (e != cudaSuccess) ok = false; return e == cudaSuccess; };
-    for (int s = 0; s < 2 && ok; ++s) {
-        Slot &sl = slot[s];
-        chk(cudaStreamCreateWithFlags(&sl.stream, cudaStreamNonBlocking));
-        chk(cudaMalloc(&sl.t, t_seq * chunk));
-        if (use_draft) chk(cudaMalloc(&sl.d, d_seq * chunk));
-        chk(cudaMalloc(&sl.cand, c_seq * chunk));
-        chk(cudaMalloc(&sl.unif, u_seq * chunk));
-        chk(cudaMalloc(&sl.len, sizeof(int32_t) * chunk));
-        chk(cudaMalloc(&sl.tok, tok_seq * chunk));
-        chk(cudaMalloc(&sl.status, sizeof(int32_t) * chunk));
-        if (out_residual) chk(cudaMalloc(&sl.res, res_seq * chunk));
-        chk(cudaMalloc(&sl.ws, ws_bytes));
+    for (HostSlot &sl : hs.slot) {
+        if (!sl.stream) chk(cudaStreamCreateWithFlags(&sl.stream, cudaStreamNonBlocking));
+        if (ok && sl.bytes < need) {
+            if (sl.buf) cudaFree(sl.buf);
+            sl.buf = nullptr;
+            sl.bytes = 0;
+            if (chk(cudaMalloc(&sl.buf, need))) sl.bytes = need;
+        }
     }
     int launches = 0;
     for (int b0 = 0, i = 0; b0 < B && ok && rc == MCSD_OK; b0 += chunk, ++i) {
-        Slot &sl = slot[i & 1];
+        HostSlot &sl = hs.slot[i & 1];
         const int nb = (B - b0 < chunk) ? B - b0 : chunk;
+        unsigned char *base = sl.buf;
         const unsigned char *ht = static_cast<const unsigned char *>(target_logits) + t_seq * b0;
-        chk(cudaMemcpyAsync(sl.t, ht, t_seq * nb, cudaMemcpyHostToDevice, sl.stream));
+        chk(cudaMemcpyAsync(base + o_t, ht, t_seq * nb, cudaMemcpyHostToDevice, sl.stream));
         if (use_draft) {
             const unsigned char *hd = static_cast<const unsigned char *>(draft_logits) + d_seq * b0;
-            chk(cudaMemcpyAsync(sl.d, hd, d_seq * nb, cudaMemcpyHostToDevice, sl.stream));
+            chk(cudaMemcpyAsync(base + o_d, hd, d_seq * nb, cudaMemcpyHostToDevice, sl.stream));
         }
-        chk(cudaMemcpyAsync(sl.cand, cand_tokens + static_cast<size_t>(b0) * desc->n_nodes, c_seq * nb,
+        chk(cudaMemcpyAsync(base + o_c, cand_tokens + static_cast<size_t>(b0) * desc->n_nodes, c_seq * nb,
                             cudaMemcpyHostToDevice, sl.stream));
         if (uniforms)
-            chk(cudaMemcpyAsync(sl.unif, uniforms + static_cast<size_t>(b0) * 2 * desc->n_nodes, u_seq * nb,
+            chk(cudaMemcpyAsync(base + o_u, uniforms + static_cast<size_t>(b0) * 2 * desc->n_nodes, u_seq * nb,
                                 cudaMemcpyHostToDevice, sl.stream));
+        if (!ok) break;
         cd.batch = nb;
         cd.stream = sl.stream;
-        cd.workspace = sl.ws;
+        cd.workspace = base + o_ws;
         cd.workspace_bytes = ws_bytes;
-        cd.out_status = sl.status;
-        if (ok)
-            rc = mcsd_verify(&cd, sl.t, sl.d, tree_parent, sl.cand, uniforms ? sl.unif : nullptr, temperature,
-                             replacement_mode, sl.len, sl.tok, sl.res);
+        cd.out_status = reinterpret_cast<int32_t *>(base + o_st);
+        rc = mcsd_verify(&cd, base + o_t, use_draft ? base + o_d : nullptr, tree_parent,
+                         reinterpret_cast<const int32_t *>(base + o_c),
+                         uniforms ? reinterpret_cast<const float *>(base + o_u) : nullptr, temperature,
+                         replacement_mode, reinterpret_cast<int32_t *>(base + o_len),
+                         reinterpret_cast<int32_t *>(base + o_tok),
+                         out_residual ? reinterpret_cast<float *>(base + o_res) : nullptr);
+        if (rc != MCSD_OK) break;   // nothing of this slice is copied back
         launches += g_last_launches;
-        chk(cudaMemcpyAsync(out_accept_len + b0, sl.len, sizeof(int32_t) * nb, cudaMemcpyDeviceToHost, sl.stream));
-        chk(cudaMemcpyAsync(out_tokens + static_cast<size_t>(b0) * (plan.gamma + 1), sl.tok, tok_seq * nb,
+        chk(cudaMemcpyAsync(out_accept_len + b0, base + o_len, sizeof(int32_t) * nb, cudaMemcpyDeviceToHost, sl.stream));
+        chk(cudaMemcpyAsync(out_tokens + static_cast<size_t>(b0) * (plan.gamma + 1), base + o_tok, tok_seq * nb,
                             cudaMemcpyDeviceToHost, sl.stream));
         if (out_residual)
-            chk(cudaMemcpyAsync(out_residual + static_cast<size_t>(b0) * desc->vocab, sl.res, res_seq * nb,
+            chk(cudaMemcpyAsync(out_residual + static_cast<size_t>(b0) * desc->vocab, base + o_res, res_seq * nb,
                                 cudaMemcpyDeviceToHost, sl.stream));
         if (out_status)
-            chk(cudaMemcpyAsync(out_status + b0, sl.status, sizeof(int32_t) * nb, cudaMemcpyDeviceToHost, sl.stream));
+            chk(cudaMemcpyAsync(out_status + b0, base + o_st, sizeof(int32_t) * nb, cudaMemcpyDeviceToHost, sl.stream));
     }
-    for (int s = 0; s < 2; ++s) {
-        Slot &sl = slot[s];
-        if (sl.stream) { chk(cudaStreamSynchronize(sl.stream)); }
-    }
-    for (int s = 0; s < 2; ++s) {
-        Slot &sl = slot[s];
-        cudaFree(sl.t); cudaFree(sl.d); cudaFree(sl.cand); cudaFree(sl.unif); cudaFree(sl.len);
-        cudaFree(sl.tok); cudaFree(sl.status); cudaFree(sl.res); cudaFree(sl.ws);
-        if (sl.stream) cudaStreamDestroy(sl.stream);
-    }
+    for (HostSlot &sl : hs.slot)
+        if (sl.stream) chk(cudaStreamSynchronize(sl.stream));
     g_last_launches = launches;
     if (rc != MCSD_OK) return rc;
     if (!ok) { cudaGetLastError(); return MCSD_ERR_CUDA; }

@@ -1,4 +1,4 @@
-// argmax_kernel (T == 0): the greedy rule of Section 4.4, one CTA per target row.
+// argmax_kernel (T == 0): the greedy rule of Section 4.5, one CTA per target row.
 #pragma once
 
 #include "mcsd_common.cuh"

@@ -15,15 +15,26 @@ namespace mcsd {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxCluster = 8;
-// Polls of a bounded wait before it gives up; with the back-off between polls the
-// bound is about two seconds, far beyond any legitimate wait.
+// Per-warp statistics entries a leaf row can have (cluster size * warps per CTA of the node kernel).
+constexpr int kLeafEntries = kMaxCluster * 4;
+// Polls of a bounded wait before it gives up; a poll suspends the thread for up to
+// kWaitSuspendNs, so the bound is about two seconds, far beyond any legitimate wait.
 constexpr uint32_t kWaitPolls = 1u << 21;
+// Longest time one poll may keep a thread suspended (a hint to the hardware).
+constexpr uint32_t kWaitSuspendNs = 1000u;
 
+// What the node kernel leaves per node with children (32 bytes, two 16-byte stores).
 struct __align__(16) NodeStats {
     float r_t, r_d;  // references of the sums: ceil(row maximum * scale), log2 units
     float z_t, z_d;  // sum_x exp2(l * scale - r)
-    float c, s;      // final c_n and S_n of the node (0 and 1 for a leaf)
-    int32_t pad0, pad1;
+    // The residual left when every candidate was rejected is max(p - c q, 0) (unnormalised).
+    // The sum that follows the LAST rejection is not formed by the node kernel: nothing is
+    // tested against that residual, only a walk that stops here draws from it, and the walk
+    // kernel forms the sum then.  Should it be zero, the residual before that rejection,
+    // max(p - c_prev q, 0), is the one that is kept.
+    float c, c_prev;
+    int32_t status;  // MCSD_STATUS_* bits met at this node
+    int32_t pad;
 };
 
 struct NodeParams {
@@ -34,8 +45,7 @@ struct NodeParams {
     int32_t *node_accept;
     float *node_ratio;  // may be null
     NodeStats *stats;   // [B][n_nodes], written for nodes with children
-    float2 *leaf_part;  // [B][n_nodes - n_internal][32] per-warp (reference, sum) of every leaf row
-    int32_t *status;  // [B]
+    float2 *leaf_part;  // [B][n_nodes - n_internal][kLeafEntries] per-warp (reference, sum) of every leaf row
     long long ld_t, ld_d;
     int32_t B, n_nodes, n_internal, V;
     int32_t slice;   // vocabulary elements owned by one CTA of the cluster
@@ -45,6 +55,8 @@ struct NodeParams {
     // follows each of its sequences from the root through the accepted children and evaluates
     // only the nodes on that walk.
     int32_t mode;
+    uint32_t wait_polls;      // poll budget of the exchange wait (kWaitPolls unless a test shortens it)
+    uint32_t test_extra_tx;   // 0; a test of the expiry path arms the exchange barrier for this many bytes nobody sends
     float scale;     // log2(e) / T rounded to float ...
     float scale_lo;  // ... and what the rounding dropped (for the candidates' own probabilities)
     uint16_t child_first[MCSD_MAX_NODES];
@@ -171,19 +183,22 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
+    // the last operand lets the hardware keep the thread suspended for up to that many
+    // nanoseconds while the phase is pending, instead of returning to a polling loop
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kWaitSuspendNs) : "memory");
     return ok != 0;
 }
-// Bounded wait with back-off (a waiting thread must not eat the issue slots of the
-// working ones): false when the poll budget ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitPolls; ++i) {
+// Bounded wait: false when the poll budget ran out.  A poll that finds the phase pending
+// suspends the thread in hardware (see above), so a waiting thread does not eat the issue
+// slots of the working ones.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t polls = kWaitPolls) {
+    for (uint32_t i = 0; i < polls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(i < 64 ? 64 : 1000);
+        if (i >= 64) __nanosleep(1000);   // (whatever the hardware makes of the hint, a long wait backs off)
     }
     return false;
 }
@@ -351,6 +366,102 @@ __device__ __forceinline__ int warp_multi_sum(const float (&v)[N], int lane, flo
     w[0] += __shfl_xor_sync(0xffffffffu, w[0], 1);
     out = w[0];
     return idx;
+}
+
+// ------------------------------------------------------------------ inverse CDF in token order
+// "x ~ P" for non-negative weights P over the vocabulary, made deterministic by a supplied
+// uniform u: the smallest x with sum_{y<=x} P(y) > u * sum_y P(y); tokens of weight 0 are
+// never returned (Algorithm 1 / 2, "x_end ~ p"; Eq. 1 for the candidate draws).
+// The vocabulary is cut into contiguous runs, one per warp; a run into S steps of 32
+// groups (one group of 4 or 8 consecutive elements per lane).  Every lane keeps the float
+// sums g[S] of its own groups.  The search goes run -> step -> lane -> element; everything
+// above the lane level (run totals, their prefix sums, the position of the quantile inside
+// the run, the step totals' prefix sums) is carried in double, so that the only float
+// roundings left are inside one step (1/512 of the vocabulary or less).
+
+// Total of every step of this warp's run: lane st * (32 / S) holds the total of step st.
+template <int S>
+__device__ __forceinline__ float step_totals(const float (&g)[S], int lane) {
+    float tj;
+    warp_multi_sum<S>(g, lane, tj);
+    return tj;
+}
+// Total of the run: the step totals added in ascending order, in double (all lanes).
+template <int S>
+__device__ __forceinline__ double run_total(float tj) {
+    double r = 0.0;
+#pragma unroll
+    for (int st = 0; st < S; ++st) r += static_cast<double>(__shfl_sync(0xffffffffu, tj, st * (32 / S)));
+    return r;
+}
+// The run that holds the quantile u of the whole distribution.  m: total of run `lane`
+// (0 for lanes beyond the runs).  Every warp that calls this with the same totals finds the
+// same run.  Returns the run index, or -1 if the distribution has no mass (total 0 or NaN);
+// tgt receives the quantile's position inside the run.
+__device__ __forceinline__ int pick_run(double m, float u, int lane, double &tgt) {
+    double inc = m;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    const double total = __shfl_sync(0xffffffffu, inc, 31);
+    const double target = static_cast<double>(u) * total;
+    const unsigned hit = __ballot_sync(0xffffffffu, m > 0.0 && inc > target);
+    const unsigned pos = __ballot_sync(0xffffffffu, m > 0.0);
+    // (rounding, or u >= 1, may put the quantile past the end: the last run with mass)
+    const int pick = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
+    if (pick < 0 || !(total > 0.0)) return -1;
+    tgt = target - __shfl_sync(0xffffffffu, inc - m, pick);
+    return pick;
+}
+// Inside the run (called by the whole warp that owns it): the step ps and the lane l whose
+// group holds the quantile; rem (meaningful in lane l) is the quantile's position inside that
+// group.  False if the run has no mass.
+template <int S>
+__device__ __forceinline__ bool search_run(const float (&g)[S], float tj, double tgt, int lane,
+                                           int &ps, int &l, float &rem) {
+    ps = -1;
+    int last_s = -1;
+    double runsum = 0.0, before = 0.0;
+#pragma unroll
+    for (int st = 0; st < S; ++st) {
+        const float ms = __shfl_sync(0xffffffffu, tj, st * (32 / S));
+        if (ms > 0.f) {
+            last_s = st;
+            if (ps < 0 && runsum + static_cast<double>(ms) > tgt) { ps = st; before = runsum; }
+        }
+        runsum += static_cast<double>(ms);
+    }
+    float t2 = static_cast<float>(tgt - before);
+    if (ps < 0) { ps = last_s; t2 = INFINITY; }   // past the run's own sum: its last element with mass
+    if (ps < 0) return false;
+    float gs = g[0];
+#pragma unroll
+    for (int st = 1; st < S; ++st) gs = (ps == st) ? g[st] : gs;
+    const float gi = warp_scan_incl(gs, lane);
+    const unsigned h2 = __ballot_sync(0xffffffffu, gs > 0.f && gi > t2);
+    const unsigned p2 = __ballot_sync(0xffffffffu, gs > 0.f);
+    if (!p2) return false;
+    l = h2 ? __ffs(h2) - 1 : 31 - __clz(p2);
+    rem = t2 - (gi - gs);
+    return true;
+}
+// Inside one group: the first element whose running sum of positive weights exceeds rem,
+// else the last element with positive weight, else -1.
+template <int GV>
+__device__ __forceinline__ int pick_element(const float (&w)[GV], float rem) {
+    float acc = 0.f;
+    int pe = -1, last = -1;
+#pragma unroll
+    for (int e = 0; e < GV; ++e) {
+        if (w[e] > 0.f) {
+            acc += w[e];
+            last = e;
+            if (pe < 0 && acc > rem) pe = e;
+        }
+    }
+    return pe < 0 ? last : pe;
 }
 
 }  // namespace mcsd

@@ -11,14 +11,14 @@
 //                    the k candidates of the node are tested in order (Algorithm 1 /
 //                    Algorithm 2), so every logit row is read from HBM exactly once.
 //   argmax_kernel    (mcsd_argmax.cuh)  T == 0.  One CTA per target row; argmax with lowest
-//                    index on ties and the "candidate equals argmax" test (Section 4.4).
+//                    index on ties and the "candidate equals argmax" test (Section 4.5).
 //   walk_kernel      (mcsd_walk.cuh)  One row of CTAs per sequence: follows the accepted
 //                    children from the root (Section 3), writes the accepted tokens and the
 //                    endpoint token, and rebuilds the residual distribution of the
 //                    stopping node.
 //   sample_kernel    (mcsd_sample.cuh)  The k candidate draws of a node, with or without
 //                    replacement (Eq. 1).
-//   naive_kernel     (mcsd_naive.cuh)  The sample-and-match baseline of Section 4.3.
+//   naive_kernel     (mcsd_naive.cuh)  The sample-and-match baseline of Section 4.5.
 //   layout_kernel    (mcsd_layout.cuh)  Mask and position ids of the tree attention
 //                    (Section 3.3).
 //   gather_kernel    (mcsd_gather.cuh)  Key/value cache rows of the accepted path to their

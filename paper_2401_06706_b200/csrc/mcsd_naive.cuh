@@ -1,4 +1,4 @@
-// naive_kernel: the sample-and-match baseline of the ablation (Section 4.3), one CTA per sequence.
+// naive_kernel: the sample-and-match baseline of the ablation (Section 4.5), one CTA per sequence.
 #pragma once
 
 #include "mcsd_common.cuh"
@@ -23,7 +23,7 @@ struct NaiveParams {
     uint8_t child_count[MCSD_MAX_NODES];
 };
 
-// Multi-candidate naive sampling, the baseline that Section 4.4 and Appendix C compare
+// Multi-candidate naive sampling, the baseline that Section 4.5 and Appendix C compare
 // with: at the node the walk stands on, draw x from the target distribution (inverse CDF
 // with the node's second uniform); if a child carries x move to the first such child,
 // otherwise x is the endpoint token.  The draws depend on one another level by level and
@@ -37,7 +37,7 @@ naive_kernel(const __grid_constant__ NaiveParams P)
     constexpr int GV = E::kVec;
     constexpr int kStep = 32 * GV;
     constexpr int kMaxSteps = MCSD_MAX_VOCAB / kWalkWarps / kStep;
-    __shared__ float s_wtot[kWalkWarps];
+    __shared__ double s_wtot[kWalkWarps];
     __shared__ float s_red[kWalkWarps];
     __shared__ int s_pick, s_next;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -82,7 +82,6 @@ naive_kernel(const __grid_constant__ NaiveParams P)
         const float ref = int_ref(warp_max(s_red[lane]) * P.scale);
         ref0 = ref == -INFINITY ? 0.f : ref;
         float g[kMaxSteps];
-        float mass = 0.f;
 #pragma unroll
         for (int st = 0; st < kMaxSteps; ++st) {
             g[st] = 0.f;
@@ -92,67 +91,33 @@ naive_kernel(const __grid_constant__ NaiveParams P)
                 weights(x0, w);
 #pragma unroll
                 for (int e = 0; e < GV; ++e) g[st] += w[e];
-                mass += g[st];
             }
         }
-        mass = warp_sum(mass);
+        const float tj = step_totals<kMaxSteps>(g, lane);
+        const double mass = run_total<kMaxSteps>(tj);
         if (lane == 0) s_wtot[warp] = mass;
         if (tid == 0) s_pick = -1;
         __syncthreads();
         // the draw: run, step, lane, element
         const float u = P.unif[2 * (nb + n) + 1];
-        const float m = s_wtot[lane];
-        total = warp_sum(m);
-        const float target = u * total;
-        const float inc = warp_scan_incl(m, lane);
-        const unsigned hit = __ballot_sync(0xffffffffu, m > 0.f && inc > target);
-        const unsigned pos = __ballot_sync(0xffffffffu, m > 0.f);
-        const int pick = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
-        if (pick >= 0 && total > 0.f && warp == pick) {
-            const float tgt = target - __shfl_sync(0xffffffffu, inc - m, pick);
-            float tj;
-            warp_multi_sum<kMaxSteps>(g, lane, tj);
-            int ps = -1, last_s = -1;
-            float runsum = 0.f, ps_before = 0.f;
+        double tgt = 0.0;
+        const double m = s_wtot[lane];
+        const int pick = pick_run(m, u, lane, tgt);
+        {
+            double t = m;   // the row's mass, for the distribution written at the end
 #pragma unroll
-            for (int st = 0; st < kMaxSteps; ++st) {
-                const float ms = __shfl_sync(0xffffffffu, tj, st * (32 / kMaxSteps));
-                if (ms > 0.f) {
-                    last_s = st;
-                    if (ps < 0 && runsum + ms > tgt) { ps = st; ps_before = runsum; }
-                }
-                runsum += ms;
-            }
-            float t2 = tgt - ps_before;
-            if (ps < 0) { ps = last_s; t2 = INFINITY; }
-            if (ps >= 0) {
-                float gs = g[0];
-#pragma unroll
-                for (int st = 1; st < kMaxSteps; ++st) gs = (ps == st) ? g[st] : gs;
-                const float gi = warp_scan_incl(gs, lane);
-                const unsigned h2 = __ballot_sync(0xffffffffu, gs > 0.f && gi > t2);
-                const unsigned p2 = __ballot_sync(0xffffffffu, gs > 0.f);
-                if (p2) {
-                    const int l = h2 ? __ffs(h2) - 1 : 31 - __clz(p2);
-                    if (lane == l) {
-                        const int x0 = x_lo + ps * kStep + lane * GV;
-                        float w[GV];
-                        weights(x0, w);
-                        const float rem = t2 - (gi - gs);
-                        float acc = 0.f;
-                        int pe = -1, last = -1;
-#pragma unroll
-                        for (int e = 0; e < GV; ++e) {
-                            if (w[e] > 0.f) {
-                                acc += w[e];
-                                last = e;
-                                if (pe < 0 && acc > rem) pe = e;
-                            }
-                        }
-                        if (pe < 0) pe = last;
-                        if (pe >= 0) s_pick = x0 + pe;
-                    }
-                }
+            for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            total = static_cast<float>(t);
+        }
+        if (pick >= 0 && warp == pick) {
+            int ps, l;
+            float rem;
+            if (search_run<kMaxSteps>(g, tj, tgt, lane, ps, l, rem) && lane == l) {
+                const int x0 = x_lo + ps * kStep + lane * GV;
+                float w[GV];
+                weights(x0, w);
+                const int pe = pick_element<GV>(w, rem);
+                if (pe >= 0) s_pick = x0 + pe;
             }
         }
         __syncthreads();
@@ -185,7 +150,7 @@ naive_kernel(const __grid_constant__ NaiveParams P)
         if (P.out_path_nodes)
             for (int i = len; i <= P.gamma; ++i) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + i] = -1;
         P.out_accept_len[b] = len;
-        if (x < 0) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
+        P.status[b] = x < 0 ? MCSD_STATUS_NO_MASS : 0;   // written, not accumulated: nothing clears it beforehand
     }
     if (P.out_residual) {
         // the distribution the endpoint token was drawn from: the stopping node's p

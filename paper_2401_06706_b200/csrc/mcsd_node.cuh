@@ -27,6 +27,7 @@ struct Action {
     float c_try;   // c of the residual sum to form next
     int more;      // 1: form that sum and run another round; 0: the node is decided
     int accepted;  // path mode, with more == 0: the accepted child of the node, or -1
+    int poisoned;  // the leader's wait for this round expired: from here on the CTA's results are void
 };
 
 // Candidate data of the next items, fetched ahead of use by warp 0 so that no DRAM
@@ -126,6 +127,8 @@ node_kernel(const __grid_constant__ NodeParams P)
         return E::kBytes == 4 ? g0 + j * 32 : (j * H + h) * NT + tid;
     };
 
+    // the walk stage may be set up while this kernel runs; it waits for this kernel's results itself
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         mbar_init(full_addr, 1);
         mbar_init(xbar_addr(0), 1);
@@ -152,7 +155,10 @@ node_kernel(const __grid_constant__ NodeParams P)
     // lanes beyond the entry count.
     auto exchange_send = [&](float4 mine) {
         const uint32_t s = round & 1u;
-        if (tid == 0) mbar_arrive_expect_tx(xbar_addr(s), static_cast<uint32_t>(n_entries) * 16u);
+        // (once a wait has expired nothing is armed or sent any more: the barriers' phases no
+        // longer follow the rounds)
+        if (poisoned) return;
+        if (tid == 0) mbar_arrive_expect_tx(xbar_addr(s), static_cast<uint32_t>(n_entries) * 16u + P.test_extra_tx);
         if (lane < static_cast<int>(csize)) {
             const uint32_t dst = map_to_rank(smem_u32(&xch.slot[s][crank * NW + warp]), lane);
             st_async_f4(dst, mine, map_to_rank(xbar_addr(s), lane));
@@ -162,12 +168,13 @@ node_kernel(const __grid_constant__ NodeParams P)
     auto exchange_leader_wait = [&](float4 identity) -> float4 {
         const uint32_t s = round & 1u;
         // once a wait has expired the results are void and later rounds do not wait again
-        if (!poisoned && !mbar_wait(xbar_addr(s), (round >> 1) & 1u)) poisoned = 1;
+        if (!poisoned && !mbar_wait(xbar_addr(s), (round >> 1) & 1u, P.wait_polls)) poisoned = 1;
         return lane < n_entries ? xch.slot[s][lane] : identity;
     };
     // all warps: ends the round (the other warps have been waiting here for the leader)
     auto exchange_release = [&]() {
         __syncthreads();
+        poisoned |= act[round & 1u].poisoned;
         ++round;
     };
 
@@ -363,7 +370,7 @@ node_kernel(const __grid_constant__ NodeParams P)
             // (the walk kernel combines them) and goes on: no exchange, no barrier.
             const float st = warp_sum(zt);
             if (lane == 0)
-                P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * 32 +
+                P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * kLeafEntries +
                             crank * NW + warp] = make_float2(rt, st);
             if (crank == 0 && tid == 0) P.node_accept[node_idx] = -1;
             if (PATH) {  // the walk ends at this leaf: on to the cluster's next sequence
@@ -490,11 +497,14 @@ node_kernel(const __grid_constant__ NodeParams P)
         //
         // leader state of the rejection loop, in units where W' = W * K, K = Z_t * Z_d:
         double c = 0.0, S = 1.0, Wk = 0.0, K = 0.0, c_try = 0.0;
+        float c_prev = 0.f;  // c before the last rejection
         double px = 0.0, qx = 0.0;  // lane i of the leader: candidate i's p and q, times K
-        int cand_i = 0, attempt = 0, accepted = -1, my_tok = -1;
+        int cand_i = 0, accepted = -1, my_tok = -1;
         float u_acc = 2.f;
         // tests candidates from cand_i on until one is accepted (returns 0), all are rejected
-        // (returns 0) or one is rejected and its residual sum is needed (returns 1, c_try set)
+        // (returns 0) or one is rejected and its residual sum is needed (returns 1, c_try set).
+        // The sum after the LAST rejection is not needed here (nothing is tested against that
+        // residual): c moves on, the walk kernel forms the sum if a walk stops at this node.
         auto leader_decide = [&]() -> int {
             while (cand_i < k) {
                 const int i = cand_i;
@@ -519,7 +529,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                 c_try = c;
                 if (Wk > 0.0) c_try = (P.mode == 1) ? c + S * K / Wk : c + S;
                 if (P.mode == 1 && !zero_q) { Wk -= qxi; if (!(Wk > 0.0)) Wk = 0.0; }
-                attempt = 0;
+                if (i + 1 >= k) { c_prev = static_cast<float>(c); c = c_try; cand_i = k; return 0; }
                 return 1;
             }
             return 0;
@@ -540,7 +550,7 @@ node_kernel(const __grid_constant__ NodeParams P)
             bool cand_ok = false;
             if (lane < k) {
                 my_tok = ring.tok[s3][lane];
-                u_acc = ring.u[s3][lane];
+                u_acc = fminf(ring.u[s3][lane], 1.f);  // supplied in place of r ~ U(0,1): not below 1 (NaN too) counts as 1
                 cand_ok = my_tok >= 0 && my_tok < P.V;
                 if (cand_ok) {
                     const uint32_t wt = ring.tl[s2][lane], wd = ring.dl[s2][lane];
@@ -555,7 +565,10 @@ node_kernel(const __grid_constant__ NodeParams P)
             const float Z_d = warp_sum(ent.w * exp2i(ent.z - R_d));
             const bool t_ok = Z_t > 0.f && Z_t < INFINITY;  // false for an all -inf or NaN row
             const bool d_ok = Z_d > 0.f && Z_d < INFINITY;
-            if (!t_ok) status_bits |= MCSD_STATUS_NO_MASS;
+            // (a target row without mass: nothing can be accepted and a walk that stops here finds no
+            // token; a draft row without mass: nothing to test against, every candidate is rejected and
+            // p is kept; both count as a residual update that found no mass)
+            if (!t_ok || !d_ok) status_bits |= MCSD_STATUS_DEGENERATE;
             // candidates' probabilities, both multiplied by K so that no division is needed:
             // px' = 2^(l_t*scale - R_t) * Z_d, qx' = 2^(l_d*scale - R_d) * Z_t
             K = static_cast<double>(Z_t) * static_cast<double>(Z_d);
@@ -569,6 +582,7 @@ node_kernel(const __grid_constant__ NodeParams P)
                 act[round & 1u].stats = make_float4(R_t, R_d, t_ok ? 1.f / Z_t : 0.f, (t_ok && d_ok) ? Z_t / Z_d : 0.f);
                 act[round & 1u].c_try = static_cast<float>(c_try);
                 act[round & 1u].more = more;
+                act[round & 1u].poisoned = poisoned;
                 if (PATH) act[round & 1u].accepted = accepted;
                 if (crank == 0) *reinterpret_cast<float4 *>(&P.stats[node_idx]) = make_float4(R_t, R_d, Z_t, Z_d);
             }
@@ -610,20 +624,15 @@ node_kernel(const __grid_constant__ NodeParams P)
             if (warp == 0) {
                 const float4 ent = exchange_leader_wait(make_float4(0.f, 0.f, 0.f, 0.f));
                 const float S_new = warp_sum(ent.x);
-                int next;
-                if (S_new > 0.f) {
-                    if (attempt == 0) { c = c_try; S = static_cast<double>(S_new); }
-                    ++cand_i;
-                    next = leader_decide();
-                } else {
-                    // zero residual mass: keep the previous residual (recompute its sums once)
-                    status_bits |= MCSD_STATUS_DEGENERATE;
-                    if (attempt == 0) { attempt = 1; c_try = c; next = 1; }
-                    else { ++cand_i; next = leader_decide(); }
-                }
+                // zero residual mass: the previous residual, i.e. (c, S), is kept
+                if (S_new > 0.f) { c = c_try; S = static_cast<double>(S_new); }
+                else status_bits |= MCSD_STATUS_DEGENERATE;
+                ++cand_i;
+                const int next = leader_decide();
                 if (lane == 0) {
                     act[round & 1u].c_try = static_cast<float>(c_try);
                     act[round & 1u].more = next;
+                    act[round & 1u].poisoned = poisoned;
                     if (PATH) act[round & 1u].accepted = accepted;
                 }
             }
@@ -635,15 +644,14 @@ node_kernel(const __grid_constant__ NodeParams P)
         // ---- per-node results (the endpoint token is drawn by the walk kernel, and only
         // for the node where a walk stops)
         if (warp == 0) {
+            if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
+            status_bits = __reduce_or_sync(0xffffffffu, status_bits);
             if (crank == 0 && lane == 0) {
                 P.node_accept[node_idx] = accepted;
                 reinterpret_cast<float4 *>(&P.stats[node_idx])[1] =
-                    make_float4(static_cast<float>(c), static_cast<float>(S), 0.f, 0.f);
+                    make_float4(static_cast<float>(c), c_prev, __int_as_float(status_bits), 0.f);
             }
         }
-        if (poisoned) status_bits |= MCSD_STATUS_TIMEOUT;
-        status_bits = __reduce_or_sync(0xffffffffu, status_bits);
-        if (status_bits && lane == 0) atomicOr(P.status + b, status_bits);
         if (PATH) {
             // the walk goes on at the accepted child, or ends here
             const int acc = act[(round - 1u) & 1u].accepted;
@@ -655,6 +663,9 @@ node_kernel(const __grid_constant__ NodeParams P)
     }
 
     if (warp == kFetchWarp) cp_async_wait_all();
+    // After an expired wait the rounds were no longer waited for: give stores that peers issued
+    // before they noticed time to land (they take about a microsecond) before anybody leaves.
+    if (poisoned) __nanosleep(20000);
     // no CTA may leave while a peer can still write into its shared memory
     cluster_sync_all();
 }

@@ -46,7 +46,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
     // steps of a warp's run: CTAs of 1024 threads cover the largest vocabulary, smaller ones half of it
     constexpr int kMaxSteps = (NT == 1024 ? MCSD_MAX_VOCAB : MCSD_MAX_VOCAB / 2) / kW / kStep;
     static_assert(kMaxSteps <= 16, "the per-lane group sums are kept in registers");
-    __shared__ float s_wtot[32];
+    __shared__ double s_wtot[32];
     __shared__ float s_red[32];
     __shared__ int s_redi[32];
     __shared__ int32_t s_rem_tok[MCSD_MAX_CHILDREN];
@@ -234,15 +234,11 @@ sample_kernel(const __grid_constant__ SampleParams P)
     __syncthreads();
     const float ref = warp_max(lane < kW ? s_red[lane] : -INFINITY);
     float fb[NB];   // 2^(batch reference - row reference)
-    float mass = 0.f;
 #pragma unroll
     for (int bi = 0; bi < NB; ++bi) {
         fb[bi] = exp2i(rb[bi] - ref);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            g[bi * U + u] *= fb[bi];
-            mass += g[bi * U + u];
-        }
+        for (int u = 0; u < U; ++u) g[bi * U + u] *= fb[bi];
     }
     // the weights of one group again, bit for bit as they went into g (st: the group's step)
     auto weights = [&](int x0, int st, float *w) {
@@ -258,98 +254,60 @@ sample_kernel(const __grid_constant__ SampleParams P)
 #pragma unroll
         for (int e = 0; e < GV; ++e) w[e] = ex2f(fmaf(v[e], P.scale, -r0)) * f;
     };
-    mass = warp_sum(mass);
-    if (lane == 0) s_wtot[warp] = mass;
+    {
+        const double run_mass = run_total<kMaxSteps>(step_totals<kMaxSteps>(g, lane));
+        if (lane == 0) s_wtot[warp] = run_mass;
+    }
     __syncthreads();
 
     int n_rem = 0;  // tokens taken out so far (Eq. 1); the same in every thread
     for (int i = 0; i < k; ++i) {
         const float u = P.unif_draw[static_cast<long long>(b) * P.n_nodes + first + i];
         // the run that holds the quantile (every warp finds the same one)
-        const float m = lane < kW ? s_wtot[lane] : 0.f;
-        const float total = warp_sum(m);
-        const float target = u * total;
-        const float inc = warp_scan_incl(m, lane);
-        const unsigned hit = __ballot_sync(0xffffffffu, m > 0.f && inc > target);
-        const unsigned pos = __ballot_sync(0xffffffffu, m > 0.f);
-        const int pick = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
+        double tgt = 0.0;
+        const int pick = pick_run(lane < kW ? s_wtot[lane] : 0.0, u, lane, tgt);
         int found = -1;
-        if (pick >= 0 && total > 0.f && warp == pick) {
-            const float tgt = target - __shfl_sync(0xffffffffu, inc - m, pick);
-            float tj;
-            warp_multi_sum<kMaxSteps>(g, lane, tj);
-            int ps = -1, last_s = -1;
-            float runsum = 0.f, ps_before = 0.f;
+        double new_mass = -1.0;   // (Eq. 1) what is left of this warp's run after the draw
+        if (pick >= 0 && warp == pick) {
+            const float tj = step_totals<kMaxSteps>(g, lane);
+            int ps, l;
+            float rem;
+            if (search_run<kMaxSteps>(g, tj, tgt, lane, ps, l, rem)) {
+                int pe = -1;
+                if (lane == l) {
+                    const int x0 = x_lo + ps * kStep + lane * GV;
+                    float w[GV];
+                    weights(x0, ps, w);
+                    // tokens drawn before (Eq. 1) have left the distribution
+                    for (int j = 0; j < n_rem; ++j) {
+                        const int gone = s_rem_tok[j] - x0;
 #pragma unroll
-            for (int st = 0; st < kMaxSteps; ++st) {
-                const float ms = __shfl_sync(0xffffffffu, tj, st * (32 / kMaxSteps));
-                if (ms > 0.f) {
-                    last_s = st;
-                    if (ps < 0 && runsum + ms > tgt) { ps = st; ps_before = runsum; }
-                }
-                runsum += ms;
-            }
-            float t2 = tgt - ps_before;
-            if (ps < 0) { ps = last_s; t2 = INFINITY; }   // rounding: take the run's last element with mass
-            if (ps >= 0) {
-                float gs = g[0];
-#pragma unroll
-                for (int st = 1; st < kMaxSteps; ++st) gs = (ps == st) ? g[st] : gs;
-                const float gi = warp_scan_incl(gs, lane);
-                const unsigned h2 = __ballot_sync(0xffffffffu, gs > 0.f && gi > t2);
-                const unsigned p2 = __ballot_sync(0xffffffffu, gs > 0.f);
-                if (p2) {
-                    const int l = h2 ? __ffs(h2) - 1 : 31 - __clz(p2);
-                    int pe = -1, last = -1;
-                    if (lane == l) {
-                        const int x0 = x_lo + ps * kStep + lane * GV;
-                        float w[GV];
-                        weights(x0, ps, w);
-                        const float rem = t2 - (gi - gs);
-                        float acc = 0.f;
-#pragma unroll
-                        for (int e = 0; e < GV; ++e) {
-                            bool gone = false;
-                            for (int j = 0; j < n_rem; ++j) gone |= s_rem_tok[j] == x0 + e;
-                            if (!gone && w[e] > 0.f) {
-                                acc += w[e];
-                                last = e;
-                                if (pe < 0 && acc > rem) pe = e;
-                            }
-                        }
-                        if (pe < 0) pe = last;
-                        if (pe >= 0 && P.mode == 1) {
-                            // Eq. 1: the drawn token leaves the distribution.  The group's sum is
-                            // formed again from the tokens that remain (subtracting would lose
-                            // everything when the drawn token dominated the group)
-                            float rest = 0.f;
-#pragma unroll
-                            for (int e = 0; e < GV; ++e) {
-                                bool gone = e == pe;
-                                for (int j = 0; j < n_rem; ++j) gone |= s_rem_tok[j] == x0 + e;
-                                if (!gone) rest += w[e];
-                            }
-#pragma unroll
-                            for (int st = 0; st < kMaxSteps; ++st)
-                                if (st == ps) g[st] = rest;
-                        }
+                        for (int e = 0; e < GV; ++e) w[e] = (gone == e) ? 0.f : w[e];
                     }
-                    found = __shfl_sync(0xffffffffu, pe < 0 ? -1 : x_lo + ps * kStep + lane * GV + pe, l);
-                    if (P.mode == 1 && found >= 0) {
-                        // ... and so is the run's total, from the lanes' current group sums
-                        float rs = 0.f;
+                    pe = pick_element<GV>(w, rem);
+                    if (pe >= 0 && P.mode == 1) {
+                        // ... and so does this one: the group's sum is formed again from the
+                        // tokens that remain (subtracting would lose everything when the drawn
+                        // token dominated the group)
+                        float rest = 0.f;
 #pragma unroll
-                        for (int st = 0; st < kMaxSteps; ++st) rs += g[st];
-                        rs = warp_sum(rs);
-                        if (lane == 0) s_wtot[warp] = rs;
+                        for (int e = 0; e < GV; ++e) rest += (e == pe) ? 0.f : w[e];
+#pragma unroll
+                        for (int st = 0; st < kMaxSteps; ++st)
+                            if (st == ps) g[st] = rest;
                     }
                 }
+                found = __shfl_sync(0xffffffffu, pe < 0 ? -1 : x_lo + ps * kStep + lane * GV + pe, l);
+                // ... and the run's total, from the lanes' current group sums
+                if (P.mode == 1 && found >= 0) new_mass = run_total<kMaxSteps>(step_totals<kMaxSteps>(g, lane));
             }
             if (lane == 0) s_pick = found;
         }
-        if (pick < 0 || !(total > 0.f)) { if (tid == 0) s_pick = -1; }
+        if (pick < 0) { if (tid == 0) s_pick = -1; }
         __syncthreads();
         found = s_pick;
+        // (written only now: until the barrier above other warps may still have been reading the totals)
+        if (new_mass >= 0.0 && lane == 0) s_wtot[warp] = new_mass;
         if (tid == 0) {
             out[i] = found;
             if (found < 0 && P.status) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);

@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(lib):
     assert set(names) == set(binding.EXPORTS)
     for name in names:
         assert getattr(lib, name) is not None
-    assert lib.mcsd_version() == 101
+    assert lib.mcsd_version() == 102
 
 
 def test_header_constants_match_binding():
@@ -40,6 +40,23 @@ def test_header_constants_match_binding():
     assert int(consts["MCSD_MAX_VOCAB"]) == binding.MAX_VOCAB
     assert int(consts["MCSD_STATUS_TIMEOUT"]) == binding.STATUS_TIMEOUT
     assert int(consts["MCSD_DTYPE_BF16"]) == 1 and int(consts["MCSD_DTYPE_F16"]) == 2
+    for name in ("CLUSTER", "EPT", "DIRECT", "SAMPLE_AHEAD", "WAIT_POLLS", "TEST_EXTRA_TX", "PDL"):
+        assert int(consts["MCSD_OPT_" + name]) == getattr(binding, "OPT_" + name)
+
+
+def test_options_are_set_read_back_and_validated(lib):
+    n = int(re.search(r"#define\s+MCSD_OPT_COUNT\s+(\d+)", open(os.path.join(ROOT, "include", "mcsd.h")).read()).group(1))
+    before = [binding.mcsd_get_option(i) for i in range(n)]
+    try:
+        for i in range(n):
+            binding.mcsd_set_option(i, 3)
+            assert binding.mcsd_get_option(i) == 3
+        for bad in (-1, n, 99):
+            assert lib.mcsd_set_option(bad, 1) == -2 and lib.mcsd_get_option(bad) == -2
+        assert lib.mcsd_set_option(0, -5) == -2
+    finally:
+        for i, val in enumerate(before):
+            binding.mcsd_set_option(i, val)
 
 
 def test_tree_depth_and_contract(lib):
@@ -105,6 +122,8 @@ def test_host_validation_codes(lib):
     assert call(d2, parent) == -3
     d2, _ = _desc(ws=ws); d2.vocab = 0
     assert call(d2, parent) == -2
+    d2, _ = _desc(ws=ws); d2.reserved = 1
+    assert call(d2, parent) == -2
     d2, _ = _desc(ws=ws); d2.vocab = 70000; d2.ld_target = d2.ld_draft = 70000
     assert call(d2, parent) == -10
     d2, _ = _desc(ws=ws); d2.ld_target = 63
@@ -117,7 +136,7 @@ def test_host_validation_codes(lib):
     d2, _ = _desc(); assert call(d2, parent) == -8                     # no workspace
     d2, _ = _desc(ws=(0x10000, 16)); assert call(d2, parent) == -8     # too small
     d2, _ = _desc(ws=(0x10010, 1 << 20)); assert call(d2, parent) == -8  # misaligned
-    for code in range(-10, 1):
+    for code in range(-11, 1):
         assert len(binding.status_string(code)) > 0
     assert binding.status_string(-99) == "unknown code"
 

@@ -28,6 +28,7 @@ def test_mask_and_positions(kconfig):
 @pytest.mark.parametrize("entry,mode,T", [("mcsd_verify", 0, 1.0), ("mcsd_verify", 1, 0.7), ("mcsd_verify_path", 1, 1.0),
                                           ("mcsd_verify", 2, 1.0), ("mcsd_verify", 0, 0.0)])
 def test_accepted_path_nodes(entry, mode, T):
+    from oracle import compare as cmp
     w = synth.Workload("pathnodes", 48, 5000, "4x2x2x1", "fp32", "normal", 2.5, 1.0, 0.7, T, min(mode, 1), 77)
     inp = synth.make_inputs(w, "cuda")
     v = binding.Verifier(w.batch, inp.parent, w.vocab, torch.float32, "cuda")
@@ -36,12 +37,18 @@ def test_accepted_path_nodes(entry, mode, T):
     t, d, c, u = inp.host_f32()
     ref = oracle.verify(t, d if (T > 0 and mode != 2) else None, inp.parent, c, u, T, mode)
     want = oracle.path_nodes(ref, inp.stats["gamma"])
-    same = out.accept_len.cpu().numpy() == ref.accept_len        # (sequences with a near-tie flip would differ)
-    assert same.mean() > 0.95
-    assert np.array_equal(out.path_nodes.cpu().numpy()[same], want[same])
-    # the tokens on the path are the tokens of those nodes
     pn = out.path_nodes.cpu().numpy()
     tok = out.tokens.cpu().numpy()
+    # the comparison rule: a walk may leave the oracle's only at a test inside the near-tie band
+    # (naive sampling: at a draw inside the boundary tolerance); every other sequence is exact
+    rep = cmp.compare(t, d, inp.parent, c, u, T, mode, "fp32", oracle_result=ref, accept_len=out.accept_len.cpu().numpy(),
+                      tokens=tok, residual=out.residual.cpu().numpy(), status=out.status.cpu().numpy(), path_nodes=pn)
+    assert rep.ok, rep.failures[:5]
+    keep = np.ones(w.batch, dtype=bool)
+    keep[rep.excluded] = False
+    assert keep.sum() >= w.batch - 2
+    assert np.array_equal(pn[keep], want[keep])
+    # the tokens on the path are the tokens of those nodes
     for b in range(w.batch):
         L = int(out.accept_len[b])
         assert (pn[b, L:] == -1).all() and (c[b, pn[b, :L]] == tok[b, :L]).all()

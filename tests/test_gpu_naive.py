@@ -1,4 +1,4 @@
-"""MCSD_MODE_NAIVE (multi-candidate naive sampling, the ablation baseline of Section 4.4) against
+"""MCSD_MODE_NAIVE (multi-candidate naive sampling, the ablation baseline of Section 4.5) against
 the oracle's mode 2 on the same seeded inputs: accepted lengths and tokens identical except where
 the draw's uniform lies within 1e-5 (CDF units) of an interval boundary, residual within the
 parity tolerance."""

@@ -9,7 +9,7 @@ import pytest
 import torch
 
 from paper_2401_06706_b200 import binding, synth
-from gpu_util import assert_parity, run_library, to_np
+from gpu_util import assert_parity, library_options, run_library, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -99,25 +99,25 @@ def test_aligned_rows_whose_vocabulary_ends_inside_a_vector(dtype, vocab, T):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-@pytest.mark.parametrize("cluster,ept", [(1, 64), (2, 16), (4, 16), (8, 16), (8, 32), (2, 64), (4, 32)])
-def test_forced_cluster_shapes(cluster, ept, dtype, monkeypatch):
-    """Every cluster size / per-thread share computes the same thing (128 threads per CTA)."""
-    monkeypatch.setenv("MCSD_CLUSTER", str(cluster))
-    monkeypatch.setenv("MCSD_EPT", str(ept))
+@pytest.mark.parametrize("cluster,ept", [(1, 64), (2, 16), (4, 16), (8, 16), (8, 32), (2, 64), (4, 32), (3, 16), (7, 32)])
+def test_forced_cluster_shapes(cluster, ept, dtype):
+    """Every cluster size / per-thread share computes the same thing (128 threads per CTA; with the
+    larger shapes some CTAs of the cluster own nothing but -inf)."""
     vocab = min(cluster * ept * 128 - 24, 9000)
     w = synth.Workload("forced", 6, vocab, "4x2x1", dtype, "normal", 2.5, 1.0, 1.0, 1.0, 1, 31 + cluster + ept)
     inp = synth.make_inputs(w, "cuda")
-    _, out = run_library(inp)
+    with library_options(cluster=cluster, ept=ept):
+        _, out = run_library(inp)
     assert_parity(inp, out)
 
 
-def test_direct_path_matches_bulk_copy_path(monkeypatch):
+def test_direct_path_matches_bulk_copy_path():
     w = synth.Workload("direct", 6, 32000, "4x2", "bf16", "normal", 2.5, 0.8, 1.5, 1.0, 0, 99)
     inp = synth.make_inputs(w, "cuda")
     _, a = run_library(inp)
     a_acc, a_bon, a_res = to_np(a.node_accept), to_np(a.node_bonus), to_np(a.residual)
-    monkeypatch.setenv("MCSD_DIRECT", "1")
-    _, b = run_library(inp)
+    with library_options(direct=1):
+        _, b = run_library(inp)
     assert np.array_equal(a_acc, to_np(b.node_accept)) and np.array_equal(a_bon, to_np(b.node_bonus))
     assert np.array_equal(a_res, to_np(b.residual))
     assert_parity(inp, b)
@@ -168,7 +168,7 @@ def test_degenerate_inputs_set_status_and_never_hang():
     _, out = run_library(inp)
     rep = assert_parity(inp, out)
     st = to_np(out.status)
-    assert st[0] & binding.STATUS_BAD_TOKEN
+    assert st[0] & binding.STATUS_BAD_TOKEN       # the root is on every walk
     assert not (st & binding.STATUS_TIMEOUT).any()
 
 
@@ -196,6 +196,7 @@ def test_staged_entry_points_equal_the_fused_call():
     torch.cuda.synchronize()
     assert np.array_equal(ref[0], to_np(o2.accept_len)) and np.array_equal(ref[1], to_np(o2.tokens))
     assert np.array_equal(ref[2], to_np(o2.residual))
+    assert np.array_equal(to_np(out.status), to_np(o2.status))
     assert binding.mcsd_last_launch_count() == 1
 
 
@@ -238,15 +239,33 @@ def test_sweep_points_sampled(idx):
     assert_parity(inp, out, 0, min(16, w.batch))
 
 
+def _parity_in_chunks(inp, out, chunk=64, **kw):
+    """Oracle parity on every sequence, a chunk at a time (the float32 host copies of 512 sequences
+    would be 19.5 GB at once); the near-tie share is judged on the totals."""
+    from oracle import compare as cmp
+    w = inp.workload
+    tests = near = flipped = tolerated = draws = 0
+    for b0 in range(0, w.batch, chunk):
+        rep = assert_parity(inp, out, b0, min(w.batch, b0 + chunk), **kw)
+        tests += rep.n_tests; near += rep.n_near_tie; flipped += rep.n_flipped
+        tolerated += rep.n_bonus_tolerated; draws += rep.n_bonus_draws
+    assert near <= max(cmp.NEAR_TIE_MIN_EVENTS, cmp.NEAR_TIE_SHARE * tests), (near, tests)
+    assert tolerated <= cmp.boundary_draw_limit(w.vocab, draws), (tolerated, draws)
+    return {"tests": tests, "near_ties": near, "flipped": flipped, "bonus_tolerated": tolerated, "bonus_draws": draws}
+
+
 @pytest.mark.skipif(os.environ.get("MCSD_SKIP_LARGE") == "1", reason="large case disabled")
-def test_largest_configuration_sampled_parity_and_properties():
-    """B = 512, 4x4x2x2x1, fp32 (19.5 GB of logits), in the launch shape the bench times: oracle
-    parity on sampled sequences, structural properties on all of them."""
-    w = NAMED["cfg5_largest"]
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_largest_configuration_full_parity_and_properties(dtype):
+    """B = 512, 4x4x2x2x1, V = 32000 (19.5 GB of fp32 logits), in the launch shape the bench times:
+    oracle parity on ALL 512 sequences, node by node, plus structural properties."""
+    from dataclasses import replace
+    w = replace(NAMED["cfg5_largest"], dtype=dtype)
     inp = synth.make_inputs(w, "cuda")
     _, out = run_library(inp)
-    for b0 in (0, 255, 500):
-        assert_parity(inp, out, b0, b0 + 6)
+    totals = _parity_in_chunks(inp, out)
+    print(dtype, totals)
+    assert totals["tests"] > 60000
     acc, bon = to_np(out.node_accept), to_np(out.node_bonus)
     tok, ln = to_np(out.tokens), to_np(out.accept_len)
     first, count = synth.children_ranges(inp.parent)
@@ -334,7 +353,7 @@ def test_largest_configuration_path_form_and_sampler(dtype):
     assert torch.equal(a_len, b.accept_len) and torch.equal(a_tok, b.tokens) and torch.equal(a_st, b.status)
     assert torch.equal(a_res, b.residual)
     for b0 in (0, 300, 506):
-        assert_parity(inp, b, b0, b0 + 6)
+        assert_parity(inp, b, b0, b0 + 6, sequential=True)
     # sampler
     gen = torch.Generator(device="cuda")
     gen.manual_seed(99)
@@ -351,5 +370,4 @@ def test_largest_configuration_path_form_and_sampler(dtype):
         sl = slice(b0, b0 + 4)
         rep = cmp.compare_samples(inp.draft[sl].to(torch.float32).cpu().numpy(), inp.parent, u[sl].cpu().numpy(), 1.0, 1,
                                   c[sl], 0, None)
-        assert rep.ok, rep.failures[:5]
-        assert rep.n_tolerated <= max(3, 1e-6 * w.vocab * rep.n_draws)
+        assert rep.ok, rep.failures[:5]       # (includes the bound on draws that differ inside the tolerance)

@@ -55,6 +55,19 @@ def test_all_candidates_rejected_on_zero_mass_draws_from_the_kept_p(mode):
         assert np.allclose(res.residual[0], [0.125, 0.5, 0.25, 0.125], rtol=1e-7)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_zero_residual_mass_on_a_long_row_whose_sum_is_not_exactly_one(mode):
+    """The same with a softmax over 4000 logits, whose float64 sum is 1 only up to rounding: two
+    candidates that are not tokens leave p and q bit for bit as they were (Algorithm 2 removes
+    nothing from q, so it does not renormalise it either)."""
+    rng = np.random.default_rng(31)
+    p = oracle.softmax((rng.standard_normal(4000) * 2.5).astype(np.float32), 1.0)
+    r = oracle.mcss(p, p.copy(), [4000, -1], [0.5, 0.5], mode)
+    assert r.accepted == -1 and r.status == (DEGENERATE | BAD_TOKEN)
+    assert np.array_equal(r.p, p) and np.array_equal(r.q, p)
+    assert r.S[0] == 0.0 and r.S[1] == 0.0
+
+
 # ------------------------------------------------------------------ no mass
 @pytest.mark.parametrize("bad", ["all_minus_inf", "nan", "plus_inf"])
 @pytest.mark.parametrize("mode", [0, 1, 2])

@@ -1,4 +1,4 @@
-"""Pins of the oracle's naive-sampling mode (mode 2; the baseline of Section 2 that Section 4.4
+"""Pins of the oracle's naive-sampling mode (mode 2; the baseline of Section 2 that Section 4.5
 and Appendix C compare multi-candidate speculative sampling with): the emitted token is a draw
 from p whatever the candidates are, it is accepted exactly when a candidate carries it, and
 averaged over candidates drawn from q its rejection probability is sum_x p(x)(1-q(x))^k, which

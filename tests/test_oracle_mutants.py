@@ -22,11 +22,11 @@ MUTANTS = [
      [pins.test_k1_is_textbook_speculative_sampling]),
     ("residual_not_normalised", "p[x] = (d > 0.0 ? d : 0.0) / s;", "p[x] = (d > 0.0 ? d : 0.0);",
      [lambda: pins.test_output_token_is_distributed_as_p(4, 3, 0)]),
-    ("alg2_q_not_zeroed", "if (valid) q[xt] = 0.0;", ";",
+    ("alg2_q_not_zeroed", "            q[xt] = 0.0;\n            double w = 0.0;", "            double w = 0.0;",
      [lambda: pins.test_output_token_is_distributed_as_p(4, 3, 1)]),
     ("alg2_q_not_renormalised", "for (int32_t x = 0; x < V; ++x) q[x] /= w;", ";",
      [lambda: pins.test_output_token_is_distributed_as_p(4, 3, 1)]),
-    ("alg2_applied_to_alg1", "if (mode == 1) {", "if (mode == 0) {",
+    ("alg2_applied_to_alg1", "if (mode == 1 && valid && q[xt] > 0.0) {", "if (mode == 0 && valid && q[xt] > 0.0) {",
      [lambda: pins.test_rejection_probability_is_the_normaliser_and_rejected_tokens_stay_zero(0)]),
     ("zero_q_accepted", "if (qx > 0.0) {", "if (qx >= 0.0) {",
      [pins.test_forced_rejection_on_zero_draft_probability]),
@@ -91,8 +91,8 @@ MUTANTS = [
      [lambda: epins.test_target_row_without_mass_at_the_root("plus_inf", 2)]),
     ("uniform_cap_missing", "if (!(r[i] < 1.0)) r[i] = 1.0;", ";",
      [epins.test_uniform_not_below_one_counts_as_one]),
-    ("draft_without_mass_falls_through", "if (qbuf[0] != qbuf[0]) {", "if (0) {",
-     [lambda: epins.test_draft_row_without_mass_rejects_everything_and_draws_from_p(1)]),
+    ("alg2_renormalises_when_nothing_was_removed", "if (mode == 1 && valid && q[xt] > 0.0) {", "if (mode == 1) { if (!valid) xt = 0;",
+     [lambda: epins.test_zero_residual_mass_on_a_long_row_whose_sum_is_not_exactly_one(1)]),
 ]
 
 

@@ -308,7 +308,7 @@ def test_forced_rejection_on_zero_draft_probability():
 
 # ---------------------------------------------------------------- temperature 0
 def test_temperature_zero_is_greedy_matching():
-    """Section 4.4: at temperature 0 acceptance means 'candidate equals the target argmax';
+    """Section 4.5: at temperature 0 acceptance means 'candidate equals the target argmax';
     the endpoint is the target argmax of the stopping node; draft logits are unused."""
     rng = np.random.default_rng(19)
     ks = [3, 2, 1]

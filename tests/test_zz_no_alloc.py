@@ -6,26 +6,41 @@ allocation, a process whose device memory is already handed out.  They cannot su
 scratch buffer that mcsd_verify expects in its descriptor, so mcsd_verify_static keeps that
 scratch in an array compiled into the library.  This file checks, through the C ABI, that
 
-  * the call gives exactly what mcsd_verify gives on the same inputs,
+  * the call gives bit for bit what mcsd_verify gives on the same inputs (both run the same
+    kernels) and agrees with the CPU oracle,
   * a second call right after it, on other inputs, is not disturbed by what the first one
     left in the shared array,
+  * the call really allocates nothing: the device's free memory is the same before and after,
+  * it also works when the caller passes no status buffer (the status words then live in the
+    built-in array),
   * a job whose scratch need exceeds the built-in array is turned away with the dedicated
     error code and nothing is enqueued.
 
 The file name sorts last on purpose: with `pytest -x` every other test has run before this one.
 """
 import ctypes
+import os
+import re
 
 import numpy as np
 import pytest
 import torch
 
 from paper_2401_06706_b200 import binding, synth
+from gpu_util import assert_parity
 
 pytestmark = pytest.mark.gpu
 
-STATIC_BYTES = 4 << 20
-ERR_STATIC_LIMIT = -11
+
+def _header_constant(name):
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    text = open(os.path.join(root, "include", "mcsd.h")).read()
+    m = re.search(r"#define\s+" + name + r"\s+\(?\(?(-?\d+)u?\s*(?:<<\s*(\d+))?\)?", text)
+    return int(m.group(1)) << int(m.group(2) or 0)
+
+
+STATIC_BYTES = _header_constant("MCSD_STATIC_WORKSPACE_BYTES")
+ERR_STATIC_LIMIT = _header_constant("MCSD_ERR_STATIC_LIMIT")
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -46,46 +61,75 @@ def _both_ways(w):
     other = binding.Verifier(w.batch, inp.parent, w.vocab, dt, "cuda")
     other.desc.workspace = None
     other.desc.workspace_bytes = 0
+    other.mcsd_verify_static(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)   # first call on the device: address lookup
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     b = other.mcsd_verify_static(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
     torch.cuda.synchronize()
-    return a, b
+    assert torch.cuda.mem_get_info()[0] == free_before, "mcsd_verify_static changed the device's free memory"
+    return inp, a, b
 
 
-def _same(a, b, tol):
+def _same(inp, a, b):
+    # the two entry points run the same kernels on the same inputs: every output bit agrees
     assert torch.equal(a.accept_len, b.accept_len)
     assert torch.equal(a.tokens, b.tokens)
     assert torch.equal(a.status, b.status)
-    err = float((a.residual - b.residual).abs().max())
-    assert err <= tol, err
+    assert torch.equal(a.path_nodes, b.path_nodes)
+    assert torch.equal(a.residual.view(torch.int32), b.residual.view(torch.int32))
+    # ... and the new entry point agrees with the oracle directly, under the parity tolerances
+    assert_parity(inp, b)
 
 
 def test_static_scratch_matches_caller_scratch_on_two_calls_in_a_row():
-    # residual tolerances of the parity tests: 1e-5 for fp32 logits, 2e-3 for 2-byte logits
     first = synth.Workload("static_a", 8, 32000, "4x2x2x1", "bf16", "normal", 2.5, 0.8, 1.5, 1.0, 1, 9001)
     second = synth.Workload("static_b", 5, 5000, "2x2", "fp32", "normal", 2.5, 1.0, 1.0, 0.8, 0, 9002)
-    _same(*_both_ways(first), 2e-3)
-    _same(*_both_ways(second), 1e-5)
+    _same(*_both_ways(first))
+    _same(*_both_ways(second))
     # and the first one again, now that the array holds the second job's leftovers
-    _same(*_both_ways(first), 2e-3)
+    _same(*_both_ways(first))
 
 
 def test_static_scratch_at_temperature_zero():
     w = synth.Workload("static_t0", 6, 4096, "4x2", "fp16", "normal", 3.0, 1.0, 2.0, 0.0, 0, 9003)
-    _same(*_both_ways(w), 0.0)
+    _same(*_both_ways(w))
+
+
+def test_status_words_inside_the_built_in_array():
+    """A caller that passes no status buffer: the status words live in the built-in array; the
+    other outputs are what the call with a status buffer gives."""
+    w = synth.Workload("static_nostatus", 7, 6000, "3x2", "fp32", "normal", 2.5, 1.0, 1.0, 1.0, 1, 9004)
+    inp = synth.make_inputs(w, "cuda")
+    a = binding.Verifier(w.batch, inp.parent, w.vocab, torch.float32, "cuda")
+    ra = a.mcsd_verify_static(inp.target, inp.draft, inp.cand, inp.unif, 1.0, 1)
+    torch.cuda.synchronize()
+    b = binding.Verifier(w.batch, inp.parent, w.vocab, torch.float32, "cuda")
+    b.desc.out_status = None
+    b.desc.workspace = None
+    b.desc.workspace_bytes = 0
+    rb = b.mcsd_verify_static(inp.target, inp.draft, inp.cand, inp.unif, 1.0, 1)
+    torch.cuda.synchronize()
+    assert torch.equal(ra.accept_len, rb.accept_len) and torch.equal(ra.tokens, rb.tokens)
+    assert torch.equal(ra.residual, rb.residual)
 
 
 def test_job_beyond_the_built_in_array_is_rejected():
+    """A tiny vocabulary with many nodes: the scratch need is beyond the array while every
+    input and output buffer exists at full size, so even a call that was wrongly let through
+    would stay inside its buffers."""
     lib = binding.load_library()
-    parent = synth.tree_from_kconfig([4, 4, 2, 2, 1])
-    st = synth.tree_stats(parent)
-    d = binding.McsdDesc()
-    d.batch, d.n_nodes, d.n_internal, d.vocab = 512, st["n_nodes"], st["n_internal"], 32000
-    d.dtype, d.ld_target, d.ld_draft = 0, 32000, 32000
-    assert lib.mcsd_workspace_bytes(ctypes.byref(d)) > STATIC_BYTES
-    # validation comes before any pointer is touched, so dummy non-null pointers are enough
-    one = torch.zeros(4, dtype=torch.int32, device="cuda")
-    rc = lib.mcsd_verify_static(ctypes.byref(d), one.data_ptr(), one.data_ptr(), parent.ctypes.data,
-                                one.data_ptr(), one.data_ptr(), 1.0, 0, one.data_ptr(), one.data_ptr(), None)
-    assert rc == ERR_STATIC_LIMIT
-    assert "mcsd_verify_static" in binding.status_string(rc)
+    w = synth.Workload("static_big", 2048, 8, "4x4x2x2x1", "fp32", "normal", 2.5, 1.0, 1.0, 1.0, 0, 9005)
+    inp = synth.make_inputs(w, "cuda")
+    v = binding.Verifier(w.batch, inp.parent, w.vocab, torch.float32, "cuda")
+    assert lib.mcsd_workspace_bytes(ctypes.byref(v.desc)) > STATIC_BYTES
+    v.tokens.fill_(-77)
+    with pytest.raises(binding.McsdError) as e:
+        v.mcsd_verify_static(inp.target, inp.draft, inp.cand, inp.unif, 1.0, 0)
+    assert e.value.code == ERR_STATIC_LIMIT
+    assert "mcsd_verify_static" in binding.status_string(e.value.code)
     torch.cuda.synchronize()
+    assert bool((v.tokens == -77).all())          # nothing was enqueued
+    # the same job is fine with caller-owned scratch
+    out = v.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, 1.0, 0)
+    torch.cuda.synchronize()
+    assert bool((out.tokens[:, 0] >= 0).all())
