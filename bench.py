@@ -3,6 +3,8 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
+With --gpus N > 1 and no torchrun around it the script starts its own N ranks (one per GPU).
+
 A step is one pass of the whole hot path (per-node softmax statistics, rejection loop,
 endpoint tokens, tree walk, terminal residual) over one batch of synthetic trees whose
 logits are already resident in HBM.  The default workload is the largest point of the
@@ -46,18 +48,23 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+TRAFFIC_PROFILE = os.path.join("profiles", "node_kernel_cfg5_batch16_ncu_full.md")
+
+
 def recorded_traffic(units: int):
     """DRAM bytes per launch of the node kernel from the committed ncu summary, scaled by the
     number of tree nodes per launch (the capture ran a smaller batch of the same workload and
-    the traffic grows in proportion to the rows read)."""
+    the traffic grows in proportion to the rows read).  Returns (bytes, source, scale factor);
+    bytes is None when the summary is missing."""
     import re
-    path = os.path.join(ROOT, "profiles", "node_kernel_cfg5_batch16_ncu_full.md")
     try:
-        with open(path) as f:
+        with open(os.path.join(ROOT, TRAFFIC_PROFILE)) as f:
             m = re.search(r"dram_bytes_per_launch=(\d+) units_per_launch=(\d+)", f.read())
-        return float(m.group(1)) * units / float(m.group(2))
+        scale = units / float(m.group(2))
+        return float(m.group(1)) * scale, (f"{TRAFFIC_PROFILE}: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture "
+                                            f"at {m.group(2)} tree nodes per launch, scaled by the nodes per launch"), scale
     except Exception:
-        return None
+        return None, "no recorded capture", None
 
 
 class ClockSampler:
@@ -110,6 +117,28 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def spawn_command(argv, n: int, port: int):
+    """The command that starts n ranks of this script on one node (what a plain
+    `python bench.py --gpus n` runs when no launcher is around it)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def spawn_ranks(args):
+    """--gpus N > 1 without a launcher: start N ranks (one process per GPU) and pass their output on.
+    NCCL's log is switched on (to files, so that stdout stays the one JSON line)."""
+    if args.impl != "reference" and torch.cuda.device_count() < args.gpus:
+        raise SystemExit(f"--gpus {args.gpus}: only {torch.cuda.device_count()} CUDA devices are visible")
+    env = dict(os.environ)
+    if "NCCL_DEBUG" not in env:
+        env["NCCL_DEBUG"] = "INFO"
+        env["NCCL_DEBUG_FILE"] = os.path.join(env.get("TMPDIR", "/tmp"), "mcsd_bench_nccl.%h.%p.log")
+    if args.impl == "reference":     # only rank 0 works there: it may use every core
+        env.setdefault("OMP_NUM_THREADS", str(os.cpu_count() or 1))
+    port = 29500 + os.getpid() % 2000
+    return subprocess.call(spawn_command(sys.argv[1:], args.gpus, port), env=env)
 
 
 def dist_env():
@@ -167,9 +196,18 @@ def oracle_sample(inp: synth.Inputs, n_seq: int):
     res = oracle.verify(t, d if w.temperature > 0 else None, inp.parent, c, u, w.temperature, w.mode)
     dt = time.perf_counter() - t0
     nodes = n_seq * inp.stats["n_draft"]
+    # the same oracle on one thread, on a smaller sample (one sequence at a time leaves OpenMP nothing to split)
+    n_one = min(n_seq, 8)
+    t1 = time.perf_counter()
+    for b in range(n_one):
+        oracle.verify(t[b:b + 1], d[b:b + 1] if (d is not None and w.temperature > 0) else None, inp.parent,
+                      c[b:b + 1], u[b:b + 1], w.temperature, w.mode)
+    dt1 = time.perf_counter() - t1
     return {"value": nodes / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"first {n_seq} of {w.batch} sequences of the same inputs, {dt:.2f} s wall, all-node form, "
-                      f"OpenMP over sequences"}, res
+                      f"OpenMP over sequences",
+            "single_thread": {"value": n_one * inp.stats["n_draft"] / dt1, "unit": UNIT, "cores": 1,
+                              "sample": f"first {n_one} sequences one at a time, {dt1:.2f} s wall"}}, res
 
 
 # ----------------------------------------------------------------------------- reference arm
@@ -225,6 +263,35 @@ def workload_config(w: synth.Workload, st, **extra):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
+def timed_steps(step, n_steps: int, dist, dev, clock_index):
+    """n_steps calls of step(events) between barriers and synchronisations; CUDA events around the whole
+    region and around the node stage of every step; clocks sampled meanwhile.  Returns (elapsed ms of
+    the slowest rank, node-stage ms per step of this rank, clock record or None)."""
+    node_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(n_steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(clock_index) if clock_index is not None else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_host0 = time.time()
+    start.record()
+    for i in range(n_steps):
+        step(node_events[i])
+    stop.record()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    t_host1 = time.time()
+    elapsed_ms = max_over_ranks(dist, start.elapsed_time(stop), dev)
+    node_ms = [a.elapsed_time(b) for a, b in node_events]
+    clocks = sampler.stop(t_host0, t_host1) if sampler else None
+    return elapsed_ms, node_ms, clocks
+
+
 def run_cuda(args):
     from paper_2401_06706_b200 import binding
     rank, world, local = dist_env()
@@ -278,29 +345,7 @@ def run_cuda(args):
 
     # timed region: K steps between barriers and synchronisations, CUDA events on the
     # launching stream; the node kernel of every step is bracketed by its own events
-    node_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                   for _ in range(args.steps)]
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
-    if sampler:
-        sampler.start()
-        time.sleep(0.25)
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    t_host0 = time.time()
-    start.record()
-    for i in range(args.steps):
-        step(node_events[i])
-    stop.record()
-    torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-    t_host1 = time.time()
-    elapsed_ms = start.elapsed_time(stop)
-    node_ms = [a.elapsed_time(b) for a, b in node_events]
-    elapsed_ms = max_over_ranks(dist, elapsed_ms, dev)
-    clocks = sampler.stop(t_host0, t_host1) if sampler else None
+    elapsed_ms, node_ms, clocks = timed_steps(step, args.steps, dist, dev, torch.cuda.current_device() if rank == 0 else None)
     status_bits = int(ver.status.max().item()) if w.batch else 0
 
     ms_per_step = elapsed_ms / args.steps
@@ -309,7 +354,8 @@ def run_cuda(args):
     # roofline of the dominant kernel (the per-node kernel): algorithmic bytes per launch =
     # every target row once + every draft row once (none at temperature 0) + 12 bytes of
     # candidate token and uniforms per node
-    algo_bytes = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
+    logit_bytes = inp.logit_bytes()
+    algo_bytes = logit_bytes + 12 * w.batch * st["n_nodes"]
     if args.form == "path":
         # only the rows of visited nodes are read: len+1 target rows per sequence and one draft
         # row per visited node that has children (every node above the leaf level)
@@ -320,6 +366,9 @@ def run_cuda(args):
     node_ms_avg = sum(node_ms) / len(node_ms)
     achieved = algo_bytes / (node_ms_avg * 1e-3) / 1e9
     peak, peak_kind = measured_peaks()
+    traffic, traffic_source, traffic_scale = (recorded_traffic(w.batch * st["n_nodes"])
+                                              if (w.name == "cfg5_largest" and w.dtype == "fp32" and args.form == "all_node")
+                                              else (None, "no capture of this kernel variant and workload", None))
     roofline = {"bound": "hbm", "kernel": ("node_kernel" if w.temperature > 0 else "argmax_kernel") +
                 (" (one launch per level; the figure covers the whole call, which is bound by launch and "
                  "exchange latency, not by HBM)" if args.form == "path" else ""),
@@ -327,8 +376,21 @@ def run_cuda(args):
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_avg": node_ms_avg,
                 "kernel_ms_min": min(node_ms), "step_share": node_ms_avg / ms_per_step,
-                "traffic": recorded_traffic(w.batch * st["n_nodes"])
-                if (w.name == "cfg5_largest" and w.dtype == "fp32" and args.form == "all_node") else None}
+                "traffic": traffic, "traffic_source": traffic_source, "traffic_scale": traffic_scale}
+
+    # the same steps again, many more of them: the power cap pulls the SM clock down after the first
+    # hundred milliseconds, and the kernel's time follows the clock.  Clocks come from the sampler;
+    # no clock setting is touched.
+    sustained = None
+    if args.sustained_steps > 0 and world == 1:
+        s_ms, s_node, s_clk = timed_steps(step, args.sustained_steps, None, dev, torch.cuda.current_device())
+        k_ms = sum(s_node) / len(s_node)
+        sustained = {"steps": args.sustained_steps, "ms_per_step": s_ms / args.sustained_steps, "kernel_ms_avg": k_ms,
+                     "achieved": algo_bytes / (k_ms * 1e-3) / 1e9, "frac": algo_bytes / (k_ms * 1e-3) / 1e9 / peak,
+                     "sm_mhz": s_clk["sm_mhz"] if s_clk else None, "reasons": s_clk["reasons"] if s_clk else None,
+                     "power_w_max": s_clk.get("power_w_max") if s_clk else None,
+                     "kernel_ms_x_mhz": (k_ms * s_clk["sm_mhz"]) if (s_clk and s_clk["sm_mhz"]) else None,
+                     "timed_region_kernel_ms_x_mhz": (node_ms_avg * clocks["sm_mhz"]) if (clocks and clocks["sm_mhz"]) else None}
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside
     e2e = None
@@ -340,6 +402,16 @@ def run_cuda(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline, ref = oracle_sample(inp, args.oracle_seqs)
         parity = parity_on_sample(inp, ver, ref, min(args.oracle_seqs, w.batch))
+    accept_len_mean = float(ver.accept_len.float().mean().item()) if w.batch else 0.0
+
+    # sub-record: the same workload with 2-byte logits (the precision the paper ran in, Section 4.1)
+    half = None
+    if (rank == 0 and world == 1 and not args.no_half and w.dtype == "fp32" and args.form == "all_node"
+            and w.temperature > 0):
+        from dataclasses import replace
+        del inp, ver
+        torch.cuda.empty_cache()
+        half = half_record(replace(w, dtype="bf16"), dev, args, peak)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -347,12 +419,15 @@ def run_cuda(args):
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": workload_config(w, st, form=args.form, parallelism=f"replicas x{world} (batch split, no collective)",
                                           l2="inputs (%.2f GB per GPU) far larger than the 126 MB L2" %
-                                          (inp.logit_bytes() / 1e9) if inp.logit_bytes() > 4 * 126e6 else
+                                          (logit_bytes / 1e9) if logit_bytes > 4 * 126e6 else
                                           "inputs smaller than 4x L2: latency/L2-bound point",
-                                          logit_gb_per_gpu=inp.logit_bytes() / 1e9),
-                "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                                          logit_gb_per_gpu=logit_bytes / 1e9),
+                "roofline": roofline, "sustained": sustained, "bf16": half, "cpu_baseline": cpu_baseline, "e2e": e2e,
                 "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
                 "hbm_gbs_whole_step": algo_bytes / (ms_per_step * 1e-3) / 1e9,
+                "us_per_call": ms_per_step * 1e3,
+                "rows_per_sec": world * w.batch * (st["n_nodes"] + (st["n_internal"] if w.temperature > 0 else 0)) / (ms_per_step * 1e-3),
+                "accept_len_mean": accept_len_mean,
                 "device_status_bits": status_bits, "parity_on_oracle_sample": parity}
         print(json.dumps(line), flush=True)
     if dist:
@@ -370,14 +445,72 @@ def parity_on_sample(inp, ver, ref, n_seq):
     out = rep.summary()
     out["ok"] = rep.ok
     out["accept_len_mean"] = float(ref.accept_len.mean())
+    # acceptance rate of the synthetic inputs: share of nodes with children that accepted one of their
+    # candidates (all nodes of the sampled trees), for comparison with the paper's alpha (Section 4.1)
+    n_int = inp.stats["n_internal"]
+    out["alpha_hat"] = float((ref.node_accept[:, :n_int] >= 0).mean()) if n_int else None
     return out
 
 
-def run_e2e(args, w, inp, dist, world, dev):
+def half_record(w, dev, args, peak):
+    """Node stage and whole step of the same workload with 2-byte logits: kernel ms, GB/s, fraction of
+    the peak, clocks, parity on a sample."""
     from paper_2401_06706_b200 import binding
-    from dataclasses import replace
-    nb = min(w.batch, args.e2e_batch)
+    inp = synth.make_inputs(w, dev)
     st = inp.stats
+    ver = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[w.dtype], dev)
+
+    def step(events):
+        e0, e1 = events
+        e0.record()
+        ver.mcsd_verify_nodes(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+        e1.record()
+        ver.mcsd_verify_walk(inp.target, inp.draft, inp.cand, inp.unif, w.temperature)
+
+    dummy = (torch.cuda.Event(), torch.cuda.Event())
+    for _ in range(max(args.warmup, 3)):
+        step(dummy)
+    n = max(20, min(args.steps, 100))
+    ms, node_ms, clk = timed_steps(step, n, None, dev, torch.cuda.current_device())
+    algo = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
+    k_ms = sum(node_ms) / len(node_ms)
+    rec = {"logit_dtype": w.dtype, "steps": n, "ms_per_step": ms / n, "kernel_ms_avg": k_ms, "kernel_ms_min": min(node_ms),
+           "algorithmic_bytes_per_launch": algo, "achieved": algo / (k_ms * 1e-3) / 1e9, "unit": "GB/s",
+           "frac": algo / (k_ms * 1e-3) / 1e9 / peak, "value": w.batch * st["n_draft"] / (ms / n * 1e-3), "clocks": clk}
+    if not args.no_cpu_baseline:
+        # cpu_baseline leg of this sub-record: the oracle timed on the first sequences of these inputs;
+        # what it computed is then compared with the kernels' output on those sequences
+        rec["cpu_baseline"], ref = oracle_sample(inp, min(64, args.oracle_seqs))
+        rec["parity_on_oracle_sample"] = parity_on_sample(inp, ver, ref, min(64, args.oracle_seqs, w.batch))
+    return rec
+
+
+def host_mem_available() -> int:
+    try:
+        with open("/proc/meminfo") as f:
+            for line in f:
+                if line.startswith("MemAvailable:"):
+                    return int(line.split()[1]) * 1024
+    except Exception:
+        pass
+    return 0
+
+
+def run_e2e(args, w, inp, dist, world, dev):
+    """The same metric through mcsd_verify_host: inputs in pinned HOST memory, every copy in both
+    directions inside the timed region.  The whole batch of the workload per step when the host can
+    pin it, else the largest part that fits (said in the record)."""
+    from paper_2401_06706_b200 import binding
+    st = inp.stats
+    per_seq = inp.logit_bytes() // max(w.batch, 1) + 12 * st["n_nodes"]
+    nb, why = w.batch, "the whole batch"
+    if args.e2e_batch > 0:
+        nb, why = min(w.batch, args.e2e_batch), "--e2e-batch"
+    else:
+        avail = host_mem_available()
+        while nb > 1 and avail and 2 * per_seq * nb + (8 << 30) > avail:     # an unpinned copy exists while pinning
+            nb //= 2
+            why = f"host memory: {avail / 2**30:.0f} GiB available"
     pin = lambda t: None if t is None else t[:nb].cpu().pin_memory()
     target, cand, unif = pin(inp.target), pin(inp.cand), pin(inp.unif)
     draft = pin(inp.draft) if w.temperature > 0 else None
@@ -391,7 +524,7 @@ def run_e2e(args, w, inp, dist, world, dev):
     def step():
         binding.mcsd_verify_host(target, draft, inp.parent, cand, unif, w.temperature, w.mode, out=out)
 
-    step()
+    step()                              # the first call allocates the staging buffers the library then keeps
     steps = max(1, min(args.steps, args.e2e_steps))
     if dist:
         dist.barrier()
@@ -402,11 +535,14 @@ def run_e2e(args, w, inp, dist, world, dev):
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
     dt = max_over_ranks(dist, dt, dev)
+    binding.mcsd_release_host_staging()
     value = world * nb * st["n_draft"] * steps / dt
     return {"value": value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-            "ms_per_step": dt / steps * 1e3, "steps": steps, "batch": nb,
-            "note": "mcsd_verify_host on pinned host buffers; device allocation, copies in both directions and "
-                    "kernels inside the timed region; bound by the host link"}
+            "ms_per_step": dt / steps * 1e3, "steps": steps, "batch": nb, "batch_reason": why,
+            "h2d_gbs": h2d * steps / dt / 1e9,
+            "note": "mcsd_verify_host on pinned host buffers; copies in both directions and kernels inside the timed "
+                    "region (the library's device staging buffers are allocated by the untimed first call); bound by "
+                    "the host link: h2d_gbs is what the copies achieved"}
 
 
 # ----------------------------------------------------------------------------- sweep
@@ -424,7 +560,11 @@ def run_sweep(args):
     binding.load_library()
     peak, peak_kind = measured_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    points = [w for w in synth.sweep_workloads() if args.sweep_filter in w.name]
+    if args.named:
+        # the named configurations 1 to 4 (the latency-bound ones), parity on every sequence
+        points = [w for name, w in synth.named_workloads().items() if name != "cfg5_largest" and args.sweep_filter in name]
+    else:
+        points = [w for w in synth.sweep_workloads() if args.sweep_filter in w.name]
     out = open(args.sweep_out, "w") if args.sweep_out else None
     for w in points:
         inp = synth.make_inputs(w, dev)
@@ -432,6 +572,16 @@ def run_sweep(args):
         ver = binding.Verifier(w.batch, inp.parent, w.vocab, synth.TORCH_DTYPES[w.dtype], dev)
         for _ in range(5):
             ver.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+        # back to back, inputs resident in L2 where they fit: what a decoding loop that verifies the
+        # logits it has just produced sees
+        torch.cuda.synchronize()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record()
+        for _ in range(args.sweep_hot_calls):
+            ver.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+        h1.record()
+        torch.cuda.synchronize()
+        us_hot = h0.elapsed_time(h1) * 1e3 / max(args.sweep_hot_calls, 1)
         times = []
         for _ in range(args.sweep_calls):
             flush.fill_(1)
@@ -442,7 +592,7 @@ def run_sweep(args):
             torch.cuda.synchronize()
             times.append(e0.elapsed_time(e1))
         med, best = statistics.median(times), min(times)
-        n_par = min(w.batch, args.sweep_parity_seqs)
+        n_par = w.batch if args.named else min(w.batch, args.sweep_parity_seqs)
         # cpu_baseline leg of the point: the oracle on its first sequences, timed; its output is
         # what the kernels' output is compared with
         t, d, c, u = inp.host_f32(0, n_par)
@@ -454,7 +604,9 @@ def run_sweep(args):
                               residual=ver.residual[:n_par].cpu().numpy(), status=ver.status[:n_par].cpu().numpy())
         algo = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
         rec = {"workload": w.name, "dtype": w.dtype, "batch": w.batch, "kconfig": w.kconfig, "sigma": w.draft_sigma,
-               "mode": w.mode, "algorithmic_mb": algo / 1e6, "us_median": med * 1e3, "us_min": best * 1e3,
+               "mode": w.mode, "temperature": w.temperature, "vocab": w.vocab, "algorithmic_mb": algo / 1e6,
+               "us_median": med * 1e3, "us_min": best * 1e3, "us_back_to_back": us_hot,
+               "launches_per_call": binding.mcsd_last_launch_count(),
                "nodes_per_s": w.batch * st["n_draft"] / (med * 1e-3), "gbs": algo / (med * 1e-3) / 1e9,
                "frac_of_peak": algo / (med * 1e-3) / 1e9 / peak, "peak_kind": peak_kind,
                "regime": "hbm" if algo > 4 * 126e6 else "latency/L2-bound point (inputs < 4x L2)",
@@ -465,7 +617,7 @@ def run_sweep(args):
         if out:
             out.write(json.dumps(rec) + "\n")
             out.flush()
-        print(f"{w.name:40s} {rec['algorithmic_mb']:9.1f} MB {rec['us_median']:9.1f} us {rec['gbs']:7.0f} GB/s "
+        print(f"{w.name:40s} {rec['algorithmic_mb']:9.1f} MB {rec['us_median']:9.1f} us (hot {us_hot:7.1f}) {rec['gbs']:7.0f} GB/s "
               f"{rec['frac_of_peak']:.3f} tau-1={rec['accept_len_mean']:.2f} parity={'ok' if rep.ok else 'FAIL'}", flush=True)
         del inp, ver
         torch.cuda.empty_cache()
@@ -566,10 +718,14 @@ def main():
     ap.add_argument("--workload", default="cfg5_largest")
     ap.add_argument("--oracle-seqs", type=int, default=256,
                     help="sequences of the workload the CPU oracle is timed on")
-    ap.add_argument("--e2e-batch", type=int, default=128, help="sequences per end-to-end step")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-batch", type=int, default=0,
+                    help="sequences per end-to-end step (0: the whole batch if the host has the memory to pin it)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sustained-steps", type=int, default=300,
+                    help="further steps after the timed region for the sustained-clock record (0: none)")
+    ap.add_argument("--no-half", action="store_true", help="skip the sub-record with 2-byte logits")
     ap.add_argument("--batch", type=int, default=0, help="override the batch of the workload (profiling)")
     ap.add_argument("--logit-dtype", default="", choices=["", "fp32", "bf16", "fp16"],
                     help="override the logit type of the workload (profiling)")
@@ -582,9 +738,14 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the bench line")
     ap.add_argument("--sweep-filter", default="", help="only sweep points whose name contains this text")
     ap.add_argument("--sweep-out", default="", help="file for one JSON line per sweep point")
+    ap.add_argument("--named", action="store_true",
+                    help="with --sweep: the named configurations 1 to 4 instead of the sweep points, parity on every sequence")
     ap.add_argument("--sweep-calls", type=int, default=20)
+    ap.add_argument("--sweep-hot-calls", type=int, default=100)
     ap.add_argument("--sweep-parity-seqs", type=int, default=16)
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.sweep:
+        raise SystemExit(spawn_ranks(args))
     if args.sweep:
         run_sweep(args)
     elif args.impl == "reference":

@@ -65,7 +65,7 @@ extern "C" {
 
 /* 101: mcsd_desc gained node_residual at its end (a caller built against 100 must be rebuilt)
  * 102: out_status describes the walk only and is written, not accumulated; mcsd_set_option,
- *      mcsd_get_option, mcsd_release_host_staging; desc->reserved is checked */
+ *      mcsd_get_option, mcsd_release_host_staging; desc->reserved is checked; mcsd_shard_* */
 #define MCSD_VERSION 102
 
 /* logit element types (both logit tensors share one) */
@@ -362,6 +362,90 @@ int mcsd_gather_accepted_kv(void *cache, int64_t n_slabs, int64_t slab_stride, i
                             int64_t seq_stride, int64_t pos_stride, int64_t row_bytes,
                             int64_t n_positions, const int32_t *prefix_len, const int32_t *path_nodes,
                             const int32_t *accept_len, int32_t gamma, void *stream);
+
+/*
+ * Verification with the vocabulary split over several devices.  Section 4.1 runs its largest
+ * target models across two GPUs; when the LM head stays column-split, device s holds only
+ * columns [col_begin, col_begin + n_cols) of both logit tensors.  Algorithms 1 and 2 need, per
+ * node, a handful of sums over the whole vocabulary (the two softmax normalisers, then one
+ * residual sum per rejection that is followed by another test), so the step becomes a sequence
+ * of rounds: every shard forms the partial sums of its columns, the CALLER gathers the partials
+ * of all shards with a collective of its own (an all-gather of a few floats per node: NCCL,
+ * MPI, ...; the library links none), and every shard takes the same decisions from the gathered
+ * values.  Nothing but these partials, the candidates' own logits and, at the end, one token per
+ * sequence crosses devices; no logit does.  The partials are formed over the same runs of columns
+ * and in the same order as mcsd_verify forms them inside one device, so node_accept,
+ * accept_len and the accepted tokens are identical to mcsd_verify's on the full tensors.
+ *
+ * One call sequence per step, the same on every shard (S = n_shards, R = mcsd_shard_rounds):
+ *   mcsd_shard_partials(round 0)            -> part_out, cand_logits_out
+ *   gather part_out -> stats_all [S][B*n_nodes][entries_per_shard] float4   (kept until the end)
+ *   gather cand_logits_out -> cand_logits_all [S][B*n_nodes] float2
+ *   mcsd_shard_decide(round 0, part_all = stats_all)
+ *   for r = 1 .. R:  mcsd_shard_partials(round r) -> part_out; gather -> part_all;
+ *                    mcsd_shard_decide(round r, part_all)
+ *   for attempt = 0, 1:  mcsd_shard_endpoint(attempt) -> totals_out [B][entries_per_shard] double;
+ *                    gather -> totals_all [S][B][entries_per_shard];  mcsd_shard_finish(attempt)
+ *   reduce endpoint_part over the shards (maximum: the shard that holds the token wrote it, the
+ *   others -1);  mcsd_shard_commit puts it behind the accepted tokens.
+ * (attempt 1 only touches sequences whose residual after the last rejection had no mass and
+ * returns at once for all others.)  All buffers are device memory of the caller; the partial
+ * and gathered buffers may be reused from step to step.  Temperature must be > 0 (the argmax
+ * rule needs no sums; MCSD_ERR_UNSUPPORTED) and the mode Algorithm 1 or 2.
+ */
+typedef struct mcsd_shard_desc {
+    int32_t batch, n_nodes, n_internal;
+    int32_t vocab;          /* V of the WHOLE vocabulary                                      */
+    int32_t dtype;          /* MCSD_DTYPE_*                                                   */
+    int32_t reserved;       /* must be 0                                                      */
+    int32_t n_shards, shard;/* 1 <= n_shards <= 32, 0 <= shard < n_shards                     */
+    int64_t ld_target;      /* elements between rows of this shard's target_slice, >= n_cols  */
+    int64_t ld_draft;
+    void *stream;
+    void *workspace;        /* device scratch of this shard, 256-byte aligned, at least        */
+    size_t workspace_bytes; /* mcsd_shard_workspace_bytes() bytes; must survive the whole step */
+    float *node_ratio;      /* optional [B][n_nodes], as in mcsd_desc                          */
+    int32_t *node_accept;   /* optional [B][n_nodes]: accepted child of every node with children,
+                               or -1 (entries of leaves are not written); NULL: kept in the workspace */
+} mcsd_shard_desc;
+
+/* The column range shard `shard` of `n_shards` must hold, and the entries per shard of the
+ * exchanged buffers.  Ranges are whole runs of the node kernel's column partition for this
+ * vocabulary and dtype; trailing shards may be empty.  Host only, no device needed. */
+int mcsd_shard_columns(int32_t vocab, int32_t dtype, int32_t n_shards, int32_t shard, int32_t *col_begin,
+                       int32_t *n_cols, int32_t *entries_per_shard);
+/* Bytes of mcsd_shard_desc.workspace; 0 for an invalid descriptor. */
+size_t mcsd_shard_workspace_bytes(const mcsd_shard_desc *desc);
+/* Rounds after round 0 a tree needs: (largest number of children of a node) - 1; negative
+ * MCSD_ERR_* for a malformed tree. */
+int mcsd_shard_rounds(const int32_t *tree_parent, int32_t n_nodes);
+/* Partial sums of this shard's columns.  target_slice [B][n_nodes][ld_target], draft_slice
+ * [B][n_internal][ld_draft] (device); part_out [B*n_nodes][entries_per_shard] float4;
+ * cand_logits_out [B*n_nodes] float2 (round 0 only).  Round r >= 1 reads what
+ * mcsd_shard_decide(round r - 1) left in the workspace. */
+int mcsd_shard_partials(const mcsd_shard_desc *desc, const void *target_slice, const void *draft_slice,
+                        const int32_t *tree_parent, const int32_t *cand_tokens, float temperature, int32_t round,
+                        void *part_out, void *cand_logits_out);
+/* Decisions of Algorithm 1 / 2 from the gathered partials (identical on every shard). */
+int mcsd_shard_decide(const mcsd_shard_desc *desc, const int32_t *tree_parent, const int32_t *cand_tokens,
+                      const float *uniforms, float temperature, int replacement_mode, int32_t round,
+                      const void *part_all, const void *cand_logits_all);
+/* Mass of every run of the residual of the node where each walk stops, and that residual
+ * (unnormalised) in out_residual_slice [B][n_cols] (may be NULL). */
+int mcsd_shard_endpoint(const mcsd_shard_desc *desc, const void *target_slice, const void *draft_slice,
+                        const int32_t *tree_parent, float temperature, int32_t attempt, const void *stats_all,
+                        void *totals_out, float *out_residual_slice);
+/* Walk outputs (the same on every shard), this shard's part of the endpoint draw
+ * (endpoint_part[b] = token or -1) and the scaling of out_residual_slice. */
+int mcsd_shard_finish(const mcsd_shard_desc *desc, const void *target_slice, const void *draft_slice,
+                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                      float temperature, int32_t attempt, const void *stats_all, const void *totals_all,
+                      int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_status, int32_t *out_path_nodes,
+                      int32_t *endpoint_part, float *out_residual_slice);
+
+/* out_tokens[b][accept_len[b]] = endpoint_all[b] (the reduced endpoint_part). */
+int mcsd_shard_commit(const mcsd_shard_desc *desc, const int32_t *tree_parent, const int32_t *endpoint_all,
+                      const int32_t *accept_len, int32_t *out_tokens);
 
 /* Frees the device staging buffers and streams mcsd_verify_host keeps on the current
  * device (allocating again on its next call).  Returns MCSD_OK or MCSD_ERR_CUDA. */

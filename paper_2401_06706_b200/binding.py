@@ -25,7 +25,9 @@ MAX_NODES, MAX_CHILDREN, MAX_VOCAB = 512, 32, 65536
 EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_host", "mcsd_verify_static", "mcsd_verify_path", "mcsd_sample_candidates", "mcsd_tree_attention_layout",
            "mcsd_gather_accepted_kv",
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
-           "mcsd_version", "mcsd_set_option", "mcsd_get_option", "mcsd_release_host_staging")
+           "mcsd_version", "mcsd_set_option", "mcsd_get_option", "mcsd_release_host_staging",
+           "mcsd_shard_columns", "mcsd_shard_workspace_bytes", "mcsd_shard_rounds", "mcsd_shard_partials",
+           "mcsd_shard_decide", "mcsd_shard_endpoint", "mcsd_shard_finish", "mcsd_shard_commit")
 OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL = range(7)
 
 
@@ -38,6 +40,15 @@ class McsdDesc(ctypes.Structure):
                 ("node_accept", ctypes.c_void_p), ("node_bonus", ctypes.c_void_p),
                 ("node_ratio", ctypes.c_void_p), ("out_status", ctypes.c_void_p),
                 ("out_path_nodes", ctypes.c_void_p), ("node_residual", ctypes.c_void_p)]
+
+
+class McsdShardDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_nodes", ctypes.c_int32), ("n_internal", ctypes.c_int32),
+                ("vocab", ctypes.c_int32), ("dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("n_shards", ctypes.c_int32), ("shard", ctypes.c_int32),
+                ("ld_target", ctypes.c_int64), ("ld_draft", ctypes.c_int64),
+                ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("node_ratio", ctypes.c_void_p), ("node_accept", ctypes.c_void_p)]
 
 
 class McsdError(RuntimeError):
@@ -96,6 +107,23 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_get_option.restype = ctypes.c_int
     lib.mcsd_release_host_staging.argtypes = []
     lib.mcsd_release_host_staging.restype = ctypes.c_int
+    sp = ctypes.POINTER(McsdShardDesc)
+    lib.mcsd_shard_columns.argtypes = [i32, i32, i32, i32, vp, vp, vp]
+    lib.mcsd_shard_columns.restype = ctypes.c_int
+    lib.mcsd_shard_workspace_bytes.argtypes = [sp]
+    lib.mcsd_shard_workspace_bytes.restype = ctypes.c_size_t
+    lib.mcsd_shard_rounds.argtypes = [vp, i32]
+    lib.mcsd_shard_rounds.restype = ctypes.c_int
+    lib.mcsd_shard_partials.argtypes = [sp, vp, vp, vp, vp, f32, i32, vp, vp]
+    lib.mcsd_shard_partials.restype = ctypes.c_int
+    lib.mcsd_shard_decide.argtypes = [sp, vp, vp, vp, f32, ctypes.c_int, i32, vp, vp]
+    lib.mcsd_shard_decide.restype = ctypes.c_int
+    lib.mcsd_shard_endpoint.argtypes = [sp, vp, vp, vp, f32, i32, vp, vp, vp]
+    lib.mcsd_shard_endpoint.restype = ctypes.c_int
+    lib.mcsd_shard_finish.argtypes = [sp, vp, vp, vp, vp, vp, f32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.mcsd_shard_finish.restype = ctypes.c_int
+    lib.mcsd_shard_commit.argtypes = [sp, vp, vp, vp, vp]
+    lib.mcsd_shard_commit.restype = ctypes.c_int
     if path is None:
         _lib = lib
     return lib
@@ -378,3 +406,166 @@ def mcsd_verify_host(target, draft, parent, cand, unif, temperature: float, mode
                                 _ptr(unif), float(temperature), int(mode), _ptr(accept_len), _ptr(tokens),
                                 _ptr(residual), _ptr(status)))
     return VerifyOutput(accept_len, tokens, residual, status)
+
+
+# ---------------------------------------------------------------- vocabulary split over several devices
+def mcsd_shard_columns(vocab: int, dtype: torch.dtype, n_shards: int, shard: int):
+    """(col_begin, n_cols, entries_per_shard) of one shard; host only (see mcsd.h)."""
+    a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _check(load_library().mcsd_shard_columns(int(vocab), MCSD_DTYPE[dtype], int(n_shards), int(shard),
+                                             ctypes.addressof(a), ctypes.addressof(b), ctypes.addressof(c)))
+    return a.value, b.value, c.value
+
+
+class ShardedVerifier:
+    """One shard of the verification with the vocabulary split over several devices: holds the
+    descriptor, the workspace and the exchange buffers of its device and exposes the stage calls of
+    mcsd.h under their own names (argument marshalling only).  `sharded_verify` runs a step."""
+
+    def __init__(self, batch: int, parent, vocab: int, dtype: torch.dtype, n_shards: int, shard: int, device="cuda"):
+        self.lib = load_library()
+        self.parent = np.ascontiguousarray(parent, dtype=np.int32)
+        self.device = torch.device(device)
+        self.batch, self.vocab, self.dtype = int(batch), int(vocab), dtype
+        self.n_nodes, self.n_internal = int(self.parent.shape[0]), _n_internal(self.parent)
+        self.n_shards, self.shard = int(n_shards), int(shard)
+        self.col_begin, self.n_cols, self.eps = mcsd_shard_columns(vocab, dtype, n_shards, shard)
+        self.gamma = mcsd_tree_depth(self.parent)
+        rounds = self.lib.mcsd_shard_rounds(self.parent.ctypes.data, self.n_nodes)
+        _check(rounds if rounds < 0 else 0)
+        self.rounds = rounds
+        d = self.desc = McsdShardDesc()
+        d.batch, d.n_nodes, d.n_internal, d.vocab = self.batch, self.n_nodes, self.n_internal, self.vocab
+        d.dtype, d.n_shards, d.shard = MCSD_DTYPE[dtype], self.n_shards, self.shard
+        d.ld_target = d.ld_draft = max(self.n_cols, 1)
+        ws = int(self.lib.mcsd_shard_workspace_bytes(ctypes.byref(d)))
+        if ws == 0:
+            _check(-2)
+        self.workspace = torch.zeros(ws + 256, dtype=torch.uint8, device=self.device)
+        d.workspace = (self.workspace.data_ptr() + 255) // 256 * 256
+        d.workspace_bytes = ws
+        n_items = self.batch * self.n_nodes
+        f32 = dict(dtype=torch.float32, device=self.device)
+        i32 = dict(dtype=torch.int32, device=self.device)
+        # exchanged buffers: this shard's part, and what the collective gathers from all shards
+        self.part = torch.zeros((n_items, self.eps, 4), **f32)
+        self.cval = torch.zeros((n_items, 2), **f32)
+        self.totals = torch.zeros((self.batch, self.eps), dtype=torch.float64, device=self.device)
+        self.stats_all = torch.zeros((self.n_shards, n_items, self.eps, 4), **f32)
+        self.part_all = torch.zeros((self.n_shards, n_items, self.eps, 4), **f32)
+        self.cval_all = torch.zeros((self.n_shards, n_items, 2), **f32)
+        self.totals_all = torch.zeros((self.n_shards, self.batch, self.eps), dtype=torch.float64, device=self.device)
+        self.endpoint_part = torch.full((self.batch,), -1, **i32)
+        self.accept_len = torch.empty(self.batch, **i32)
+        self.tokens = torch.empty((self.batch, self.gamma + 1), **i32)
+        self.status = torch.zeros(self.batch, **i32)
+        self.path_nodes = torch.empty((self.batch, self.gamma + 1), **i32)
+        self.residual = torch.zeros((self.batch, max(self.n_cols, 1)), **f32)
+        self.node_accept = torch.full((self.batch, self.n_nodes), -1, **i32)
+        d.node_accept = self.node_accept.data_ptr()
+
+    def _bind(self, target, draft):
+        if self.n_cols:
+            assert target.dtype == self.dtype and target.shape == (self.batch, self.n_nodes, self.n_cols)
+            self.desc.ld_target = _row_stride(target)
+            if self.n_internal:
+                assert draft.shape == (self.batch, self.n_internal, self.n_cols)
+                self.desc.ld_draft = _row_stride(draft)
+        self.desc.stream = torch.cuda.current_stream(self.device).cuda_stream
+
+    def mcsd_shard_partials(self, target, draft, cand, temperature: float, rnd: int):
+        self._bind(target, draft)
+        _check(self.lib.mcsd_shard_partials(ctypes.byref(self.desc), _ptr(target), _ptr(draft), self.parent.ctypes.data,
+                                            _ptr(cand), float(temperature), int(rnd), _ptr(self.part), _ptr(self.cval)))
+
+    def mcsd_shard_decide(self, cand, unif, temperature: float, mode: int, rnd: int):
+        self.desc.stream = torch.cuda.current_stream(self.device).cuda_stream
+        gathered = self.stats_all if rnd == 0 else self.part_all
+        _check(self.lib.mcsd_shard_decide(ctypes.byref(self.desc), self.parent.ctypes.data, _ptr(cand), _ptr(unif),
+                                          float(temperature), int(mode), int(rnd), _ptr(gathered), _ptr(self.cval_all)))
+
+    def mcsd_shard_endpoint(self, target, draft, temperature: float, attempt: int):
+        self._bind(target, draft)
+        _check(self.lib.mcsd_shard_endpoint(ctypes.byref(self.desc), _ptr(target), _ptr(draft), self.parent.ctypes.data,
+                                            float(temperature), int(attempt), _ptr(self.stats_all), _ptr(self.totals),
+                                            _ptr(self.residual)))
+
+    def mcsd_shard_finish(self, target, draft, cand, unif, temperature: float, attempt: int):
+        self._bind(target, draft)
+        _check(self.lib.mcsd_shard_finish(ctypes.byref(self.desc), _ptr(target), _ptr(draft), self.parent.ctypes.data,
+                                          _ptr(cand), _ptr(unif), float(temperature), int(attempt), _ptr(self.stats_all),
+                                          _ptr(self.totals_all), _ptr(self.accept_len), _ptr(self.tokens),
+                                          _ptr(self.status), _ptr(self.path_nodes), _ptr(self.endpoint_part),
+                                          _ptr(self.residual)))
+
+
+    def mcsd_shard_commit(self):
+        self.desc.stream = torch.cuda.current_stream(self.device).cuda_stream
+        _check(self.lib.mcsd_shard_commit(ctypes.byref(self.desc), self.parent.ctypes.data, _ptr(self.endpoint_part),
+                                          _ptr(self.accept_len), _ptr(self.tokens)))
+
+
+class DistComm:
+    """The collectives of a step over torch.distributed (NCCL between GPUs): all-gathers of a few
+    floats per node and one maximum of an int32 per sequence.  No logit crosses devices."""
+
+    def __init__(self, group=None):
+        import torch.distributed as dist
+        self.dist, self.group = dist, group
+
+    def all_gather(self, shards, name_local: str, name_all: str):
+        (sh,) = shards
+        self.dist.all_gather_into_tensor(getattr(sh, name_all).view(-1), getattr(sh, name_local).contiguous().view(-1),
+                                         group=self.group)
+
+    def all_reduce_max(self, shards, name: str):
+        (sh,) = shards
+        self.dist.all_reduce(getattr(sh, name), op=self.dist.ReduceOp.MAX, group=self.group)
+
+
+class LocalComm:
+    """The same collectives between shard objects that live in one process (several shards on one
+    device, for tests): plain copies."""
+
+    def all_gather(self, shards, name_local: str, name_all: str):
+        for dst in shards:
+            for src in shards:
+                getattr(dst, name_all)[src.shard].copy_(getattr(src, name_local))
+
+    def all_reduce_max(self, shards, name: str):
+        best = torch.stack([getattr(sh, name) for sh in shards]).max(dim=0).values
+        for sh in shards:
+            getattr(sh, name).copy_(best)
+
+
+def sharded_verify(shards, targets, drafts, cand, unif, temperature: float, mode: int, comm) -> VerifyOutput:
+    """One verification step over column-split logits, following the call sequence of mcsd.h.
+    shards: the ShardedVerifier objects this process drives (one per rank under torch.distributed; all of
+    them when several shards are emulated on one device), targets / drafts: their column slices, in the
+    same order; cand, unif: replicated inputs.  Returns the outputs of the first shard; its `residual`
+    holds that shard's columns of the distribution."""
+    T = float(temperature)
+    for sh, t, d in zip(shards, targets, drafts):
+        sh.mcsd_shard_partials(t, d, cand, T, 0)
+    comm.all_gather(shards, "part", "stats_all")
+    comm.all_gather(shards, "cval", "cval_all")
+    for sh in shards:
+        sh.mcsd_shard_decide(cand, unif, T, mode, 0)
+    for rnd in range(1, shards[0].rounds + 1):
+        for sh, t, d in zip(shards, targets, drafts):
+            sh.mcsd_shard_partials(t, d, cand, T, rnd)
+        comm.all_gather(shards, "part", "part_all")
+        for sh in shards:
+            sh.mcsd_shard_decide(cand, unif, T, mode, rnd)
+    for attempt in (0, 1):
+        for sh, t, d in zip(shards, targets, drafts):
+            sh.mcsd_shard_endpoint(t, d, T, attempt)
+        comm.all_gather(shards, "totals", "totals_all")
+        for sh, t, d in zip(shards, targets, drafts):
+            sh.mcsd_shard_finish(t, d, cand, unif, T, attempt)
+    comm.all_reduce_max(shards, "endpoint_part")
+    for sh in shards:
+        sh.mcsd_shard_commit()
+    sh = shards[0]
+    return VerifyOutput(sh.accept_len, sh.tokens, sh.residual, sh.status, node_accept=sh.node_accept,
+                        path_nodes=sh.path_nodes)

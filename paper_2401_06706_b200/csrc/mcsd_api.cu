@@ -788,6 +788,311 @@ int mcsd_gather_accepted_kv(void *cache, int64_t n_slabs, int64_t slab_stride, i
     return MCSD_OK;
 }
 
+// ---- verification with the vocabulary split over several devices ------------------------
+namespace {
+
+struct ShardLayout {
+    int ept, run, n_entries, eps_max, entry_begin, eps, col_begin, n_cols;
+};
+
+// Runs are those of the node kernel for this vocabulary and dtype (32 * elements per thread);
+// shard s owns the entries [s * eps_max, (s + 1) * eps_max) that exist.
+int shard_layout(int vocab, int dtype, int n_shards, int shard, ShardLayout *L)
+{
+    if (n_shards < 1 || n_shards > 32 || shard < 0 || shard >= n_shards) return MCSD_ERR_SHAPE;
+    NodeConfig cfg;
+    const int rc = choose_config(vocab, dtype, true, &cfg);
+    if (rc != MCSD_OK) return rc;
+    L->ept = cfg.ept;
+    L->run = 32 * cfg.ept;
+    L->n_entries = (vocab + L->run - 1) / L->run;
+    L->eps_max = (L->n_entries + n_shards - 1) / n_shards;
+    L->entry_begin = shard * L->eps_max;
+    int e_end = L->entry_begin + L->eps_max;
+    if (e_end > L->n_entries) e_end = L->n_entries;
+    L->eps = e_end > L->entry_begin ? e_end - L->entry_begin : 0;
+    L->col_begin = L->entry_begin * L->run < vocab ? L->entry_begin * L->run : vocab;
+    int col_end = e_end * L->run;
+    if (col_end > vocab) col_end = vocab;
+    L->n_cols = col_end > L->col_begin ? col_end - L->col_begin : 0;
+    return MCSD_OK;
+}
+
+struct ShardWorkspace {
+    float4 *act;
+    float2 *req;
+    float *s_hist;
+    int32_t *node_accept;
+    NodeStats *stats;
+    int32_t *retry;
+    size_t bytes;
+};
+
+ShardWorkspace carve_shard(void *base, long long n_items, int batch)
+{
+    ShardWorkspace w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        unsigned char *p = base ? static_cast<unsigned char *>(base) + off : nullptr;
+        off += align_up(bytes, 256);
+        return p;
+    };
+    w.act = reinterpret_cast<float4 *>(take(sizeof(float4) * n_items));
+    w.req = reinterpret_cast<float2 *>(take(sizeof(float2) * n_items));
+    w.s_hist = reinterpret_cast<float *>(take(sizeof(float) * MCSD_MAX_CHILDREN * n_items));
+    w.node_accept = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
+    w.stats = reinterpret_cast<NodeStats *>(take(sizeof(NodeStats) * n_items));
+    w.retry = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
+    w.bytes = off;
+    return w;
+}
+
+int check_shard_desc(const mcsd_shard_desc *d, ShardLayout *L)
+{
+    if (!d) return MCSD_ERR_NULL;
+    if (d->reserved != 0) return MCSD_ERR_SHAPE;
+    if (d->batch < 0 || d->n_nodes < 1 || d->vocab < 1 || d->n_internal < 0 || d->n_internal > d->n_nodes)
+        return MCSD_ERR_SHAPE;
+    if (d->n_nodes > MCSD_MAX_NODES || d->vocab > MCSD_MAX_VOCAB) return MCSD_ERR_UNSUPPORTED;
+    if (static_cast<long long>(d->batch) * d->n_nodes > 0x7fffffffLL) return MCSD_ERR_UNSUPPORTED;
+    if (d->dtype != MCSD_DTYPE_F32 && d->dtype != MCSD_DTYPE_BF16 && d->dtype != MCSD_DTYPE_F16) return MCSD_ERR_DTYPE;
+    const int rc = shard_layout(d->vocab, d->dtype, d->n_shards, d->shard, L);
+    if (rc != MCSD_OK) return rc;
+    if (d->ld_target < L->n_cols || (d->n_internal > 0 && d->ld_draft < L->n_cols)) return MCSD_ERR_STRIDE;
+    return MCSD_OK;
+}
+
+int fill_shard_params(const mcsd_shard_desc *d, const int32_t *parent, float T, int mode, ShardParams *p, TreePlan *plan,
+                      ShardLayout *L)
+{
+    int rc = check_shard_desc(d, L);
+    if (rc != MCSD_OK) return rc;
+    rc = plan_tree_cached(parent, d->n_nodes, d->n_internal, plan);
+    if (rc != MCSD_OK) return rc;
+    if (!(T > 0.f) || std::isinf(T)) return T == 0.f ? MCSD_ERR_UNSUPPORTED : MCSD_ERR_TEMPERATURE;
+    if (mode != MCSD_MODE_WITH_REPLACEMENT && mode != MCSD_MODE_WITHOUT_REPLACEMENT) return MCSD_ERR_MODE;
+    const long long n_items = static_cast<long long>(d->batch) * d->n_nodes;
+    const ShardWorkspace need = carve_shard(nullptr, n_items, d->batch);
+    if (!d->workspace || reinterpret_cast<uintptr_t>(d->workspace) % 256 != 0 || d->workspace_bytes < need.bytes)
+        return MCSD_ERR_WORKSPACE;
+    const ShardWorkspace ws = carve_shard(d->workspace, n_items, d->batch);
+    *p = ShardParams();
+    p->ld_t = d->ld_target; p->ld_d = d->ld_draft;
+    p->B = d->batch; p->n_nodes = d->n_nodes; p->n_internal = d->n_internal; p->V = d->vocab;
+    p->col_begin = L->col_begin; p->n_cols = L->n_cols; p->eps = L->eps; p->entry_begin = L->entry_begin;
+    p->n_entries = L->n_entries; p->eps_max = L->eps_max; p->n_shards = d->n_shards; p->mode = mode;
+    p->gamma = plan->gamma;
+    const double scale_d = 1.4426950408889634 / static_cast<double>(T);
+    p->scale = static_cast<float>(scale_d);
+    p->scale_lo = static_cast<float>(scale_d - static_cast<double>(p->scale));
+    p->act = ws.act; p->req = ws.req; p->s_hist = ws.s_hist; p->stats = ws.stats;
+    p->node_accept = d->node_accept ? d->node_accept : ws.node_accept;
+    p->retry = ws.retry;
+    p->node_ratio = d->node_ratio;
+    std::memcpy(p->child_first, plan->child_first, sizeof(p->child_first));
+    std::memcpy(p->child_count, plan->child_count, sizeof(p->child_count));
+    for (int n = 0; n < d->n_nodes; ++n) p->parent[n] = static_cast<int16_t>(parent[n]);
+    return MCSD_OK;
+}
+
+unsigned shard_grid(long long warps)
+{
+    int dev = 0, n_sm = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    long long ctas = (warps + 3) / 4;
+    const long long cap = static_cast<long long>(n_sm) * 16;
+    if (ctas > cap) ctas = cap;
+    return static_cast<unsigned>(ctas < 1 ? 1 : ctas);
+}
+
+#define MCSD_SHARD_LAUNCH(kernel, dtype, ept, grid, stream, params)                                             \
+    do {                                                                                                        \
+        switch ((dtype) * 100 + (ept)) {                                                                        \
+        case MCSD_DTYPE_F32 * 100 + 16: kernel<MCSD_DTYPE_F32, 16><<<grid, kShardThreads, 0, stream>>>(params); break;   \
+        case MCSD_DTYPE_F32 * 100 + 32: kernel<MCSD_DTYPE_F32, 32><<<grid, kShardThreads, 0, stream>>>(params); break;   \
+        case MCSD_DTYPE_F32 * 100 + 64: kernel<MCSD_DTYPE_F32, 64><<<grid, kShardThreads, 0, stream>>>(params); break;   \
+        case MCSD_DTYPE_BF16 * 100 + 16: kernel<MCSD_DTYPE_BF16, 16><<<grid, kShardThreads, 0, stream>>>(params); break; \
+        case MCSD_DTYPE_BF16 * 100 + 32: kernel<MCSD_DTYPE_BF16, 32><<<grid, kShardThreads, 0, stream>>>(params); break; \
+        case MCSD_DTYPE_BF16 * 100 + 64: kernel<MCSD_DTYPE_BF16, 64><<<grid, kShardThreads, 0, stream>>>(params); break; \
+        case MCSD_DTYPE_F16 * 100 + 16: kernel<MCSD_DTYPE_F16, 16><<<grid, kShardThreads, 0, stream>>>(params); break;   \
+        case MCSD_DTYPE_F16 * 100 + 32: kernel<MCSD_DTYPE_F16, 32><<<grid, kShardThreads, 0, stream>>>(params); break;   \
+        default: kernel<MCSD_DTYPE_F16, 64><<<grid, kShardThreads, 0, stream>>>(params); break;                          \
+        }                                                                                                       \
+    } while (0)
+
+}  // namespace
+
+int mcsd_shard_columns(int32_t vocab, int32_t dtype, int32_t n_shards, int32_t shard, int32_t *col_begin,
+                       int32_t *n_cols, int32_t *entries_per_shard)
+{
+    if (vocab < 1 || vocab > MCSD_MAX_VOCAB) return MCSD_ERR_SHAPE;
+    if (dtype != MCSD_DTYPE_F32 && dtype != MCSD_DTYPE_BF16 && dtype != MCSD_DTYPE_F16) return MCSD_ERR_DTYPE;
+    ShardLayout L;
+    const int rc = shard_layout(vocab, dtype, n_shards, shard, &L);
+    if (rc != MCSD_OK) return rc;
+    if (col_begin) *col_begin = L.col_begin;
+    if (n_cols) *n_cols = L.n_cols;
+    if (entries_per_shard) *entries_per_shard = L.eps_max;
+    return MCSD_OK;
+}
+
+size_t mcsd_shard_workspace_bytes(const mcsd_shard_desc *desc)
+{
+    ShardLayout L;
+    if (check_shard_desc(desc, &L) != MCSD_OK) return 0;
+    return carve_shard(nullptr, static_cast<long long>(desc->batch) * desc->n_nodes, desc->batch).bytes;
+}
+
+int mcsd_shard_rounds(const int32_t *tree_parent, int32_t n_nodes)
+{
+    TreePlan plan;
+    const int rc = plan_tree(tree_parent, n_nodes, -1, &plan);
+    if (rc != MCSD_OK) return rc;
+    int k_max = 0;
+    for (int n = 0; n < n_nodes; ++n) k_max = plan.child_count[n] > k_max ? plan.child_count[n] : k_max;
+    return k_max > 1 ? k_max - 1 : 0;
+}
+
+int mcsd_shard_partials(const mcsd_shard_desc *desc, const void *target_slice, const void *draft_slice,
+                        const int32_t *tree_parent, const int32_t *cand_tokens, float temperature, int32_t round,
+                        void *part_out, void *cand_logits_out)
+{
+    ShardParams p;
+    TreePlan plan;
+    ShardLayout L;
+    int rc = fill_shard_params(desc, tree_parent, temperature, MCSD_MODE_WITH_REPLACEMENT, &p, &plan, &L);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0) return MCSD_OK;
+    if (!part_out || !cand_tokens || (round == 0 && !cand_logits_out)) return MCSD_ERR_NULL;
+    if (L.n_cols > 0 && (!target_slice || (desc->n_internal > 0 && !draft_slice))) return MCSD_ERR_NULL;
+    if (round < 0 || round >= MCSD_MAX_CHILDREN) return MCSD_ERR_SHAPE;
+    p.target = target_slice; p.draft = draft_slice; p.cand = cand_tokens; p.round = round;
+    p.part_out = static_cast<float4 *>(part_out);
+    p.cval_out = static_cast<float2 *>(cand_logits_out);
+    p.vector_ok = (rows_aligned16(target_slice, desc->ld_target, desc->dtype) &&
+                   (desc->n_internal == 0 || rows_aligned16(draft_slice, desc->ld_draft, desc->dtype))) ? 1 : 0;
+    cudaStream_t st = static_cast<cudaStream_t>(desc->stream);
+    const long long n_items = static_cast<long long>(desc->batch) * desc->n_nodes;
+    if (L.eps > 0) {
+        const unsigned grid = shard_grid(n_items * L.eps);
+        MCSD_SHARD_LAUNCH(shard_partials_kernel, desc->dtype, L.ept, grid, st, p);
+        if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+        g_last_launches += 1;
+    }
+    if (round == 0) {
+        const unsigned grid = static_cast<unsigned>((n_items + 255) / 256 < 2048 ? (n_items + 255) / 256 : 2048);
+        switch (desc->dtype) {
+        case MCSD_DTYPE_F32: shard_candidates_kernel<MCSD_DTYPE_F32><<<grid, 256, 0, st>>>(p); break;
+        case MCSD_DTYPE_BF16: shard_candidates_kernel<MCSD_DTYPE_BF16><<<grid, 256, 0, st>>>(p); break;
+        default: shard_candidates_kernel<MCSD_DTYPE_F16><<<grid, 256, 0, st>>>(p); break;
+        }
+        if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+        g_last_launches += 1;
+    }
+    return MCSD_OK;
+}
+
+int mcsd_shard_decide(const mcsd_shard_desc *desc, const int32_t *tree_parent, const int32_t *cand_tokens,
+                      const float *uniforms, float temperature, int replacement_mode, int32_t round,
+                      const void *part_all, const void *cand_logits_all)
+{
+    ShardParams p;
+    TreePlan plan;
+    ShardLayout L;
+    int rc = fill_shard_params(desc, tree_parent, temperature, replacement_mode, &p, &plan, &L);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0 || desc->n_internal == 0) return MCSD_OK;
+    if (!part_all || !cand_logits_all || !cand_tokens || !uniforms) return MCSD_ERR_NULL;
+    if (round < 0 || round >= MCSD_MAX_CHILDREN) return MCSD_ERR_SHAPE;
+    p.cand = cand_tokens; p.unif = uniforms; p.round = round;
+    p.part_all = static_cast<const float4 *>(part_all);
+    p.cval_all = static_cast<const float2 *>(cand_logits_all);
+    const unsigned grid = shard_grid(static_cast<long long>(desc->batch) * desc->n_internal);
+    shard_decide_kernel<<<grid, kShardThreads, 0, static_cast<cudaStream_t>(desc->stream)>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches = 1;
+    return MCSD_OK;
+}
+
+int mcsd_shard_endpoint(const mcsd_shard_desc *desc, const void *target_slice, const void *draft_slice,
+                        const int32_t *tree_parent, float temperature, int32_t attempt, const void *stats_all,
+                        void *totals_out, float *out_residual_slice)
+{
+    ShardParams p;
+    TreePlan plan;
+    ShardLayout L;
+    int rc = fill_shard_params(desc, tree_parent, temperature, MCSD_MODE_WITH_REPLACEMENT, &p, &plan, &L);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0 || L.eps == 0) return MCSD_OK;
+    if (!target_slice || (desc->n_internal > 0 && !draft_slice) || !stats_all || !totals_out) return MCSD_ERR_NULL;
+    if (attempt != 0 && attempt != 1) return MCSD_ERR_SHAPE;
+    p.target = target_slice; p.draft = draft_slice; p.attempt = attempt;
+    p.stats_all = static_cast<const float4 *>(stats_all);
+    p.tot_out = static_cast<double *>(totals_out);
+    p.out_residual = out_residual_slice;
+    const unsigned grid = shard_grid(static_cast<long long>(desc->batch) * L.eps);
+    cudaStream_t st = static_cast<cudaStream_t>(desc->stream);
+    MCSD_SHARD_LAUNCH(shard_endpoint_kernel, desc->dtype, L.ept, grid, st, p);
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches = 1;
+    return MCSD_OK;
+}
+
+int mcsd_shard_finish(const mcsd_shard_desc *desc, const void *target_slice, const void *draft_slice,
+                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                      float temperature, int32_t attempt, const void *stats_all, const void *totals_all,
+                      int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_status, int32_t *out_path_nodes,
+                      int32_t *endpoint_part, float *out_residual_slice)
+{
+    ShardParams p;
+    TreePlan plan;
+    ShardLayout L;
+    int rc = fill_shard_params(desc, tree_parent, temperature, MCSD_MODE_WITH_REPLACEMENT, &p, &plan, &L);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0) return MCSD_OK;
+    if (!stats_all || !totals_all || !cand_tokens || !uniforms || !out_accept_len || !out_tokens || !out_status ||
+        !endpoint_part)
+        return MCSD_ERR_NULL;
+    if (L.n_cols > 0 && (!target_slice || (desc->n_internal > 0 && !draft_slice))) return MCSD_ERR_NULL;
+    if (attempt != 0 && attempt != 1) return MCSD_ERR_SHAPE;
+    p.target = target_slice; p.draft = draft_slice; p.cand = cand_tokens; p.unif = uniforms; p.attempt = attempt;
+    p.stats_all = static_cast<const float4 *>(stats_all);
+    p.tot_all = static_cast<const double *>(totals_all);
+    p.out_accept_len = out_accept_len; p.out_tokens = out_tokens; p.out_status = out_status;
+    p.out_path_nodes = out_path_nodes; p.endpoint_part = endpoint_part;
+    p.out_residual = out_residual_slice;
+    const unsigned grid = shard_grid(desc->batch);
+    cudaStream_t st = static_cast<cudaStream_t>(desc->stream);
+    MCSD_SHARD_LAUNCH(shard_finish_kernel, desc->dtype, L.ept, grid, st, p);
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches = 1;
+    return MCSD_OK;
+}
+
+int mcsd_shard_commit(const mcsd_shard_desc *desc, const int32_t *tree_parent, const int32_t *endpoint_all,
+                      const int32_t *accept_len, int32_t *out_tokens)
+{
+    ShardLayout L;
+    int rc = check_shard_desc(desc, &L);
+    if (rc != MCSD_OK) return rc;
+    TreePlan plan;
+    rc = plan_tree_cached(tree_parent, desc->n_nodes, desc->n_internal, &plan);
+    if (rc != MCSD_OK) return rc;
+    g_last_launches = 0;
+    if (desc->batch == 0) return MCSD_OK;
+    if (!endpoint_all || !accept_len || !out_tokens) return MCSD_ERR_NULL;
+    shard_commit_kernel<<<(desc->batch + 255) / 256, 256, 0, static_cast<cudaStream_t>(desc->stream)>>>(
+        endpoint_all, accept_len, out_tokens, desc->batch, plan.gamma);
+    if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+    g_last_launches = 1;
+    return MCSD_OK;
+}
+
 // ---- mcsd_verify_static: the scratch memory is an array built into the library --------
 // In host code the name below is only a handle for the runtime; the address kernels can
 // use comes from cudaGetSymbolAddress, looked up once per device.

@@ -23,6 +23,9 @@
 //                    (Section 3.3).
 //   gather_kernel    (mcsd_gather.cuh)  Key/value cache rows of the accepted path to their
 //                    committed positions.
+//   shard_*_kernel   (mcsd_shard.cuh)  The verification with the vocabulary split over several
+//                    devices: per-run partial statistics, decisions from the gathered partials,
+//                    endpoint token and residual per shard.
 // mcsd_common.cuh holds what they share.
 //
 // How the rejection loop avoids rewriting the residual.  After n rejections the
@@ -49,3 +52,4 @@
 #include "mcsd_naive.cuh"
 #include "mcsd_layout.cuh"
 #include "mcsd_gather.cuh"
+#include "mcsd_shard.cuh"

@@ -56,6 +56,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
     constexpr int GV = E::kVec;
     __shared__ int s_term, s_len, s_stat;
     __shared__ int32_t s_acc[MCSD_MAX_NODES], s_tok[MCSD_MAX_NODES];
+    __shared__ uint8_t s_nst[MCSD_MAX_NODES];   // status bits the node stage left at every node with children
     constexpr int kW = NT / 32;  // warps
     __shared__ double s_wtot[32];
     __shared__ float s_leaf[2];
@@ -79,13 +80,14 @@ walk_kernel(const __grid_constant__ WalkParams P)
         for (int i = tid; i < P.n_nodes; i += NT) {
             s_acc[i] = P.node_accept[nb + i];
             s_tok[i] = P.cand[nb + i];
+            s_nst[i] = (P.scale != 0.f && i < P.n_internal) ? static_cast<uint8_t>(P.stats[nb + i].status) : 0;
         }
         __syncthreads();
         if (tid == 0) {
             int st = 0;
             // bounded by the depth of the tree even if node_accept were corrupt
             for (int hop = 0; hop < P.gamma; ++hop) {
-                if (P.scale != 0.f && n < P.n_internal) st |= P.stats[nb + n].status;
+                st |= s_nst[n];
                 const int nx = s_acc[n];
                 if (nx <= n || nx >= P.n_nodes) break;
                 n = nx;
@@ -93,7 +95,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
                 if (P.out_path_nodes) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + len] = n;
                 ++len;
             }
-            if (P.scale != 0.f && n < P.n_internal) st |= P.stats[nb + n].status;
+            st |= s_nst[n];
             for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
             if (P.out_path_nodes)
                 for (int i = len; i <= P.gamma; ++i) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + i] = -1;
@@ -169,6 +171,8 @@ walk_kernel(const __grid_constant__ WalkParams P)
     int x_hi = x_lo + run;
     x_hi = x_hi > P.V ? P.V : x_hi;
 
+    // whole 16-byte stores where the row of `out` allows it
+    const bool out_vec = out && (reinterpret_cast<uintptr_t>(out) % 16 == 0);
     float kappa = fminf(c * dq, 3.0e38f);
     int extra_bits = 0;
     float g[kMaxSteps];
@@ -210,9 +214,15 @@ walk_kernel(const __grid_constant__ WalkParams P)
                 float w[GV];
                 weights(x0, w);
 #pragma unroll
-                for (int e = 0; e < GV; ++e) {
-                    g[st] += w[e];
-                    if (out && x0 + e < P.V) out[x0 + e] = w[e];
+                for (int e = 0; e < GV; ++e) g[st] += w[e];
+                if (out_vec && x0 + GV <= P.V) {
+#pragma unroll
+                    for (int e = 0; e < GV; e += 4)
+                        *reinterpret_cast<float4 *>(out + x0 + e) = make_float4(w[e], w[e + 1], w[e + 2], w[e + 3]);
+                } else if (out) {
+#pragma unroll
+                    for (int e = 0; e < GV; ++e)
+                        if (x0 + e < P.V) out[x0 + e] = w[e];
                 }
             }
         }
@@ -243,9 +253,18 @@ walk_kernel(const __grid_constant__ WalkParams P)
         for (int st = 0; st < kMaxSteps; ++st) {
             const int x0 = x_lo + st * kStep + lane * GV;
             if (x0 < x_hi) {
+                if (out_vec && x0 + GV <= P.V) {
 #pragma unroll
-                for (int e = 0; e < GV; ++e)
-                    if (x0 + e < P.V) out[x0 + e] *= inv_s;
+                    for (int e = 0; e < GV; e += 4) {
+                        float4 v = *reinterpret_cast<float4 *>(out + x0 + e);
+                        v.x *= inv_s; v.y *= inv_s; v.z *= inv_s; v.w *= inv_s;
+                        *reinterpret_cast<float4 *>(out + x0 + e) = v;
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < GV; ++e)
+                        if (x0 + e < P.V) out[x0 + e] *= inv_s;
+                }
             }
         }
     }

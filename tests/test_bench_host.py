@@ -2,7 +2,7 @@
 every rank takes its own seeded batch of the same shape (replicas, no data-path
 collective), the elapsed time reported is the slowest rank's, the value is the whole job's.
 Also: the reference arm of bench.py runs the CPU oracle and prints the agreed JSON line,
-and only rank 0 does so."""
+and only rank 0 does so; and `bench.py --gpus N` without a launcher starts its own N ranks."""
 import json
 import os
 import subprocess
@@ -68,3 +68,19 @@ def test_reference_arm_prints_the_contract_line_on_rank_zero_only():
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["config"]["workload"] == "cfg1_tiny"
     other = _run_reference({"RANK": "1", "WORLD_SIZE": "2"})
     assert other.returncode == 0 and other.stdout.strip() == ""
+
+
+def test_gpus_n_without_a_launcher_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no WORLD_SIZE around it: the script starts two ranks itself
+    (shown on the reference arm, which needs no GPU); stdout is still the one JSON line of rank 0."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg1_tiny",
+           "--steps", "1", "--warmup", "1", "--gpus", "2"]
+    out = subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=600)
+    assert out.returncode == 0, out.stderr
+    lines = [ln for ln in out.stdout.strip().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+    cmd = bench.spawn_command(["--gpus", "2"], 2, 29999)
+    assert "torch.distributed.run" in cmd and "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd
