@@ -582,6 +582,28 @@ def run_sweep(args):
         h1.record()
         torch.cuda.synchronize()
         us_hot = h0.elapsed_time(h1) * 1e3 / max(args.sweep_hot_calls, 1)
+        # the same call captured in a CUDA graph and replayed: the chain of kernels on the GPU without
+        # the host's share (the call neither allocates nor synchronises, so it can be captured)
+        us_graph = None
+        if args.named:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                ver.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                ver.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif, w.temperature, w.mode)
+            graph.replay()
+            torch.cuda.synchronize()
+            h0.record()
+            for _ in range(args.sweep_hot_calls):
+                graph.replay()
+            h1.record()
+            torch.cuda.synchronize()
+            us_graph = h0.elapsed_time(h1) * 1e3 / max(args.sweep_hot_calls, 1)
+            del graph
         times = []
         for _ in range(args.sweep_calls):
             flush.fill_(1)
@@ -605,7 +627,7 @@ def run_sweep(args):
         algo = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
         rec = {"workload": w.name, "dtype": w.dtype, "batch": w.batch, "kconfig": w.kconfig, "sigma": w.draft_sigma,
                "mode": w.mode, "temperature": w.temperature, "vocab": w.vocab, "algorithmic_mb": algo / 1e6,
-               "us_median": med * 1e3, "us_min": best * 1e3, "us_back_to_back": us_hot,
+               "us_median": med * 1e3, "us_min": best * 1e3, "us_back_to_back": us_hot, "us_graph_replay": us_graph,
                "launches_per_call": binding.mcsd_last_launch_count(),
                "nodes_per_s": w.batch * st["n_draft"] / (med * 1e-3), "gbs": algo / (med * 1e-3) / 1e9,
                "frac_of_peak": algo / (med * 1e-3) / 1e9 / peak, "peak_kind": peak_kind,
@@ -617,7 +639,8 @@ def run_sweep(args):
         if out:
             out.write(json.dumps(rec) + "\n")
             out.flush()
-        print(f"{w.name:40s} {rec['algorithmic_mb']:9.1f} MB {rec['us_median']:9.1f} us (hot {us_hot:7.1f}) {rec['gbs']:7.0f} GB/s "
+        print(f"{w.name:40s} {rec['algorithmic_mb']:9.1f} MB {rec['us_median']:9.1f} us (hot {us_hot:7.1f}, graph "
+              f"{us_graph if us_graph is not None else float('nan'):6.1f}) {rec['gbs']:7.0f} GB/s "
               f"{rec['frac_of_peak']:.3f} tau-1={rec['accept_len_mean']:.2f} parity={'ok' if rep.ok else 'FAIL'}", flush=True)
         del inp, ver
         torch.cuda.empty_cache()

@@ -125,7 +125,10 @@ extern "C" {
                                     the bounded wait runs out and MCSD_STATUS_TIMEOUT is reported      */
 #define MCSD_OPT_PDL 6           /* 1 (default): the walk stage is launched as a programmatic dependent
                                     of the node stage; 0: plain stream order                         */
-#define MCSD_OPT_COUNT 7
+#define MCSD_OPT_TEST_SHRINK_RANGES 7 /* checked build only, test of the checker: every registered extent is
+                                         cut short by this many bytes, so that valid reads of the last bytes of
+                                         a tensor are reported (and skipped)                                  */
+#define MCSD_OPT_COUNT 8
 
 typedef struct mcsd_desc {
     int32_t batch;      /* B: number of trees                                         */
@@ -470,6 +473,13 @@ int mcsd_tree_depth(const int32_t *tree_parent, int32_t n_nodes);
 /* Number of kernel launches the last successful mcsd_verify / stage call on this
  * host thread enqueued (for launch accounting in benchmarks). */
 int mcsd_last_launch_count(void);
+
+/* The checked build of the library (libmcsd_debug.so, compiled with MCSD_DEBUG_BOUNDS) verifies every
+ * read of caller memory by the verification, walk, argmax, naive-sampling and candidate-sampling
+ * kernels against the extents the descriptor implies; a read outside them is skipped and counted,
+ * nothing traps.  Returns the number of such reads since the last reset on the current device
+ * (synchronises the device), resets the count if `reset` is not 0; -1 in the normal build. */
+long long mcsd_debug_bounds_hits(int reset);
 
 /* Static description of a return code. */
 const char *mcsd_status_string(int code);

@@ -17,6 +17,7 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmcsd.so")
+DEBUG_LIB_PATH = os.path.join(_HERE, "libmcsd_debug.so")      # the checked build (see mcsd_debug_bounds_hits)
 
 MCSD_DTYPE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 STATUS_DEGENERATE, STATUS_BAD_TOKEN, STATUS_NO_MASS, STATUS_TIMEOUT = 1, 2, 4, 8
@@ -27,8 +28,8 @@ EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
            "mcsd_version", "mcsd_set_option", "mcsd_get_option", "mcsd_release_host_staging",
            "mcsd_shard_columns", "mcsd_shard_workspace_bytes", "mcsd_shard_rounds", "mcsd_shard_partials",
-           "mcsd_shard_decide", "mcsd_shard_endpoint", "mcsd_shard_finish", "mcsd_shard_commit")
-OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL = range(7)
+           "mcsd_shard_decide", "mcsd_shard_endpoint", "mcsd_shard_finish", "mcsd_shard_commit", "mcsd_debug_bounds_hits")
+OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL, OPT_TEST_SHRINK_RANGES = range(8)
 
 
 class McsdDesc(ctypes.Structure):
@@ -124,6 +125,8 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_shard_finish.restype = ctypes.c_int
     lib.mcsd_shard_commit.argtypes = [sp, vp, vp, vp, vp]
     lib.mcsd_shard_commit.restype = ctypes.c_int
+    lib.mcsd_debug_bounds_hits.argtypes = [ctypes.c_int]
+    lib.mcsd_debug_bounds_hits.restype = ctypes.c_longlong
     if path is None:
         _lib = lib
     return lib
@@ -161,6 +164,10 @@ def mcsd_get_option(option: int) -> int:
     rc = load_library().mcsd_get_option(int(option))
     _check(rc if rc < 0 else 0)
     return rc
+
+
+def mcsd_debug_bounds_hits(reset: bool = False) -> int:
+    return int(load_library().mcsd_debug_bounds_hits(1 if reset else 0))
 
 
 def mcsd_release_host_staging() -> None:

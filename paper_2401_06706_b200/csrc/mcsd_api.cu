@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <initializer_list>
 #include <mutex>
 #include <vector>
 
@@ -102,6 +103,28 @@ int plan_tree_cached(const int32_t *parent, int n_nodes, int n_internal, TreePla
 }
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Checked build: the address ranges the kernels of the next launches on `stream` may read.  An
+// empty list switches the checks off (kernels whose inputs are not registered).
+struct Range { const void *p; size_t bytes; };
+#ifdef MCSD_DEBUG_BOUNDS
+int debug_register(cudaStream_t stream, std::initializer_list<Range> ranges)
+{
+    DebugRanges r = {};
+    for (const Range &x : ranges) {
+        if (!x.p || x.bytes == 0 || r.n >= 12) continue;
+        // (MCSD_OPT_TEST_SHRINK_RANGES: a test of the checker itself registers less than is there)
+        const size_t cut = static_cast<size_t>(g_opt.v[MCSD_OPT_TEST_SHRINK_RANGES]);
+        r.lo[r.n] = reinterpret_cast<unsigned long long>(x.p);
+        r.hi[r.n] = r.lo[r.n] + (x.bytes > cut ? x.bytes - cut : 0);
+        ++r.n;
+    }
+    return cudaMemcpyToSymbolAsync(g_dbg_ranges, &r, sizeof(r), 0, cudaMemcpyHostToDevice, stream) == cudaSuccess
+               ? MCSD_OK : MCSD_ERR_CUDA;
+}
+#else
+inline int debug_register(cudaStream_t, std::initializer_list<Range>) { return MCSD_OK; }
+#endif
 
 struct Workspace {
     int32_t *node_accept;
@@ -345,6 +368,15 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         cudaMemsetAsync(c.ws.path[0], 0, sizeof(int32_t) * d->batch, c.stream) != cudaSuccess)
         return MCSD_ERR_CUDA;  // every walk starts at the root
 
+    {
+        const size_t es = static_cast<size_t>(d->dtype == MCSD_DTYPE_F32 ? 4 : 2);
+        const size_t n_all = static_cast<size_t>(d->batch) * d->n_nodes;
+        if (debug_register(c.stream, {{target, n_all * d->ld_target * es},
+                                      {T > 0.f ? draft : nullptr, static_cast<size_t>(d->batch) * d->n_internal * d->ld_draft * es},
+                                      {cand, n_all * 4}, {unif, n_all * 8}, {d->workspace, d->workspace_bytes},
+                                      {d->node_accept, n_all * 4}, {d->node_bonus, n_all * 4}}) != MCSD_OK)
+            return MCSD_ERR_CUDA;
+    }
     if (T == 0.f) {
         ArgmaxParams p = {};
         p.target = target; p.cand = cand;
@@ -427,6 +459,12 @@ int launch_naive(const Call &c, const void *target, const int32_t *cand, const f
 {
     const mcsd_desc *d = c.d;
     if (d->batch == 0) return MCSD_OK;
+    {
+        const size_t es = static_cast<size_t>(d->dtype == MCSD_DTYPE_F32 ? 4 : 2);
+        const size_t n_all = static_cast<size_t>(d->batch) * d->n_nodes;
+        if (debug_register(c.stream, {{target, n_all * d->ld_target * es}, {cand, n_all * 4}, {unif, n_all * 8}}) != MCSD_OK)
+            return MCSD_ERR_CUDA;
+    }
     NaiveParams p = {};
     p.target = target; p.cand = cand; p.unif = unif;
     p.node_accept = c.node_accept;
@@ -456,6 +494,15 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
 {
     const mcsd_desc *d = c.d;
     if (d->batch == 0) return MCSD_OK;
+    {
+        const size_t es = static_cast<size_t>(d->dtype == MCSD_DTYPE_F32 ? 4 : 2);
+        const size_t n_all = static_cast<size_t>(d->batch) * d->n_nodes;
+        if (debug_register(c.stream, {{target, n_all * d->ld_target * es},
+                                      {T > 0.f ? draft : nullptr, static_cast<size_t>(d->batch) * d->n_internal * d->ld_draft * es},
+                                      {cand, n_all * 4}, {unif, n_all * 8}, {d->workspace, d->workspace_bytes},
+                                      {d->node_accept, n_all * 4}, {d->node_bonus, n_all * 4}}) != MCSD_OK)
+            return MCSD_ERR_CUDA;
+    }
     WalkParams p = {};
     p.target = target; p.draft = draft; p.cand = cand; p.unif = unif;
     p.node_accept = c.node_accept; p.node_bonus = c.node_bonus;
@@ -484,7 +531,16 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
     using WalkKernel = void (*)(const WalkParams);
     WalkKernel fn;
     int threads;
-    if (d->vocab <= MCSD_MAX_VOCAB / 2) {
+    // 512 threads (two CTAs per SM) when the vocabulary allows it and there are more CTAs than SMs;
+    // a small batch takes 1024 threads per sequence: half the work per thread, shorter chains
+    int n_sm = 148;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    }
+    const bool want_all_early = all_nodes_allowed && ((T > 0.f && d->node_bonus) || d->node_residual);
+    if (d->vocab <= MCSD_MAX_VOCAB / 2 && (d->batch > n_sm || want_all_early)) {
         threads = 512;
         fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 512>
            : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 512> : walk_kernel<MCSD_DTYPE_F16, 512>;
@@ -559,6 +615,23 @@ int mcsd_tree_depth(const int32_t *tree_parent, int32_t n_nodes)
 }
 
 int mcsd_last_launch_count(void) { return g_last_launches; }
+
+long long mcsd_debug_bounds_hits(int reset)
+{
+#ifdef MCSD_DEBUG_BOUNDS
+    unsigned long long hits = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return MCSD_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&hits, g_dbg_hits, sizeof(hits)) != cudaSuccess) return MCSD_ERR_CUDA;
+    if (reset) {
+        const unsigned long long zero = 0;
+        if (cudaMemcpyToSymbol(g_dbg_hits, &zero, sizeof(zero)) != cudaSuccess) return MCSD_ERR_CUDA;
+    }
+    return static_cast<long long>(hits);
+#else
+    (void)reset;
+    return -1;
+#endif
+}
 
 int mcsd_set_option(int option, int value)
 {
@@ -685,6 +758,13 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
     if (!draft_logits || !cand_tokens || (temperature > 0.f && !uniforms_draw)) return MCSD_ERR_NULL;
     if (desc->ld_draft < desc->vocab) return MCSD_ERR_STRIDE;
     if (n_ctas > 0x7fffffffLL) return MCSD_ERR_UNSUPPORTED;
+    {
+        const size_t es = static_cast<size_t>(desc->dtype == MCSD_DTYPE_F32 ? 4 : 2);
+        if (debug_register(static_cast<cudaStream_t>(desc->stream),
+                           {{draft_logits, static_cast<size_t>(desc->batch) * desc->n_internal * desc->ld_draft * es},
+                            {uniforms_draw, static_cast<size_t>(desc->batch) * desc->n_nodes * 4}}) != MCSD_OK)
+            return MCSD_ERR_CUDA;
+    }
     SampleParams p = {};
     p.draft = draft_logits; p.unif_draw = uniforms_draw; p.cand = cand_tokens; p.status = desc->out_status;
     p.ld_d = desc->ld_draft;
@@ -736,6 +816,7 @@ int mcsd_tree_attention_layout(const int32_t *tree_parent, int32_t n_nodes, int3
     if (rc != MCSD_OK) return rc;
     g_last_launches = 0;
     if (!mask && !position_ids) return MCSD_OK;
+    if (debug_register(static_cast<cudaStream_t>(stream), {}) != MCSD_OK) return MCSD_ERR_CUDA;
     LayoutParams p = {};
     p.mask = mask; p.position_ids = position_ids; p.n_nodes = n_nodes; p.prefix_len = prefix_len;
     for (int n = 0; n < n_nodes; ++n) p.parent[n] = static_cast<int16_t>(tree_parent[n]);
@@ -764,6 +845,7 @@ int mcsd_gather_accepted_kv(void *cache, int64_t n_slabs, int64_t slab_stride, i
     int unit = 16;
     while (unit > 1 && (all & static_cast<unsigned long long>(unit - 1))) unit >>= 1;
     if (row_bytes / unit > 0x7fffffffLL) return MCSD_ERR_UNSUPPORTED;
+    if (debug_register(static_cast<cudaStream_t>(stream), {}) != MCSD_OK) return MCSD_ERR_CUDA;
     GatherParams p = {};
     p.cache = static_cast<unsigned char *>(cache);
     p.slab_stride = slab_stride; p.seq_stride = seq_stride; p.pos_stride = pos_stride;
@@ -876,6 +958,7 @@ int fill_shard_params(const mcsd_shard_desc *d, const int32_t *parent, float T, 
     if (!d->workspace || reinterpret_cast<uintptr_t>(d->workspace) % 256 != 0 || d->workspace_bytes < need.bytes)
         return MCSD_ERR_WORKSPACE;
     const ShardWorkspace ws = carve_shard(d->workspace, n_items, d->batch);
+    if (debug_register(static_cast<cudaStream_t>(d->stream), {}) != MCSD_OK) return MCSD_ERR_CUDA;
     *p = ShardParams();
     p->ld_t = d->ld_target; p->ld_d = d->ld_draft;
     p->B = d->batch; p->n_nodes = d->n_nodes; p->n_internal = d->n_internal; p->V = d->vocab;

@@ -63,6 +63,31 @@ struct NodeParams {
     uint8_t child_count[MCSD_MAX_NODES];
 };
 
+// ------------------------------------------------------------------ checked build
+// With -DMCSD_DEBUG_BOUNDS (the library libmcsd_debug.so) every read of caller memory that goes
+// through the helpers below is checked against the address ranges the host registered for the
+// launch: a read outside them is not performed (the helper returns zeros, or its fill value) and
+// is counted; nothing traps.  compute-sanitizer's memcheck stands behind this; the normal build
+// compiles the checks away.
+#ifdef MCSD_DEBUG_BOUNDS
+struct DebugRanges {
+    int n;                            // 0: nothing registered, nothing is checked
+    unsigned long long lo[12], hi[12];
+};
+__device__ DebugRanges g_dbg_ranges;
+__device__ unsigned long long g_dbg_hits;
+__device__ __forceinline__ bool dbg_ok(const void *p, size_t bytes) {
+    if (g_dbg_ranges.n == 0) return true;
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+    for (int i = 0; i < g_dbg_ranges.n; ++i)
+        if (a >= g_dbg_ranges.lo[i] && a + bytes <= g_dbg_ranges.hi[i]) return true;
+    atomicAdd(&g_dbg_hits, 1ull);
+    return false;
+}
+#else
+__device__ __forceinline__ constexpr bool dbg_ok(const void *, size_t) { return true; }
+#endif
+
 // ------------------------------------------------------------------ element types
 // Three-input maximum (a NaN operand is ignored, as with fmaxf).
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -81,6 +106,7 @@ template <> struct Elem<MCSD_DTYPE_F32> {
         o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
     }
     static __device__ __forceinline__ float load(const void *base, long long i) {
+        if (!dbg_ok(reinterpret_cast<const float *>(base) + i, 4)) return 0.f;
         return __ldg(reinterpret_cast<const float *>(base) + i);
     }
     // value of element i given the aligned 32-bit word that contains it
@@ -103,6 +129,7 @@ template <> struct Elem<MCSD_DTYPE_BF16> {
         o[6] = __uint_as_float(r.w << 16); o[7] = __uint_as_float(r.w & 0xffff0000u);
     }
     static __device__ __forceinline__ float load(const void *base, long long i) {
+        if (!dbg_ok(reinterpret_cast<const unsigned short *>(base) + i, 2)) return 0.f;
         unsigned short h = __ldg(reinterpret_cast<const unsigned short *>(base) + i);
         return __uint_as_float(static_cast<uint32_t>(h) << 16);
     }
@@ -135,6 +162,7 @@ template <> struct Elem<MCSD_DTYPE_F16> {
         }
     }
     static __device__ __forceinline__ float load(const void *base, long long i) {
+        if (!dbg_ok(reinterpret_cast<const __half *>(base) + i, 2)) return 0.f;
         return __half2float(__ldg(reinterpret_cast<const __half *>(base) + i));
     }
     static __device__ __forceinline__ float from_word(uint32_t w, long long i) {
@@ -205,11 +233,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
 // One bulk async copy global -> this CTA's shared memory (TMA; the copy goes to this CTA alone);
 // completion is signalled on an mbarrier of this CTA as a byte count.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    (void)dbg_ok(src, bytes);   // (counted only: the waiting side expects the bytes)
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 // Asks L2 to fetch a 16-byte-aligned range (size a multiple of 16); nothing waits on it.
 __device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+    if (!dbg_ok(src, bytes)) return;
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 // 4-byte asynchronous copy global -> shared (no register holds the value in flight).
@@ -219,6 +249,7 @@ __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void cp_async4(void *smem_dst, const void *src) {
+    if (!dbg_ok(src, 4)) return;
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() {
@@ -227,6 +258,7 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // 128-bit streaming load (read once, do not keep in L1).
 __device__ __forceinline__ uint4 ld_stream_v4(const void *p) {
     uint4 r;
+    if (!dbg_ok(p, 16)) return make_uint4(0u, 0u, 0u, 0u);
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
@@ -235,6 +267,7 @@ __device__ __forceinline__ uint4 ld_stream_v4(const void *p) {
 // A run of these has no branch between the loads, so they are all in flight together.
 __device__ __forceinline__ uint4 ld_stream_v4_if(const void *p, bool pred, uint32_t fill) {
     uint4 r;
+    pred = pred && dbg_ok(p, 16);
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\t"
                  "mov.u32 %0, %6;\n\tmov.u32 %1, %6;\n\tmov.u32 %2, %6;\n\tmov.u32 %3, %6;\n\t"
                  "@q ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];\n\t}"
@@ -245,12 +278,18 @@ __device__ __forceinline__ uint4 ld_stream_v4_if(const void *p, bool pred, uint3
 // Predicated 128-bit load that may stay in the caches (for data that is read again soon).
 __device__ __forceinline__ uint4 ld_v4_if(const void *p, bool pred, uint32_t fill) {
     uint4 r;
+    pred = pred && dbg_ok(p, 16);
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\t"
                  "mov.u32 %0, %6;\n\tmov.u32 %1, %6;\n\tmov.u32 %2, %6;\n\tmov.u32 %3, %6;\n\t"
                  "@q ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];\n\t}"
                  : "=&r"(r.x), "=&r"(r.y), "=&r"(r.z), "=&r"(r.w)
                  : "l"(p), "r"(static_cast<uint32_t>(pred)), "r"(fill));
     return r;
+}
+// 128-bit load through the read-only path (data that may be read again soon).
+__device__ __forceinline__ uint4 ldg_v4(const void *p) {
+    if (!dbg_ok(p, 16)) return make_uint4(0u, 0u, 0u, 0u);
+    return __ldg(reinterpret_cast<const uint4 *>(p));
 }
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     uint32_t r;

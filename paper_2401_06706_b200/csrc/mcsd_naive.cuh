@@ -54,7 +54,7 @@ naive_kernel(const __grid_constant__ NaiveParams P)
     const unsigned char *row = nullptr;
     auto load_group = [&](int x0, float *v) {
         if (P.vector_ok && x0 + GV <= P.V) {
-            E::unpack(__ldg(reinterpret_cast<const uint4 *>(row + static_cast<size_t>(x0) * E::kBytes)), v);
+            E::unpack(ldg_v4(row + static_cast<size_t>(x0) * E::kBytes), v);
         } else {
 #pragma unroll
             for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;

@@ -60,7 +60,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
         (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes;
     auto load_group = [&](int x0, float *v) {   // GV logits from x0 on, -inf past the vocabulary
         if (P.vector_ok && x0 + GV <= P.V) {
-            E::unpack(__ldg(reinterpret_cast<const uint4 *>(row + static_cast<size_t>(x0) * E::kBytes)), v);
+            E::unpack(ldg_v4(row + static_cast<size_t>(x0) * E::kBytes), v);
         } else {
 #pragma unroll
             for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
@@ -76,7 +76,7 @@ sample_kernel(const __grid_constant__ SampleParams P)
     auto load_group_clamped = [&](int x0, float *v) {
         if (P.vector_ok) {
             const int xc = x0 < x_last ? x0 : x_last;
-            E::unpack(__ldg(reinterpret_cast<const uint4 *>(row + static_cast<size_t>(xc) * E::kBytes)), v);
+            E::unpack(ldg_v4(row + static_cast<size_t>(xc) * E::kBytes), v);
             if (tail_mask) {
 #pragma unroll
                 for (int e = 0; e < GV; ++e) v[e] = xc + e < P.V ? v[e] : -INFINITY;

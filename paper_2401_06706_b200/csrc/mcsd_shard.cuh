@@ -74,7 +74,7 @@ __device__ __forceinline__ void run_exponentials(const unsigned char *row, int n
         const int x = (j * 32 + lane) * GV;
         float f[GV];
         if (vector_ok && x + GV <= n_valid) {
-            E::unpack(__ldg(reinterpret_cast<const uint4 *>(row + static_cast<size_t>(x) * E::kBytes)), f);
+            E::unpack(ldg_v4(row + static_cast<size_t>(x) * E::kBytes), f);
         } else {
 #pragma unroll
             for (int e = 0; e < GV; ++e) f[e] = (x + e < n_valid) ? E::load(row, x + e) : -INFINITY;

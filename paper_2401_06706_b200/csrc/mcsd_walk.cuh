@@ -56,7 +56,10 @@ walk_kernel(const __grid_constant__ WalkParams P)
     constexpr int GV = E::kVec;
     __shared__ int s_term, s_len, s_stat;
     __shared__ int32_t s_acc[MCSD_MAX_NODES], s_tok[MCSD_MAX_NODES];
-    __shared__ uint8_t s_nst[MCSD_MAX_NODES];   // status bits the node stage left at every node with children
+    // what the node stage left at every node with children, and every node's endpoint uniform: loaded
+    // up front in parallel, so that nothing the walk decides has to wait for another trip to memory
+    __shared__ NodeStats s_stats[MCSD_MAX_NODES];
+    __shared__ float s_uend[MCSD_MAX_NODES];
     constexpr int kW = NT / 32;  // warps
     __shared__ double s_wtot[32];
     __shared__ float s_leaf[2];
@@ -80,14 +83,17 @@ walk_kernel(const __grid_constant__ WalkParams P)
         for (int i = tid; i < P.n_nodes; i += NT) {
             s_acc[i] = P.node_accept[nb + i];
             s_tok[i] = P.cand[nb + i];
-            s_nst[i] = (P.scale != 0.f && i < P.n_internal) ? static_cast<uint8_t>(P.stats[nb + i].status) : 0;
+            if (P.scale != 0.f) {
+                s_uend[i] = P.unif[2 * (nb + i) + 1];
+                if (i < P.n_internal) s_stats[i] = P.stats[nb + i];
+            }
         }
         __syncthreads();
         if (tid == 0) {
             int st = 0;
             // bounded by the depth of the tree even if node_accept were corrupt
             for (int hop = 0; hop < P.gamma; ++hop) {
-                st |= s_nst[n];
+                if (P.scale != 0.f && n < P.n_internal) st |= s_stats[n].status;
                 const int nx = s_acc[n];
                 if (nx <= n || nx >= P.n_nodes) break;
                 n = nx;
@@ -95,7 +101,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
                 if (P.out_path_nodes) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + len] = n;
                 ++len;
             }
-            st |= s_nst[n];
+            if (P.scale != 0.f && n < P.n_internal) st |= s_stats[n].status;
             for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
             if (P.out_path_nodes)
                 for (int i = len; i <= P.gamma; ++i) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + i] = -1;
@@ -137,7 +143,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
     const bool internal = n < P.n_internal;
     float r_t, z_t, r_d = 0.f, z_d = 0.f, c = 0.f, c_prev = 0.f;
     if (internal) {
-        const NodeStats st = P.stats[nb + n];
+        const NodeStats st = P.all_nodes ? P.stats[nb + n] : s_stats[n];
         r_t = st.r_t; r_d = st.r_d; z_t = st.z_t; z_d = st.z_d; c = st.c; c_prev = st.c_prev;
     } else {
         if (warp == 0) {
@@ -183,8 +189,8 @@ walk_kernel(const __grid_constant__ WalkParams P)
     auto weights = [&](int x0, float *w) {
         float t[GV], d[GV];
         if (P.vector_ok && x0 + GV <= P.V) {
-            E::unpack(__ldg(reinterpret_cast<const uint4 *>(t_row + static_cast<size_t>(x0) * E::kBytes)), t);
-            if (kappa > 0.f) E::unpack(__ldg(reinterpret_cast<const uint4 *>(d_row + static_cast<size_t>(x0) * E::kBytes)), d);
+            E::unpack(ldg_v4(t_row + static_cast<size_t>(x0) * E::kBytes), t);
+            if (kappa > 0.f) E::unpack(ldg_v4(d_row + static_cast<size_t>(x0) * E::kBytes), d);
         } else {
 #pragma unroll
             for (int e = 0; e < GV; ++e) {
@@ -199,7 +205,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
             w[e] = v;
         }
     };
-    const float u_end = P.unif[2 * (nb + n) + 1];
+    const float u_end = P.all_nodes ? P.unif[2 * (nb + n) + 1] : s_uend[n];
     // at most two attempts: the residual after the last rejection and, if that one has no mass,
     // the one before it
 #pragma unroll 1

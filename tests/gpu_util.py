@@ -60,7 +60,8 @@ def library_options(**opts):
     for the duration of a block and restores what was there before."""
     ids = {"cluster": binding.OPT_CLUSTER, "ept": binding.OPT_EPT, "direct": binding.OPT_DIRECT,
            "sample_ahead": binding.OPT_SAMPLE_AHEAD, "wait_polls": binding.OPT_WAIT_POLLS,
-           "test_extra_tx": binding.OPT_TEST_EXTRA_TX, "pdl": binding.OPT_PDL}
+           "test_extra_tx": binding.OPT_TEST_EXTRA_TX, "pdl": binding.OPT_PDL,
+           "test_shrink_ranges": binding.OPT_TEST_SHRINK_RANGES}
     before = {k: binding.mcsd_get_option(ids[k]) for k in opts}
     try:
         for k, val in opts.items():
