@@ -112,8 +112,8 @@ extern "C" {
 #define MCSD_STATUS_TIMEOUT 8    /* a bounded on-chip wait expired; results invalid      */
 
 /* Options of mcsd_set_option: process-wide tuning and test overrides, 0 = library default.
- * The first four also take their initial value from the environment variable of the same
- * name (MCSD_CLUSTER, MCSD_EPT, MCSD_DIRECT, MCSD_SAMPLE_AHEAD, MCSD_PDL), read once when
+ * Some also take their initial value from the environment variable of the same
+ * name (MCSD_CLUSTER, MCSD_EPT, MCSD_DIRECT, MCSD_SAMPLE_AHEAD, MCSD_PDL, MCSD_SPLIT), read once when
  * the library is loaded. */
 #define MCSD_OPT_CLUSTER 0       /* CTAs per thread-block cluster of the node kernel (1..8)          */
 #define MCSD_OPT_EPT 1           /* vocabulary elements per thread and row of the node kernel         */
@@ -128,7 +128,10 @@ extern "C" {
 #define MCSD_OPT_TEST_SHRINK_RANGES 7 /* checked build only, test of the checker: every registered extent is
                                          cut short by this many bytes, so that valid reads of the last bytes of
                                          a tensor are reported (and skipped)                                  */
-#define MCSD_OPT_COUNT 8
+#define MCSD_OPT_SPLIT 8         /* the all-node form of mcsd_verify at temperature > 0 gives its cluster kernel only
+                                    the nodes with two or more children and streams the rows of the others with a
+                                    kernel of its own: 0 = for large launches (default), 1 = never, 2 = always    */
+#define MCSD_OPT_COUNT 9
 
 typedef struct mcsd_desc {
     int32_t batch;      /* B: number of trees                                         */

@@ -34,6 +34,7 @@ struct Options {
         v[MCSD_OPT_WAIT_POLLS] = 0;
         v[MCSD_OPT_TEST_EXTRA_TX] = 0;
         v[MCSD_OPT_PDL] = env_int("MCSD_PDL", 1);
+        v[MCSD_OPT_SPLIT] = env_int("MCSD_SPLIT", 0);
     }
 };
 Options g_opt;
@@ -131,6 +132,7 @@ struct Workspace {
     int32_t *node_bonus;
     NodeStats *stats;
     float2 *leaf_part;
+    float4 *single_part;
     int32_t *status;
     int32_t *path[2];
     size_t bytes;
@@ -138,6 +140,7 @@ struct Workspace {
 
 Workspace carve(void *base, long long n_items, long long n_leaf_items, int batch)
 {
+    const long long n_internal_items = n_items - n_leaf_items;
     Workspace w;
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -149,6 +152,7 @@ Workspace carve(void *base, long long n_items, long long n_leaf_items, int batch
     w.node_bonus = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * n_items));
     w.stats = reinterpret_cast<NodeStats *>(take(sizeof(NodeStats) * n_items));
     w.leaf_part = reinterpret_cast<float2 *>(take(sizeof(float2) * kLeafEntries * n_leaf_items));
+    w.single_part = reinterpret_cast<float4 *>(take(sizeof(float4) * kLeafEntries * n_internal_items));
     w.status = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
     w.path[0] = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
     w.path[1] = reinterpret_cast<int32_t *>(take(sizeof(int32_t) * (batch > 0 ? batch : 1)));
@@ -412,20 +416,38 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     const size_t smem = node_smem_bytes(elem_bytes(d->dtype), cfg.ept, cfg.direct);
     const int resident = resident_clusters(fn, cfg.cluster, smem, c.stream, cfg.threads);
     if (resident < 1) return MCSD_ERR_CUDA;
-    const long long n_clusters = n_items < resident ? n_items : resident;
+    // Large launches of the all-node form: the cluster kernel takes only the nodes with two or more
+    // children; the rows of all others are streamed for their statistics by a kernel of its own and
+    // the single test of the nodes with one child is made from those (MCSD_OPT_SPLIT: 1 never, 2 always).
+    int n_stream = 0, n_keep = 0, n_single = 0;
+    uint16_t stream_nodes[MCSD_MAX_NODES], keep_nodes[MCSD_MAX_NODES];
+    for (int n = 0; n < d->n_nodes; ++n) {
+        const int k = n < d->n_internal ? c.plan.child_count[n] : 0;
+        if (k >= 2) keep_nodes[n_keep++] = static_cast<uint16_t>(n);
+        else stream_nodes[n_stream++] = static_cast<uint16_t>(n);
+        n_single += k == 1;
+    }
+    const int split_opt = g_opt.v[MCSD_OPT_SPLIT];
+    const bool split = !path && n_stream > 0 && split_opt != 1 &&
+        (split_opt == 2 || n_items >= 8LL * resident);
+    const int n_list = split ? n_keep : d->n_nodes;
+    const long long n_cluster_items = path ? n_items : static_cast<long long>(d->batch) * n_list;
+    const long long n_clusters = n_cluster_items < resident ? n_cluster_items : resident;
 
     NodeParams p = {};
     p.target = target; p.draft = draft; p.cand = cand; p.unif = unif;
     p.node_accept = c.node_accept; p.node_ratio = d->node_ratio;
-    p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part;
+    p.stats = c.ws.stats; p.leaf_part = c.ws.leaf_part; p.single_part = c.ws.single_part;
     p.ld_t = d->ld_target; p.ld_d = d->ld_draft;
     p.wait_polls = g_opt.v[MCSD_OPT_WAIT_POLLS] > 0 ? static_cast<uint32_t>(g_opt.v[MCSD_OPT_WAIT_POLLS]) : kWaitPolls;
     p.test_extra_tx = static_cast<uint32_t>(g_opt.v[MCSD_OPT_TEST_EXTRA_TX]) & ~15u;
     p.B = d->batch; p.n_nodes = d->n_nodes; p.n_internal = d->n_internal; p.V = d->vocab;
     p.slice = cfg.slice;
-    p.n_items = static_cast<int32_t>(n_items);
-    p.step_b = static_cast<int32_t>(path ? n_clusters : n_clusters / d->n_nodes);
-    p.step_n = static_cast<int32_t>(path ? 0 : n_clusters % d->n_nodes);
+    p.n_items = static_cast<int32_t>(n_cluster_items);
+    p.n_list = path ? 1 : n_list;
+    p.step_b = static_cast<int32_t>(path ? n_clusters : (n_list ? n_clusters / n_list : 0));
+    p.step_n = static_cast<int32_t>(path ? 0 : (n_list ? n_clusters % n_list : 0));
+    for (int i = 0; i < d->n_nodes; ++i) p.item_node[i] = static_cast<uint16_t>(split ? (i < n_keep ? keep_nodes[i] : 0) : i);
     p.mode = mode;
     const double scale_d = 1.4426950408889634 / static_cast<double>(T);
     p.scale = static_cast<float>(scale_d);
@@ -445,11 +467,84 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
-        cudaGetLastError();
-        return MCSD_ERR_CUDA;
+    if (n_clusters > 0) {
+        if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
+            cudaGetLastError();
+            return MCSD_ERR_CUDA;
+        }
+        g_last_launches += 1;
     }
-    g_last_launches += 1;
+    if (split) {
+        StreamParams sp = {};
+        sp.target = target; sp.draft = draft;
+        sp.leaf_part = c.ws.leaf_part; sp.single_part = c.ws.single_part; sp.node_accept = c.node_accept;
+        sp.ld_t = d->ld_target; sp.ld_d = d->ld_draft;
+        sp.B = d->batch; sp.n_nodes = d->n_nodes; sp.n_internal = d->n_internal; sp.V = d->vocab;
+        sp.n_entries = cfg.cluster * (cfg.threads / 32);   // every entry the walk and decide stages read, empty runs included
+        sp.n_list = n_stream;
+        sp.vector_ok = cfg.direct ? 0 : 1;
+        sp.scale = p.scale;
+        for (int i = 0; i < n_stream; ++i) sp.item_node[i] = stream_nodes[i];
+        int dev = 0, n_sm = 148;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        const long long warps = static_cast<long long>(d->batch) * n_stream * sp.n_entries;
+        long long ctas = (warps + 3) / 4;
+        if (ctas > static_cast<long long>(n_sm) * 64) ctas = static_cast<long long>(n_sm) * 64;
+        const unsigned grid = static_cast<unsigned>(ctas);
+        switch (d->dtype * 100 + cfg.ept) {
+        case MCSD_DTYPE_F32 * 100 + 16: stream_stats_kernel<MCSD_DTYPE_F32, 16><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        case MCSD_DTYPE_F32 * 100 + 32: stream_stats_kernel<MCSD_DTYPE_F32, 32><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        case MCSD_DTYPE_F32 * 100 + 64: stream_stats_kernel<MCSD_DTYPE_F32, 64><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        case MCSD_DTYPE_BF16 * 100 + 16: stream_stats_kernel<MCSD_DTYPE_BF16, 16><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        case MCSD_DTYPE_BF16 * 100 + 32: stream_stats_kernel<MCSD_DTYPE_BF16, 32><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        case MCSD_DTYPE_BF16 * 100 + 64: stream_stats_kernel<MCSD_DTYPE_BF16, 64><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        case MCSD_DTYPE_F16 * 100 + 16: stream_stats_kernel<MCSD_DTYPE_F16, 16><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        case MCSD_DTYPE_F16 * 100 + 32: stream_stats_kernel<MCSD_DTYPE_F16, 32><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        default: stream_stats_kernel<MCSD_DTYPE_F16, 64><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
+        }
+        if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
+        g_last_launches += 1;
+    }
+    // ... and the one test of every node with exactly one child is made from those statistics
+    if (split && n_single > 0) {
+        SingleParams sp = {};
+        sp.target = target; sp.draft = draft; sp.cand = cand; sp.unif = unif;
+        sp.single_part = c.ws.single_part; sp.node_accept = c.node_accept; sp.node_ratio = d->node_ratio;
+        sp.stats = c.ws.stats;
+        sp.ld_t = d->ld_target; sp.ld_d = d->ld_draft;
+        sp.B = d->batch; sp.n_nodes = d->n_nodes; sp.n_internal = d->n_internal; sp.V = d->vocab;
+        sp.n_entries = cfg.cluster * (cfg.threads / 32);
+        sp.mode = mode;
+        sp.pdl = g_opt.v[MCSD_OPT_PDL] ? 1 : 0;
+        sp.scale = p.scale; sp.scale_lo = p.scale_lo;
+        std::memcpy(sp.child_first, c.plan.child_first, sizeof(sp.child_first));
+        std::memcpy(sp.child_count, c.plan.child_count, sizeof(sp.child_count));
+        using SingleKernel = void (*)(const SingleParams);
+        SingleKernel sk = d->dtype == MCSD_DTYPE_F32 ? single_decide_kernel<MCSD_DTYPE_F32>
+                        : d->dtype == MCSD_DTYPE_BF16 ? single_decide_kernel<MCSD_DTYPE_BF16>
+                                                      : single_decide_kernel<MCSD_DTYPE_F16>;
+        int dev = 0, n_sm = 148;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        const long long warps = static_cast<long long>(d->batch) * d->n_internal;
+        long long ctas = (warps + 3) / 4;
+        if (ctas > static_cast<long long>(n_sm) * 16) ctas = static_cast<long long>(n_sm) * 16;
+        cudaLaunchConfig_t sc = {};
+        sc.gridDim = dim3(static_cast<unsigned>(ctas));
+        sc.blockDim = dim3(kNodeThreads);
+        sc.stream = c.stream;
+        cudaLaunchAttribute sa[1];
+        sa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        sa[0].val.programmaticStreamSerializationAllowed = 1;
+        sc.attrs = sa;
+        sc.numAttrs = sp.pdl ? 1 : 0;
+        if (cudaLaunchKernelEx(&sc, sk, sp) != cudaSuccess) {
+            cudaGetLastError();
+            return MCSD_ERR_CUDA;
+        }
+        g_last_launches += 1;
+    }
     return MCSD_OK;
 }
 

@@ -46,11 +46,18 @@ struct NodeParams {
     float *node_ratio;  // may be null
     NodeStats *stats;   // [B][n_nodes], written for nodes with children
     float2 *leaf_part;  // [B][n_nodes - n_internal][kLeafEntries] per-warp (reference, sum) of every leaf row
+    float4 *single_part; // [B][n_internal][kLeafEntries] per-warp (reference, sum) of both rows of every node
+                         // with exactly one child (all-node form): such a node is decided by one test
+                         // that needs no residual, so it is decided after the kernel, from these
     long long ld_t, ld_d;
     int32_t B, n_nodes, n_internal, V;
     int32_t slice;   // vocabulary elements owned by one CTA of the cluster
-    int32_t n_items; // B * n_nodes
-    int32_t step_b, step_n;  // quotient and remainder of (clusters in the grid) / n_nodes
+    int32_t n_items; // B * n_list
+    // The nodes of a tree this launch evaluates, in ascending order: all of them, or (large
+    // launches of the all-node form) only those with two or more children, the others being left
+    // to stream_stats_kernel.  Item i is (sequence i / n_list, node item_node[i % n_list]).
+    int32_t n_list;
+    int32_t step_b, step_n;  // quotient and remainder of (clusters in the grid) / n_list
     // Path mode: the items are the sequences (step_b = clusters in the grid, step_n = 0); a cluster
     // follows each of its sequences from the root through the accepted children and evaluates
     // only the nodes on that walk.
@@ -61,6 +68,7 @@ struct NodeParams {
     float scale_lo;  // ... and what the rounding dropped (for the candidates' own probabilities)
     uint16_t child_first[MCSD_MAX_NODES];
     uint8_t child_count[MCSD_MAX_NODES];
+    uint16_t item_node[MCSD_MAX_NODES];
 };
 
 // ------------------------------------------------------------------ checked build

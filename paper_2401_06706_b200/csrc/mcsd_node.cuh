@@ -68,6 +68,14 @@ constexpr size_t node_smem_bytes(int elem_bytes, int ept, bool direct) {
 // Every decision of the rejection loop is taken by every warp of the cluster from
 // bit-identical inputs, so all CTAs of a cluster execute the same number of exchange
 // rounds (the byte counts the exchange barriers are armed with rely on it).
+//
+// Which nodes need this kernel at all: those with two or more children, whose rows must stay on
+// chip for the residual sums.  A leaf tests nothing; a node with one child needs no residual (the
+// sum after a node's last rejection is formed by the walk stage, and only where a walk stops).
+// Large launches of the all-node form therefore give this kernel only the nodes with two or more
+// children (NodeParams::item_node) and leave the others to stream_stats_kernel and
+// single_decide_kernel below; small launches, where a further kernel launch costs more than it
+// saves, and the path form take every node through this kernel.
 template <int DT, int EPT, bool DIRECT, bool PATH>
 __global__ void __launch_bounds__(kNodeThreads, node_min_blocks(EPT))
 node_kernel(const __grid_constant__ NodeParams P)
@@ -96,6 +104,10 @@ node_kernel(const __grid_constant__ NodeParams P)
     __shared__ __align__(8) unsigned long long full_bar;
     __shared__ CandRing ring;
     __shared__ Action act[2];
+    // the leader's view of the node's candidates (candidate i: its p and q times K, its uniform), kept
+    // in shared memory rather than in registers that every warp of the kernel would have to set aside
+    __shared__ double s_px[MCSD_MAX_CHILDREN], s_qx[MCSD_MAX_CHILDREN];
+    __shared__ float s_u[MCSD_MAX_CHILDREN];
 
     const int tid = threadIdx.x, lane = tid & 31;
     // (broadcast from lane 0 so that the compiler knows the warp index is warp-uniform)
@@ -178,12 +190,12 @@ node_kernel(const __grid_constant__ NodeParams P)
         ++round;
     };
 
-    // (sequence, node) of the items this cluster visits: the current one and the two after
-    // it, advanced by the precomputed quotient and remainder of the stride
-    auto advance = [&](int &b, int &n) {
+    // (sequence, position in the node list) of the items this cluster visits: the current one
+    // and the two after it, advanced by the precomputed quotient and remainder of the stride
+    auto advance = [&](int &b, int &i) {
         b += P.step_b;
-        n += P.step_n;
-        if (n >= P.n_nodes) { n -= P.n_nodes; ++b; }
+        i += P.step_n;
+        if (i >= P.n_list) { i -= P.n_list; ++b; }
     };
 
     // ---- candidate pipeline (the fetch warp only) -------------------------------------------
@@ -220,10 +232,9 @@ node_kernel(const __grid_constant__ NodeParams P)
         }
     };
 
-    int b = cluster_id / P.n_nodes, n = cluster_id - b * P.n_nodes;  // current item
+    int b = cluster_id / P.n_list, ipos = cluster_id - b * P.n_list;  // current item: sequence, list position
+    int n = P.item_node[ipos];
     if (PATH) { b = cluster_id; n = 0; }  // every walk starts at the root
-    int b1 = b, n1 = n;                                              // the next one
-    advance(b1, n1);
     uint32_t it = 0;  // iteration count of this cluster
     bool prev_internal = false;
     if (!PATH && warp == kFetchWarp) {
@@ -231,7 +242,9 @@ node_kernel(const __grid_constant__ NodeParams P)
         cp_async_wait_all();
         __syncwarp();
         fetch_logits(b, n, 0, 0);
-        fetch_tokens(b1, n1, 1);
+        int b1 = b, i1 = ipos;           // (the items that follow are found again from the current one when needed)
+        advance(b1, i1);
+        fetch_tokens(b1, P.item_node[i1], 1);
     }
     if (kPrefetch && tid == 0 && b < P.B && bulk_bytes) {
         bulk_prefetch_l2(t_slice(static_cast<long long>(b) * P.n_nodes + n), bulk_bytes);
@@ -273,19 +286,22 @@ node_kernel(const __grid_constant__ NodeParams P)
         // data of the next two items
         auto look_ahead = [&]() {
             if (!PATH && warp == kFetchWarp) {
+                int b1 = b, i1 = ipos;
+                advance(b1, i1);
+                const int n1 = P.item_node[i1];
                 if (kPrefetch && lane == 0 && b1 < P.B && bulk_bytes) {
                     bulk_prefetch_l2(t_slice(static_cast<long long>(b1) * P.n_nodes + n1), bulk_bytes);
                     if (n1 < P.n_internal) bulk_prefetch_l2(d_slice(b1, n1), bulk_bytes);
                 }
                 fetch_logits(b1, n1, (it + 1) % 3u, s2 ^ 1);
-                int b2 = b1, n2 = n1;
-                advance(b2, n2);
-                fetch_tokens(b2, n2, (it + 2) % 3u);
+                int b2 = b1, i2 = i1;
+                advance(b2, i2);
+                fetch_tokens(b2, P.item_node[i2], (it + 2) % 3u);
             }
         };
         auto next_item = [&]() {
-            b = b1; n = n1;
-            advance(b1, n1);
+            advance(b, ipos);
+            n = P.item_node[ipos];
         };
 
         // ---- target slice -> registers, as packed pairs
@@ -498,9 +514,7 @@ node_kernel(const __grid_constant__ NodeParams P)
         // leader state of the rejection loop, in units where W' = W * K, K = Z_t * Z_d:
         double c = 0.0, S = 1.0, Wk = 0.0, K = 0.0, c_try = 0.0;
         float c_prev = 0.f;  // c before the last rejection
-        double px = 0.0, qx = 0.0;  // lane i of the leader: candidate i's p and q, times K
-        int cand_i = 0, accepted = -1, my_tok = -1;
-        float u_acc = 2.f;
+        int cand_i = 0, accepted = -1;
         // tests candidates from cand_i on until one is accepted (returns 0), all are rejected
         // (returns 0) or one is rejected and its residual sum is needed (returns 1, c_try set).
         // The sum after the LAST rejection is not needed here (nothing is tested against that
@@ -508,14 +522,14 @@ node_kernel(const __grid_constant__ NodeParams P)
         auto leader_decide = [&]() -> int {
             while (cand_i < k) {
                 const int i = cand_i;
-                const int xi = __shfl_sync(0xffffffffu, my_tok, i);
-                const double ui = static_cast<double>(__shfl_sync(0xffffffffu, u_acc, i));
-                const double pxi = __shfl_sync(0xffffffffu, px, i), qxi = __shfl_sync(0xffffffffu, qx, i);
+                const int xi = ring.tok[s3][i];
+                const double ui = static_cast<double>(s_u[i]);
+                const double pxi = s_px[i], qxi = s_qx[i];
                 const bool valid = xi >= 0 && xi < P.V;
                 if (!valid) status_bits |= MCSD_STATUS_BAD_TOKEN;
                 // Algorithm 2: a token rejected earlier at this node has draft probability 0 now
                 const bool dup = P.mode == 1 &&
-                    (__ballot_sync(0xffffffffu, lane < i && my_tok == xi) != 0u);
+                    (__ballot_sync(0xffffffffu, lane < i && ring.tok[s3][lane] == xi) != 0u);
                 const bool zero_q = !valid || dup || !(qxi > 0.0) || !(Wk > 0.0);
                 double Pn = pxi - c * qxi;
                 Pn = Pn > 0.0 ? Pn : 0.0;
@@ -549,8 +563,8 @@ node_kernel(const __grid_constant__ NodeParams P)
             int int_t = 0, int_d = 0;
             bool cand_ok = false;
             if (lane < k) {
-                my_tok = ring.tok[s3][lane];
-                u_acc = fminf(ring.u[s3][lane], 1.f);  // supplied in place of r ~ U(0,1): not below 1 (NaN too) counts as 1
+                const int my_tok = ring.tok[s3][lane];
+                s_u[lane] = fminf(ring.u[s3][lane], 1.f);  // supplied in place of r ~ U(0,1): not below 1 (NaN too) counts as 1
                 cand_ok = my_tok >= 0 && my_tok < P.V;
                 if (cand_ok) {
                     const uint32_t wt = ring.tl[s2][lane], wd = ring.dl[s2][lane];
@@ -573,10 +587,12 @@ node_kernel(const __grid_constant__ NodeParams P)
             // px' = 2^(l_t*scale - R_t) * Z_d, qx' = 2^(l_d*scale - R_d) * Z_t
             K = static_cast<double>(Z_t) * static_cast<double>(Z_d);
             Wk = K;
-            if (cand_ok && t_ok && d_ok) {
-                px = static_cast<double>(frac_t) * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
-                qx = static_cast<double>(frac_d) * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
+            if (lane < k) {
+                const bool ok = cand_ok && t_ok && d_ok;
+                s_px[lane] = ok ? static_cast<double>(frac_t) * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d) : 0.0;
+                s_qx[lane] = ok ? static_cast<double>(frac_d) * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t) : 0.0;
             }
+            __syncwarp();
             const int more = leader_decide();
             if (lane == 0) {
                 act[round & 1u].stats = make_float4(R_t, R_d, t_ok ? 1.f / Z_t : 0.f, (t_ok && d_ok) ? Z_t / Z_d : 0.f);
@@ -668,6 +684,189 @@ node_kernel(const __grid_constant__ NodeParams P)
     if (poisoned) __nanosleep(20000);
     // no CTA may leave while a peer can still write into its shared memory
     cluster_sync_all();
+}
+
+// Large launches of the all-node form: the rows of the nodes that need no exchange (leaves: the
+// target row; nodes with one child: both rows) are only streamed for their statistics, and a
+// kernel that keeps nothing on chip does that with many more warps per SM and therefore far more
+// loads in flight than the cluster kernel can afford.  One warp per (sequence, node, run); runs,
+// lanes and the order of every sum are those of node_kernel, so the statistics are the same bit
+// for bit and go to the same places (leaf_part, single_part).
+struct StreamParams {
+    const void *target;
+    const void *draft;
+    float2 *leaf_part;
+    float4 *single_part;
+    int32_t *node_accept;   // -1 is written for every leaf
+    long long ld_t, ld_d;
+    int32_t B, n_nodes, n_internal, V, n_entries, n_list, vector_ok;
+    float scale;
+    uint16_t item_node[MCSD_MAX_NODES];   // leaves and nodes with one child, ascending
+};
+
+template <int DT, int EPT>
+__device__ __forceinline__ void stream_run(const unsigned char *row, int n_valid, bool vector_ok, float scale, int lane,
+                                           float &ref, float &z)
+{
+    using E = Elem<DT>;
+    constexpr int GV = E::kVec, NG = EPT / GV;
+    uint4 raw[NG];
+#pragma unroll
+    for (int j = 0; j < NG; ++j) {
+        const int x = (j * 32 + lane) * GV;
+        if (vector_ok && x + GV <= n_valid) {
+            raw[j] = ld_stream_v4(row + static_cast<size_t>(x) * E::kBytes);
+        } else {
+            // the ragged end (or rows without 16-byte alignment): element loads, -inf past the end,
+            // repacked so that both cases continue alike
+            float f[GV];
+#pragma unroll
+            for (int e = 0; e < GV; ++e) f[e] = (x + e < n_valid) ? E::load(row, x + e) : -INFINITY;
+            if constexpr (E::kBytes == 4) {
+                raw[j] = make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+            } else {
+                raw[j].x = E::to_bits(f[0]) | (E::to_bits(f[1]) << 16);
+                raw[j].y = E::to_bits(f[2]) | (E::to_bits(f[3]) << 16);
+                raw[j].z = E::to_bits(f[4]) | (E::to_bits(f[5]) << 16);
+                raw[j].w = E::to_bits(f[6]) | (E::to_bits(f[7]) << 16);
+            }
+        }
+    }
+    typename E::MaxAcc acc = E::max_init();
+#pragma unroll
+    for (int j = 0; j < NG; ++j) E::max_step(acc, raw[j]);
+    ref = int_ref(warp_max(E::max_final(acc)) * scale);
+    const float r0 = (ref == -INFINITY) ? 0.f : ref;
+    // four running sums, by element index modulo 4 in the thread's own order: what the packed
+    // accumulators of node_kernel hold
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+    for (int j = 0; j < NG; ++j) {
+        float f[GV];
+        E::unpack(raw[j], f);
+#pragma unroll
+        for (int e = 0; e < GV; e += 4) {
+            a0 += ex2f(fmaf(f[e], scale, -r0));
+            a1 += ex2f(fmaf(f[e + 1], scale, -r0));
+            a2 += ex2f(fmaf(f[e + 2], scale, -r0));
+            a3 += ex2f(fmaf(f[e + 3], scale, -r0));
+        }
+    }
+    z = (a0 + a2) + (a1 + a3);
+}
+
+template <int DT, int EPT>
+__global__ void __launch_bounds__(kNodeThreads, Elem<DT>::kBytes == 2 ? 8 : 4)
+stream_stats_kernel(const __grid_constant__ StreamParams P)
+{
+    using E = Elem<DT>;
+    constexpr int RUN = 32 * EPT;
+    const int lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const long long n_items = static_cast<long long>(P.B) * P.n_list * P.n_entries;
+    const long long warp_id = (static_cast<long long>(blockIdx.x) * kNodeThreads + threadIdx.x) >> 5;
+    const long long n_warps = (static_cast<long long>(gridDim.x) * kNodeThreads) >> 5;
+    for (long long item = warp_id; item < n_items; item += n_warps) {
+        const long long bi = item / P.n_entries;
+        const int e = static_cast<int>(item - bi * P.n_entries);
+        const int b = static_cast<int>(bi / P.n_list), n = P.item_node[bi - static_cast<long long>(b) * P.n_list];
+        int n_valid = P.V - e * RUN;    // (a run past the end of the vocabulary holds nothing: statistics (-inf, 0))
+        n_valid = n_valid > RUN ? RUN : (n_valid < 0 ? 0 : n_valid);
+        const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
+        const unsigned char *t_row = reinterpret_cast<const unsigned char *>(P.target) +
+            (node_idx * P.ld_t + static_cast<long long>(e) * RUN) * E::kBytes;
+        float rt, zt;
+        stream_run<DT, EPT>(t_row, n_valid, P.vector_ok != 0, P.scale, lane, rt, zt);
+        const float st = warp_sum(zt);
+        if (n >= P.n_internal) {
+            if (lane == 0) {
+                P.leaf_part[(static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * kLeafEntries + e] =
+                    make_float2(rt, st);
+                if (e == 0) P.node_accept[node_idx] = -1;
+            }
+            continue;
+        }
+        const unsigned char *d_row = reinterpret_cast<const unsigned char *>(P.draft) +
+            ((static_cast<long long>(b) * P.n_internal + n) * P.ld_d + static_cast<long long>(e) * RUN) * E::kBytes;
+        float rd, zd;
+        stream_run<DT, EPT>(d_row, n_valid, P.vector_ok != 0, P.scale, lane, rd, zd);
+        const float sd = warp_sum(zd);
+        if (lane == 0)
+            P.single_part[(static_cast<long long>(b) * P.n_internal + n) * kLeafEntries + e] = make_float4(rt, st, rd, sd);
+    }
+}
+
+// The one test of every node that has exactly one child (all-node form), from the per-run
+// statistics the node kernel left: one warp per node.  The arithmetic is the leader warp's.
+struct SingleParams {
+    const void *target;
+    const void *draft;
+    const int32_t *cand;
+    const float *unif;
+    const float4 *single_part;
+    int32_t *node_accept;
+    float *node_ratio;   // may be null
+    NodeStats *stats;
+    long long ld_t, ld_d;
+    int32_t B, n_nodes, n_internal, V, n_entries, mode, pdl;
+    float scale, scale_lo;
+    uint16_t child_first[MCSD_MAX_NODES];
+    uint8_t child_count[MCSD_MAX_NODES];
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kNodeThreads)
+single_decide_kernel(const __grid_constant__ SingleParams P)
+{
+    using E = Elem<DT>;
+    const int lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+    const long long n_items = static_cast<long long>(P.B) * P.n_internal;
+    const long long warp_id = (static_cast<long long>(blockIdx.x) * kNodeThreads + threadIdx.x) >> 5;
+    const long long n_warps = (static_cast<long long>(gridDim.x) * kNodeThreads) >> 5;
+    for (long long item = warp_id; item < n_items; item += n_warps) {
+        const int b = static_cast<int>(item / P.n_internal), n = static_cast<int>(item - static_cast<long long>(b) * P.n_internal);
+        if (P.child_count[n] != 1) continue;
+        const long long node_idx = static_cast<long long>(b) * P.n_nodes + n;
+        const int first = P.child_first[n];
+        const float4 ent = lane < P.n_entries ? P.single_part[item * kLeafEntries + lane]
+                                              : make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
+        const float R_t = warp_max(ent.x), R_d = warp_max(ent.z);
+        const float Z_t = warp_sum(ent.y * exp2i(ent.x - R_t));
+        const float Z_d = warp_sum(ent.w * exp2i(ent.z - R_d));
+        if (lane != 0) continue;
+        const bool t_ok = Z_t > 0.f && Z_t < INFINITY, d_ok = Z_d > 0.f && Z_d < INFINITY;
+        int status_bits = (!t_ok || !d_ok) ? MCSD_STATUS_DEGENERATE : 0;
+        const long long ci = static_cast<long long>(b) * P.n_nodes + first;
+        const int xi = P.cand[ci];
+        const double ui = static_cast<double>(fminf(P.unif[2 * ci], 1.f));
+        const bool valid = xi >= 0 && xi < P.V;
+        if (!valid) status_bits |= MCSD_STATUS_BAD_TOKEN;
+        const double K = static_cast<double>(Z_t) * static_cast<double>(Z_d);
+        double px = 0.0, qx = 0.0;
+        if (valid && t_ok && d_ok) {
+            const float lt = E::load(reinterpret_cast<const unsigned char *>(P.target) + node_idx * P.ld_t * E::kBytes, xi);
+            const float ld = E::load(reinterpret_cast<const unsigned char *>(P.draft) +
+                                     (static_cast<long long>(b) * P.n_internal + n) * P.ld_d * E::kBytes, xi);
+            int int_t, int_d;
+            const float frac_t = split_exp2(lt, P.scale, P.scale_lo, int_t);
+            const float frac_d = split_exp2(ld, P.scale, P.scale_lo, int_d);
+            px = static_cast<double>(frac_t) * exp2i_d(int_t - static_cast<int>(R_t)) * static_cast<double>(Z_d);
+            qx = static_cast<double>(frac_d) * exp2i_d(int_d - static_cast<int>(R_d)) * static_cast<double>(Z_t);
+        }
+        // the first test of a node: c = 0, S = 1, W = 1 (in units of K)
+        const double Wk = K;
+        const bool zero_q = !valid || !(qx > 0.0) || !(Wk > 0.0);
+        const double Pn = px > 0.0 ? px : 0.0;
+        const bool accept = !zero_q && ui * qx * K <= Pn * Wk;
+        if (P.node_ratio) P.node_ratio[ci] = zero_q ? -1.f : static_cast<float>(Pn / (qx * K / Wk));
+        // rejected: the residual moves on to c = S / W = 1 (0 where there is no q); its sum is the walk stage's
+        const float c_final = accept ? 0.f : ((Wk > 0.0) ? 1.f : 0.f);
+        P.node_accept[node_idx] = accept ? first : -1;
+        reinterpret_cast<float4 *>(&P.stats[node_idx])[0] = make_float4(R_t, R_d, Z_t, Z_d);
+        reinterpret_cast<float4 *>(&P.stats[node_idx])[1] = make_float4(c_final, 0.f, __int_as_float(status_bits), 0.f);
+    }
 }
 
 }  // namespace mcsd

@@ -57,11 +57,11 @@ class Guards:
 @contextlib.contextmanager
 def library_options(**opts):
     """Sets MCSD_OPT_* overrides (cluster=, ept=, direct=, sample_ahead=, wait_polls=, test_extra_tx=, pdl=)
-    for the duration of a block and restores what was there before."""
+    (and split=) for the duration of a block and restores what was there before."""
     ids = {"cluster": binding.OPT_CLUSTER, "ept": binding.OPT_EPT, "direct": binding.OPT_DIRECT,
            "sample_ahead": binding.OPT_SAMPLE_AHEAD, "wait_polls": binding.OPT_WAIT_POLLS,
            "test_extra_tx": binding.OPT_TEST_EXTRA_TX, "pdl": binding.OPT_PDL,
-           "test_shrink_ranges": binding.OPT_TEST_SHRINK_RANGES}
+           "test_shrink_ranges": binding.OPT_TEST_SHRINK_RANGES, "split": binding.OPT_SPLIT}
     before = {k: binding.mcsd_get_option(ids[k]) for k in opts}
     try:
         for k, val in opts.items():

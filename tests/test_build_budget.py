@@ -1,7 +1,7 @@
 """Register budget of the dominant kernel, checked at build time (nvcc cross-compiles without a
 GPU): four CTAs of 128 threads per SM need at most 128 registers per thread, and the all-node
-variants for 64 elements per thread must not spill with 2-byte logits (their CTAs leave almost no
-L1 for spill traffic) and only marginally with 4-byte logits."""
+variants for 64 elements per thread may spill a few words at most (with 2-byte logits their CTAs
+leave almost no L1 for spill traffic: a variant that spilled 48 bytes lost 15 %)."""
 import os
 import re
 import shutil
@@ -33,5 +33,5 @@ def test_headline_node_kernels_fit_their_register_budget(tmp_path):
     assert len(blocks) == 3, out
     for _, dtype, st, ld, regs in blocks:
         assert int(regs) <= 128
-        limit = 0 if dtype in ("1", "2") else 128
+        limit = 16 if dtype in ("1", "2") else 32
         assert int(st) <= limit and int(ld) <= limit, (dtype, st, ld)

@@ -111,6 +111,27 @@ def test_forced_cluster_shapes(cluster, ept, dtype):
     assert_parity(inp, out)
 
 
+@pytest.mark.parametrize("dtype,vocab,kconfig,mode", [("bf16", 32000, "4x2x2x1", 1), ("fp32", 32001, "2x1x1", 0),
+                                                       ("fp16", 50272, "2x2x2x2", 1), ("fp32", 1000, "4x1", 0),
+                                                       ("bf16", 9000, "1x1x1", 0), ("fp16", 5003, "3x2x1", 1)])
+def test_split_launch_equals_single_launch(dtype, vocab, kconfig, mode):
+    """Large launches give the cluster kernel only the nodes with two or more children and stream
+    the rows of the others with a kernel of its own; the results must be those of the single
+    launch bit for bit (same runs, same order of every sum), and the oracle's."""
+    w = synth.Workload("split", 7, vocab, kconfig, dtype, "normal", 2.5, 0.9, 1.2, 0.9, mode, 4500 + vocab)
+    inp = synth.make_inputs(w, "cuda")
+    outs = []
+    for split in (1, 2):                      # 1: never, 2: always
+        with library_options(split=split):
+            _, out = run_library(inp)
+            outs.append([to_np(x).copy() for x in (out.accept_len, out.tokens, out.residual, out.node_accept,
+                                                   out.node_bonus, out.status, out.node_ratio)])
+            assert_parity(inp, out)
+            assert binding.mcsd_last_launch_count() >= 1
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b, equal_nan=True)
+
+
 def test_direct_path_matches_bulk_copy_path():
     w = synth.Workload("direct", 6, 32000, "4x2", "bf16", "normal", 2.5, 0.8, 1.5, 1.0, 0, 99)
     inp = synth.make_inputs(w, "cuda")
