@@ -48,23 +48,47 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-TRAFFIC_PROFILE = os.path.join("profiles", "node_kernel_cfg5_batch16_ncu_full.md")
+TRAFFIC_PROFILES = {"stream_stats_kernel": os.path.join("profiles", "stream_stats_kernel_cfg5_batch16_ncu_full.md"),
+                    "node_kernel": os.path.join("profiles", "node_kernel_cfg5_batch16_ncu_full.md")}
 
 
-def recorded_traffic(units: int):
-    """DRAM bytes per launch of the node kernel from the committed ncu summary, scaled by the
-    number of tree nodes per launch (the capture ran a smaller batch of the same workload and
-    the traffic grows in proportion to the rows read).  Returns (bytes, source, scale factor);
-    bytes is None when the summary is missing."""
+def recorded_traffic(kernel: str, units: int):
+    """DRAM bytes per launch of a kernel from its committed ncu summary, scaled by the logit rows the
+    launch reads (the capture ran a smaller batch of the same workload and the traffic grows in
+    proportion to the rows read).  Returns (bytes, source, scale factor); bytes is None when there
+    is no summary with a `dram_bytes_per_launch=... units_per_launch=...` line."""
     import re
+    prof = TRAFFIC_PROFILES.get(kernel)
     try:
-        with open(os.path.join(ROOT, TRAFFIC_PROFILE)) as f:
+        with open(os.path.join(ROOT, prof)) as f:
             m = re.search(r"dram_bytes_per_launch=(\d+) units_per_launch=(\d+)", f.read())
         scale = units / float(m.group(2))
-        return float(m.group(1)) * scale, (f"{TRAFFIC_PROFILE}: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture "
-                                            f"at {m.group(2)} tree nodes per launch, scaled by the nodes per launch"), scale
+        return float(m.group(1)) * scale, (f"{prof}: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture "
+                                            f"at {m.group(2)} logit rows per launch, scaled by the rows per launch"), scale
     except Exception:
-        return None, "no recorded capture", None
+        return None, "no recorded capture of this kernel", None
+
+
+def kernel_breakdown(binding, call, n_calls: int):
+    """Device time of every kernel of the step, from CUDA events the library records around its own
+    launches on the launching stream (MCSD_OPT_TIME_KERNELS), over n_calls further calls; programmatic
+    dependent launch is switched off meanwhile so that the intervals do not overlap."""
+    names = ("node_kernel", "stream_stats_kernel", "single_decide_kernel", "walk_kernel")
+    before = (binding.mcsd_get_option(binding.OPT_TIME_KERNELS), binding.mcsd_get_option(binding.OPT_PDL))
+    binding.mcsd_set_option(binding.OPT_TIME_KERNELS, 1)
+    binding.mcsd_set_option(binding.OPT_PDL, 0)
+    tot, cnt = [0.0] * 4, [0] * 4
+    try:
+        for _ in range(n_calls):
+            call()
+            for i, ms in enumerate(binding.mcsd_last_kernel_times()):
+                if ms is not None:
+                    tot[i] += ms
+                    cnt[i] += 1
+    finally:
+        binding.mcsd_set_option(binding.OPT_TIME_KERNELS, before[0])
+        binding.mcsd_set_option(binding.OPT_PDL, before[1])
+    return {names[i]: tot[i] / cnt[i] for i in range(4) if cnt[i]}
 
 
 class ClockSampler:
@@ -366,17 +390,46 @@ def run_cuda(args):
     node_ms_avg = sum(node_ms) / len(node_ms)
     achieved = algo_bytes / (node_ms_avg * 1e-3) / 1e9
     peak, peak_kind = measured_peaks()
-    traffic, traffic_source, traffic_scale = (recorded_traffic(w.batch * st["n_nodes"])
-                                              if (w.name == "cfg5_largest" and w.dtype == "fp32" and args.form == "all_node")
+    # The node stage of a large launch is three kernels (the cluster kernel for the nodes with two or
+    # more children, the streaming kernel for the rows of all others, the single-test kernel).  The
+    # roofline object is for the DOMINANT one, with its own algorithmic bytes and its own duration from
+    # CUDA events around it; the whole stage follows under "stage".
+    es = inp.target.element_size()
+    _, child_count = synth.children_ranges(inp.parent)
+    n_keep = int((child_count >= 2).sum())
+    n_single = int((child_count == 1).sum())
+    n_leaf = st["n_nodes"] - st["n_internal"]
+    stage = {"kernels": "argmax_kernel" if w.temperature == 0 else "node_kernel + stream_stats_kernel + single_decide_kernel",
+             "ms_avg": node_ms_avg, "ms_min": min(node_ms), "algorithmic_bytes": algo_bytes, "achieved": achieved,
+             "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+             "step_share": node_ms_avg / ms_per_step}
+    per_kernel = None
+    kernel, k_ms, k_bytes, k_rows = ("node_kernel" if w.temperature > 0 else "argmax_kernel"), node_ms_avg, algo_bytes, None
+    if args.form == "all_node" and w.temperature > 0 and world == 1:
+        per_kernel = kernel_breakdown(binding, lambda: ver.mcsd_verify(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode),
+                                      min(args.steps, 20))
+        split = "stream_stats_kernel" in per_kernel
+        rows = {"node_kernel": w.batch * (2 * n_keep if split else st["n_nodes"] + st["n_internal"]),
+                "stream_stats_kernel": w.batch * (n_leaf + 2 * n_single)}
+        bytes_of = {k: rows[k] * w.vocab * es + (12 * w.batch * (n_keep if split else st["n_nodes"]) if k == "node_kernel" else 0)
+                    for k in rows}
+        kernel = max((k for k in per_kernel if k in rows), key=lambda k: per_kernel[k])
+        k_ms, k_bytes, k_rows = per_kernel[kernel], bytes_of[kernel], rows[kernel]
+        stage["per_kernel_ms"] = per_kernel
+        stage["per_kernel_gbs"] = {k: bytes_of[k] / (per_kernel[k] * 1e-3) / 1e9 for k in rows if k in per_kernel}
+    traffic, traffic_source, traffic_scale = (recorded_traffic(kernel, k_rows)
+                                              if (w.name == "cfg5_largest" and w.dtype == "fp32" and k_rows)
                                               else (None, "no capture of this kernel variant and workload", None))
-    roofline = {"bound": "hbm", "kernel": ("node_kernel" if w.temperature > 0 else "argmax_kernel") +
-                (" (one launch per level; the figure covers the whole call, which is bound by launch and "
-                 "exchange latency, not by HBM)" if args.form == "path" else ""),
-                "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_avg": node_ms_avg,
-                "kernel_ms_min": min(node_ms), "step_share": node_ms_avg / ms_per_step,
-                "traffic": traffic, "traffic_source": traffic_source, "traffic_scale": traffic_scale}
+    k_achieved = k_bytes / (k_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": kernel +
+                (" (the figure covers the whole call, which is bound by launch and exchange latency, not by HBM)"
+                 if args.form == "path" else ""),
+                "achieved": k_achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": k_achieved / peak, "frac_of_nominal_8TBs": k_achieved / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_launch": k_bytes, "kernel_ms_avg": k_ms,
+                "step_share": k_ms / ms_per_step,
+                "traffic": traffic, "traffic_source": traffic_source, "traffic_scale": traffic_scale,
+                "stage": stage}
 
     # the same steps again, many more of them: the power cap pulls the SM clock down after the first
     # hundred milliseconds, and the kernel's time follows the clock.  Clocks come from the sampler;
@@ -384,13 +437,14 @@ def run_cuda(args):
     sustained = None
     if args.sustained_steps > 0 and world == 1:
         s_ms, s_node, s_clk = timed_steps(step, args.sustained_steps, None, dev, torch.cuda.current_device())
-        k_ms = sum(s_node) / len(s_node)
-        sustained = {"steps": args.sustained_steps, "ms_per_step": s_ms / args.sustained_steps, "kernel_ms_avg": k_ms,
-                     "achieved": algo_bytes / (k_ms * 1e-3) / 1e9, "frac": algo_bytes / (k_ms * 1e-3) / 1e9 / peak,
+        s_k_ms = sum(s_node) / len(s_node)
+        sustained = {"steps": args.sustained_steps, "ms_per_step": s_ms / args.sustained_steps, "stage_ms_avg": s_k_ms,
+                     "what": "the whole node stage (all its kernels) over its algorithmic bytes",
+                     "achieved": algo_bytes / (s_k_ms * 1e-3) / 1e9, "frac": algo_bytes / (s_k_ms * 1e-3) / 1e9 / peak,
                      "sm_mhz": s_clk["sm_mhz"] if s_clk else None, "reasons": s_clk["reasons"] if s_clk else None,
                      "power_w_max": s_clk.get("power_w_max") if s_clk else None,
-                     "kernel_ms_x_mhz": (k_ms * s_clk["sm_mhz"]) if (s_clk and s_clk["sm_mhz"]) else None,
-                     "timed_region_kernel_ms_x_mhz": (node_ms_avg * clocks["sm_mhz"]) if (clocks and clocks["sm_mhz"]) else None}
+                     "stage_ms_x_mhz": (s_k_ms * s_clk["sm_mhz"]) if (s_clk and s_clk["sm_mhz"]) else None,
+                     "timed_region_stage_ms_x_mhz": (node_ms_avg * clocks["sm_mhz"]) if (clocks and clocks["sm_mhz"]) else None}
 
     # end to end through the host-buffer entry point: pinned host inputs, copies inside
     e2e = None
@@ -474,9 +528,12 @@ def half_record(w, dev, args, peak):
     ms, node_ms, clk = timed_steps(step, n, None, dev, torch.cuda.current_device())
     algo = inp.logit_bytes() + 12 * w.batch * st["n_nodes"]
     k_ms = sum(node_ms) / len(node_ms)
-    rec = {"logit_dtype": w.dtype, "steps": n, "ms_per_step": ms / n, "kernel_ms_avg": k_ms, "kernel_ms_min": min(node_ms),
-           "algorithmic_bytes_per_launch": algo, "achieved": algo / (k_ms * 1e-3) / 1e9, "unit": "GB/s",
-           "frac": algo / (k_ms * 1e-3) / 1e9 / peak, "value": w.batch * st["n_draft"] / (ms / n * 1e-3), "clocks": clk}
+    rec = {"logit_dtype": w.dtype, "steps": n, "ms_per_step": ms / n, "stage_ms_avg": k_ms, "stage_ms_min": min(node_ms),
+           "what": "the whole node stage (all its kernels) over its algorithmic bytes",
+           "algorithmic_bytes": algo, "achieved": algo / (k_ms * 1e-3) / 1e9, "unit": "GB/s",
+           "frac": algo / (k_ms * 1e-3) / 1e9 / peak, "value": w.batch * st["n_draft"] / (ms / n * 1e-3), "clocks": clk,
+           "per_kernel_ms": kernel_breakdown(binding, lambda: ver.mcsd_verify(inp.target, inp.draft, inp.cand, inp.unif,
+                                                                              w.temperature, w.mode), 10)}
     if not args.no_cpu_baseline:
         # cpu_baseline leg of this sub-record: the oracle timed on the first sequences of these inputs;
         # what it computed is then compared with the kernels' output on those sequences

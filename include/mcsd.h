@@ -131,7 +131,11 @@ extern "C" {
 #define MCSD_OPT_SPLIT 8         /* the all-node form of mcsd_verify at temperature > 0 gives its cluster kernel only
                                     the nodes with two or more children and streams the rows of the others with a
                                     kernel of its own: 0 = for large launches (default), 1 = never, 2 = always    */
-#define MCSD_OPT_COUNT 9
+#define MCSD_OPT_TIME_KERNELS 9  /* 1: CUDA events are recorded around every kernel the verification entry points
+                                    launch (on desc->stream); see mcsd_last_kernel_times.  With programmatic dependent
+                                    launches a kernel's interval may overlap its predecessor's tail: measure with
+                                    MCSD_OPT_PDL 0 for disjoint intervals                                          */
+#define MCSD_OPT_COUNT 10
 
 typedef struct mcsd_desc {
     int32_t batch;      /* B: number of trees                                         */
@@ -476,6 +480,13 @@ int mcsd_tree_depth(const int32_t *tree_parent, int32_t n_nodes);
 /* Number of kernel launches the last successful mcsd_verify / stage call on this
  * host thread enqueued (for launch accounting in benchmarks). */
 int mcsd_last_launch_count(void);
+
+/* With MCSD_OPT_TIME_KERNELS set: device time in milliseconds of the kernels the last mcsd_verify /
+ * mcsd_verify_nodes / mcsd_verify_walk / mcsd_verify_path call of this host thread launched, from CUDA
+ * events on its stream (waits for them): ms[0] cluster kernel (argmax kernel at temperature 0, naive
+ * kernel in MCSD_MODE_NAIVE), ms[1] streaming statistics kernel, ms[2] single-test kernel, ms[3] walk
+ * kernel; -1 where no such kernel ran.  Returns how many were filled, or a negative MCSD_ERR_*. */
+int mcsd_last_kernel_times(float *ms, int32_t n);
 
 /* The checked build of the library (libmcsd_debug.so, compiled with MCSD_DEBUG_BOUNDS) verifies every
  * read of caller memory by the verification, walk, argmax, naive-sampling and candidate-sampling

@@ -28,8 +28,8 @@ EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_
            "mcsd_workspace_bytes", "mcsd_tree_depth", "mcsd_last_launch_count", "mcsd_status_string",
            "mcsd_version", "mcsd_set_option", "mcsd_get_option", "mcsd_release_host_staging",
            "mcsd_shard_columns", "mcsd_shard_workspace_bytes", "mcsd_shard_rounds", "mcsd_shard_partials",
-           "mcsd_shard_decide", "mcsd_shard_endpoint", "mcsd_shard_finish", "mcsd_shard_commit", "mcsd_debug_bounds_hits")
-OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL, OPT_TEST_SHRINK_RANGES, OPT_SPLIT = range(9)
+           "mcsd_shard_decide", "mcsd_shard_endpoint", "mcsd_shard_finish", "mcsd_shard_commit", "mcsd_debug_bounds_hits", "mcsd_last_kernel_times")
+OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL, OPT_TEST_SHRINK_RANGES, OPT_SPLIT, OPT_TIME_KERNELS = range(10)
 
 
 class McsdDesc(ctypes.Structure):
@@ -125,6 +125,8 @@ def load_library(path: Optional[str] = None):
     lib.mcsd_shard_finish.restype = ctypes.c_int
     lib.mcsd_shard_commit.argtypes = [sp, vp, vp, vp, vp]
     lib.mcsd_shard_commit.restype = ctypes.c_int
+    lib.mcsd_last_kernel_times.argtypes = [vp, i32]
+    lib.mcsd_last_kernel_times.restype = ctypes.c_int
     lib.mcsd_debug_bounds_hits.argtypes = [ctypes.c_int]
     lib.mcsd_debug_bounds_hits.restype = ctypes.c_longlong
     if path is None:
@@ -164,6 +166,15 @@ def mcsd_get_option(option: int) -> int:
     rc = load_library().mcsd_get_option(int(option))
     _check(rc if rc < 0 else 0)
     return rc
+
+
+def mcsd_last_kernel_times():
+    """[cluster / argmax / naive, streaming statistics, single test, walk] kernel milliseconds of the last call
+    (needs MCSD_OPT_TIME_KERNELS); None where no such kernel ran."""
+    ms = (ctypes.c_float * 4)()
+    rc = load_library().mcsd_last_kernel_times(ctypes.addressof(ms), 4)
+    _check(rc if rc < 0 else 0)
+    return [None if x < 0 else float(x) for x in ms]
 
 
 def mcsd_debug_bounds_hits(reset: bool = False) -> int:

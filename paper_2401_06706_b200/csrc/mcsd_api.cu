@@ -105,6 +105,43 @@ int plan_tree_cached(const int32_t *parent, int n_nodes, int n_internal, TreePla
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// MCSD_OPT_TIME_KERNELS: CUDA events around every kernel the verification entry points launch, on
+// the stream they are launched on; mcsd_last_kernel_times reads the last call's.  Slots: 0 cluster
+// (or argmax / naive) kernel, 1 streaming kernel, 2 single-test kernel, 3 walk kernel.
+constexpr int kTimeSlots = 4;
+struct KernelTimers {
+    cudaEvent_t ev[kTimeSlots][2] = {};
+    bool used[kTimeSlots] = {};
+    bool created = false;
+};
+thread_local KernelTimers g_timers;
+
+struct ScopedTimer {
+    int slot;
+    cudaStream_t stream;
+    bool on;
+    ScopedTimer(int s, cudaStream_t st) : slot(s), stream(st), on(g_opt.v[MCSD_OPT_TIME_KERNELS] != 0)
+    {
+        if (!on) return;
+        if (!g_timers.created) {
+            for (auto &pair : g_timers.ev)
+                for (auto &e : pair) cudaEventCreate(&e);
+            g_timers.created = true;
+        }
+        cudaEventRecord(g_timers.ev[slot][0], stream);
+    }
+    ~ScopedTimer()
+    {
+        if (!on) return;
+        cudaEventRecord(g_timers.ev[slot][1], stream);
+        g_timers.used[slot] = true;
+    }
+};
+void reset_timers()
+{
+    for (bool &u : g_timers.used) u = false;
+}
+
 // Checked build: the address ranges the kernels of the next launches on `stream` may read.  An
 // empty list switches the checks off (kernels whose inputs are not registered).
 struct Range { const void *p; size_t bytes; };
@@ -332,6 +369,7 @@ int prepare(const mcsd_desc *d, const int32_t *parent, Call *c)
     c->node_bonus = d->node_bonus ? d->node_bonus : c->ws.node_bonus;
     c->status = d->out_status ? d->out_status : c->ws.status;
     c->stream = static_cast<cudaStream_t>(d->stream);
+    if (g_opt.v[MCSD_OPT_TIME_KERNELS]) reset_timers();
     return MCSD_OK;
 }
 
@@ -397,6 +435,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
         const long long cap = static_cast<long long>(n_sm) * 8;   // 8 resident CTAs of 256 threads per SM
         const unsigned grid = static_cast<unsigned>(n_items < cap ? n_items : cap);
+        ScopedTimer timer(0, c.stream);
         switch (d->dtype) {
         case MCSD_DTYPE_F32: argmax_kernel<MCSD_DTYPE_F32><<<grid, kThreads, 0, c.stream>>>(p); break;
         case MCSD_DTYPE_BF16: argmax_kernel<MCSD_DTYPE_BF16><<<grid, kThreads, 0, c.stream>>>(p); break;
@@ -468,6 +507,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     lc.attrs = attr;
     lc.numAttrs = 1;
     if (n_clusters > 0) {
+        ScopedTimer timer(0, c.stream);
         if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
             cudaGetLastError();
             return MCSD_ERR_CUDA;
@@ -492,6 +532,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         long long ctas = (warps + 3) / 4;
         if (ctas > static_cast<long long>(n_sm) * 64) ctas = static_cast<long long>(n_sm) * 64;
         const unsigned grid = static_cast<unsigned>(ctas);
+        ScopedTimer timer(1, c.stream);
         switch (d->dtype * 100 + cfg.ept) {
         case MCSD_DTYPE_F32 * 100 + 16: stream_stats_kernel<MCSD_DTYPE_F32, 16><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
         case MCSD_DTYPE_F32 * 100 + 32: stream_stats_kernel<MCSD_DTYPE_F32, 32><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
@@ -539,6 +580,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         sa[0].val.programmaticStreamSerializationAllowed = 1;
         sc.attrs = sa;
         sc.numAttrs = sp.pdl ? 1 : 0;
+        ScopedTimer timer(2, c.stream);
         if (cudaLaunchKernelEx(&sc, sk, sp) != cudaSuccess) {
             cudaGetLastError();
             return MCSD_ERR_CUDA;
@@ -658,6 +700,7 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = attr;
         lc.numAttrs = p.pdl ? 1 : 0;
+        ScopedTimer timer(3, c.stream);
         if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
             cudaGetLastError();
             return MCSD_ERR_CUDA;
@@ -726,6 +769,24 @@ long long mcsd_debug_bounds_hits(int reset)
     (void)reset;
     return -1;
 #endif
+}
+
+int mcsd_last_kernel_times(float *ms, int32_t n)
+{
+    if (!ms || n < 0) return MCSD_ERR_NULL;
+    int filled = 0;
+    for (int s = 0; s < kTimeSlots && s < n; ++s) {
+        ms[s] = -1.f;
+        if (g_timers.created && g_timers.used[s]) {
+            if (cudaEventSynchronize(g_timers.ev[s][1]) != cudaSuccess ||
+                cudaEventElapsedTime(&ms[s], g_timers.ev[s][0], g_timers.ev[s][1]) != cudaSuccess) {
+                cudaGetLastError();
+                return MCSD_ERR_CUDA;
+            }
+            ++filled;
+        }
+    }
+    return filled;
 }
 
 int mcsd_set_option(int option, int value)

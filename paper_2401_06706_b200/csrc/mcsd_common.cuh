@@ -422,9 +422,10 @@ __device__ __forceinline__ int warp_multi_sum(const float (&v)[N], int lane, flo
 // The vocabulary is cut into contiguous runs, one per warp; a run into S steps of 32
 // groups (one group of 4 or 8 consecutive elements per lane).  Every lane keeps the float
 // sums g[S] of its own groups.  The search goes run -> step -> lane -> element; everything
-// above the lane level (run totals, their prefix sums, the position of the quantile inside
-// the run, the step totals' prefix sums) is carried in double, so that the only float
-// roundings left are inside one step (1/512 of the vocabulary or less).
+// that combines runs or steps (the prefix sums of the run totals, the position of the quantile
+// inside the run, the prefix sums of the step totals) is carried in double, so that no rounding
+// of the size of the whole distribution's ulp enters: the float roundings left are those of one
+// run total (a sixteenth of the vocabulary or less) and of the sums inside one step.
 
 // Total of every step of this warp's run: lane st * (32 / S) holds the total of step st.
 template <int S>
@@ -433,13 +434,13 @@ __device__ __forceinline__ float step_totals(const float (&g)[S], int lane) {
     warp_multi_sum<S>(g, lane, tj);
     return tj;
 }
-// Total of the run: the step totals added in ascending order, in double (all lanes).
+// Total of the run (all lanes): the lanes' own sums over their groups, added across the warp.
 template <int S>
-__device__ __forceinline__ double run_total(float tj) {
-    double r = 0.0;
+__device__ __forceinline__ double run_total(const float (&g)[S]) {
+    float t = 0.f;
 #pragma unroll
-    for (int st = 0; st < S; ++st) r += static_cast<double>(__shfl_sync(0xffffffffu, tj, st * (32 / S)));
-    return r;
+    for (int st = 0; st < S; ++st) t += g[st];
+    return static_cast<double>(warp_sum(t));
 }
 // The run that holds the quantile u of the whole distribution.  m: total of run `lane`
 // (0 for lanes beyond the runs).  Every warp that calls this with the same totals finds the

@@ -93,8 +93,7 @@ naive_kernel(const __grid_constant__ NaiveParams P)
                 for (int e = 0; e < GV; ++e) g[st] += w[e];
             }
         }
-        const float tj = step_totals<kMaxSteps>(g, lane);
-        const double mass = run_total<kMaxSteps>(tj);
+        const double mass = run_total<kMaxSteps>(g);
         if (lane == 0) s_wtot[warp] = mass;
         if (tid == 0) s_pick = -1;
         __syncthreads();
@@ -112,6 +111,7 @@ naive_kernel(const __grid_constant__ NaiveParams P)
         if (pick >= 0 && warp == pick) {
             int ps, l;
             float rem;
+            const float tj = step_totals<kMaxSteps>(g, lane);
             if (search_run<kMaxSteps>(g, tj, tgt, lane, ps, l, rem) && lane == l) {
                 const int x0 = x_lo + ps * kStep + lane * GV;
                 float w[GV];

@@ -50,7 +50,8 @@ sample_kernel(const __grid_constant__ SampleParams P)
     __shared__ float s_red[32];
     __shared__ int s_redi[32];
     __shared__ int32_t s_rem_tok[MCSD_MAX_CHILDREN];
-    __shared__ int s_pick;
+    __shared__ int s_pick, s_run;
+    __shared__ double s_tgt;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / P.n_range, n = P.node_begin + (blockIdx.x - b * P.n_range);
     const int k = P.child_count[n], first = P.child_first[n];
@@ -255,22 +256,27 @@ sample_kernel(const __grid_constant__ SampleParams P)
         for (int e = 0; e < GV; ++e) w[e] = ex2f(fmaf(v[e], P.scale, -r0)) * f;
     };
     {
-        const double run_mass = run_total<kMaxSteps>(step_totals<kMaxSteps>(g, lane));
+        const double run_mass = run_total<kMaxSteps>(g);
         if (lane == 0) s_wtot[warp] = run_mass;
     }
     __syncthreads();
 
     int n_rem = 0;  // tokens taken out so far (Eq. 1); the same in every thread
     for (int i = 0; i < k; ++i) {
-        const float u = P.unif_draw[static_cast<long long>(b) * P.n_nodes + first + i];
-        // the run that holds the quantile (every warp finds the same one)
-        double tgt = 0.0;
-        const int pick = pick_run(lane < kW ? s_wtot[lane] : 0.0, u, lane, tgt);
-        int found = -1;
-        double new_mass = -1.0;   // (Eq. 1) what is left of this warp's run after the draw
+        // warp 0 finds the run that holds the quantile ...
+        if (warp == 0) {
+            const float u = P.unif_draw[static_cast<long long>(b) * P.n_nodes + first + i];
+            double t = 0.0;
+            const int r = pick_run(lane < kW ? s_wtot[lane] : 0.0, u, lane, t);
+            if (lane == 0) { s_run = r; s_tgt = t; }
+        }
+        __syncthreads();
+        const int pick = s_run;
+        // ... and the warp that owns that run finds the step, the lane and the element
         if (pick >= 0 && warp == pick) {
+            const double tgt = s_tgt;
             const float tj = step_totals<kMaxSteps>(g, lane);
-            int ps, l;
+            int ps, l, found = -1;
             float rem;
             if (search_run<kMaxSteps>(g, tj, tgt, lane, ps, l, rem)) {
                 int pe = -1;
@@ -298,23 +304,27 @@ sample_kernel(const __grid_constant__ SampleParams P)
                     }
                 }
                 found = __shfl_sync(0xffffffffu, pe < 0 ? -1 : x_lo + ps * kStep + lane * GV + pe, l);
-                // ... and the run's total, from the lanes' current group sums
-                if (P.mode == 1 && found >= 0) new_mass = run_total<kMaxSteps>(step_totals<kMaxSteps>(g, lane));
+                // ... and the run's total, from the lanes' current group sums (only warp 0 reads the
+                // totals, and not before the barrier below)
+                if (P.mode == 1 && found >= 0) {
+                    const double left = run_total<kMaxSteps>(g);
+                    if (lane == 0) s_wtot[warp] = left;
+                }
             }
-            if (lane == 0) s_pick = found;
+            if (lane == 0) {
+                s_pick = found;
+                out[i] = found;
+                if (found < 0 && P.status) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
+                if (P.mode == 1) s_rem_tok[n_rem] = found;
+            }
+        } else if (pick < 0 && tid == 0) {
+            s_pick = -1;
+            out[i] = -1;
+            if (P.status) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
+            if (P.mode == 1) s_rem_tok[n_rem] = -1;
         }
-        if (pick < 0) { if (tid == 0) s_pick = -1; }
         __syncthreads();
-        found = s_pick;
-        // (written only now: until the barrier above other warps may still have been reading the totals)
-        if (new_mass >= 0.0 && lane == 0) s_wtot[warp] = new_mass;
-        if (tid == 0) {
-            out[i] = found;
-            if (found < 0 && P.status) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
-            if (P.mode == 1) s_rem_tok[n_rem] = found;
-        }
-        if (P.mode == 1 && found >= 0) ++n_rem;
-        __syncthreads();
+        if (P.mode == 1 && s_pick >= 0) ++n_rem;
     }
 }
 

@@ -374,7 +374,7 @@ shard_endpoint_kernel(const __grid_constant__ ShardParams P)
                 }
             }
         }
-        const double mass = run_total<S>(step_totals<S>(g, lane));
+        const double mass = run_total<S>(g);
         if (lane == 0) P.tot_out[static_cast<long long>(b) * P.eps_max + e] = mass;
     }
 }

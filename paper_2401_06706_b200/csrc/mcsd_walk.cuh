@@ -182,7 +182,6 @@ walk_kernel(const __grid_constant__ WalkParams P)
     float kappa = fminf(c * dq, 3.0e38f);
     int extra_bits = 0;
     float g[kMaxSteps];
-    float tj = 0.f;
     double tgt = 0.0;
     int pick = -1;
     // weights of the GV elements starting at x0 (0 past the end of the vocabulary), times Z_t
@@ -232,8 +231,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
                 }
             }
         }
-        tj = step_totals<kMaxSteps>(g, lane);
-        const double mass = run_total<kMaxSteps>(tj);
+        const double mass = run_total<kMaxSteps>(g);
         __syncthreads();   // (second attempt: everybody has read the totals of the first)
         if (lane == 0) s_wtot[warp] = mass;
         __syncthreads();
@@ -280,6 +278,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
     // lane's group (its weights are formed once more)
     int ps, l, found = -1;
     float rem;
+    const float tj = step_totals<kMaxSteps>(g, lane);
     if (search_run<kMaxSteps>(g, tj, tgt, lane, ps, l, rem)) {
         int pe = -1;
         if (lane == l) {
