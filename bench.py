@@ -482,6 +482,7 @@ def run_cuda(args):
                 "us_per_call": ms_per_step * 1e3,
                 "rows_per_sec": world * w.batch * (st["n_nodes"] + (st["n_internal"] if w.temperature > 0 else 0)) / (ms_per_step * 1e-3),
                 "accept_len_mean": accept_len_mean,
+                "alpha_hat": parity.get("alpha_hat") if isinstance(parity, dict) else None,
                 "device_status_bits": status_bits, "parity_on_oracle_sample": parity}
         print(json.dumps(line), flush=True)
     if dist:

@@ -64,8 +64,6 @@ walk_kernel(const __grid_constant__ WalkParams P)
     __shared__ double s_wtot[32];
     __shared__ float s_leaf[2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // the node stage's results must be complete and visible before anything of them is read
-    if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
     int b, n;
     if (P.all_nodes) {
         b = blockIdx.x / P.n_nodes;
@@ -80,13 +78,16 @@ walk_kernel(const __grid_constant__ WalkParams P)
     if (!P.all_nodes) {
         // the tree's decisions and tokens come into shared memory with one parallel load, so
         // that the walk itself is not a chain of dependent global loads
+        // (the caller's inputs first: they do not depend on the node stage, whose results must be
+        // complete and visible before anything of them is read)
+        for (int i = tid; i < P.n_nodes; i += NT) {
+            s_tok[i] = P.cand[nb + i];
+            if (P.scale != 0.f) s_uend[i] = P.unif[2 * (nb + i) + 1];
+        }
+        if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int i = tid; i < P.n_nodes; i += NT) {
             s_acc[i] = P.node_accept[nb + i];
-            s_tok[i] = P.cand[nb + i];
-            if (P.scale != 0.f) {
-                s_uend[i] = P.unif[2 * (nb + i) + 1];
-                if (i < P.n_internal) s_stats[i] = P.stats[nb + i];
-            }
+            if (P.scale != 0.f && i < P.n_internal) s_stats[i] = P.stats[nb + i];
         }
         __syncthreads();
         if (tid == 0) {
@@ -113,9 +114,12 @@ walk_kernel(const __grid_constant__ WalkParams P)
         __syncthreads();
         n = s_term;
         len = s_len;
-    } else if (P.node_accept[nb + n] >= 0) {
-        if (tid == 0) P.node_bonus[nb + n] = -1;  // a walk never stops here
-        return;
+    } else {
+        if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (P.node_accept[nb + n] >= 0) {
+            if (tid == 0) P.node_bonus[nb + n] = -1;  // a walk never stops here
+            return;
+        }
     }
     float *out = P.all_nodes ? (P.node_residual ? P.node_residual + (nb + n) * P.V : nullptr)
                              : (P.out_residual ? P.out_residual + static_cast<long long>(b) * P.V : nullptr);
