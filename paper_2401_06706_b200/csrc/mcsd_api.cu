@@ -466,11 +466,12 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         else stream_nodes[n_stream++] = static_cast<uint16_t>(n);
         n_single += k == 1;
     }
-    // (measured: with 2-byte logits the split pays from about ten items per resident cluster on, with
-    // 4-byte logits, where the cluster kernel is close to the memory bandwidth anyway, only on launches
-    // that run for hundreds of microseconds)
+    // (measured: a tree without such nodes, a chain, always gains; otherwise the split pays with 2-byte
+    // logits from about fourteen items per resident cluster on, and with 4-byte logits, where the cluster
+    // kernel is close to the memory bandwidth anyway, only on launches that run for hundreds of
+    // microseconds back to back)
     const int split_opt = g_opt.v[MCSD_OPT_SPLIT];
-    const long long split_from = (d->dtype == MCSD_DTYPE_F32 ? 96LL : 8LL) * resident;
+    const long long split_from = n_keep == 0 ? 0 : (d->dtype == MCSD_DTYPE_F32 ? 96LL : 14LL) * resident;
     const bool split = !path && n_stream > 0 && split_opt != 1 && (split_opt == 2 || n_items >= split_from);
     const int n_list = split ? n_keep : d->n_nodes;
     const long long n_cluster_items = path ? n_items : static_cast<long long>(d->batch) * n_list;
