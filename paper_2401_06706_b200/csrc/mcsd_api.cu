@@ -113,9 +113,14 @@ struct KernelTimers {
     cudaEvent_t ev[kTimeSlots][2] = {};
     bool used[kTimeSlots] = {};
     bool created = false;
+    int device = -1;   // the device the events belong to
 };
 thread_local KernelTimers g_timers;
 
+inline void reset_timers_used()
+{
+    for (bool &u : g_timers.used) u = false;
+}
 struct ScopedTimer {
     int slot;
     cudaStream_t stream;
@@ -123,10 +128,19 @@ struct ScopedTimer {
     ScopedTimer(int s, cudaStream_t st) : slot(s), stream(st), on(g_opt.v[MCSD_OPT_TIME_KERNELS] != 0)
     {
         if (!on) return;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (g_timers.created && g_timers.device != dev) {   // the thread moved to another device
+            for (auto &pair : g_timers.ev)
+                for (auto &e : pair) cudaEventDestroy(e);
+            g_timers.created = false;
+            reset_timers_used();
+        }
         if (!g_timers.created) {
             for (auto &pair : g_timers.ev)
                 for (auto &e : pair) cudaEventCreate(&e);
             g_timers.created = true;
+            g_timers.device = dev;
         }
         cudaEventRecord(g_timers.ev[slot][0], stream);
     }
@@ -137,10 +151,7 @@ struct ScopedTimer {
         g_timers.used[slot] = true;
     }
 };
-void reset_timers()
-{
-    for (bool &u : g_timers.used) u = false;
-}
+void reset_timers() { reset_timers_used(); }
 
 // Checked build: the address ranges the kernels of the next launches on `stream` may read.  An
 // empty list switches the checks off (kernels whose inputs are not registered).
