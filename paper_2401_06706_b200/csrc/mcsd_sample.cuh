@@ -52,6 +52,8 @@ sample_kernel(const __grid_constant__ SampleParams P)
     __shared__ int32_t s_rem_tok[MCSD_MAX_CHILDREN];
     __shared__ int s_pick, s_run;
     __shared__ double s_tgt;
+    __shared__ int s_runs[MCSD_MAX_CHILDREN];
+    __shared__ double s_tgts[MCSD_MAX_CHILDREN];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / P.n_range, n = P.node_begin + (blockIdx.x - b * P.n_range);
     const int k = P.child_count[n], first = P.child_first[n];
@@ -261,6 +263,52 @@ sample_kernel(const __grid_constant__ SampleParams P)
     }
     __syncthreads();
 
+    if (P.mode != 1) {
+        // Independent draws (the candidates of Algorithm 1): warp 0 finds the run of every draw, the CTA
+        // meets once, and every warp serves the draws that fell into its run.
+        if (warp == 0) {
+            const double m = lane < kW ? s_wtot[lane] : 0.0;
+            for (int i = 0; i < k; ++i) {
+                const float u = P.unif_draw[static_cast<long long>(b) * P.n_nodes + first + i];
+                double t = 0.0;
+                const int r = pick_run(m, u, lane, t);
+                if (lane == 0) { s_runs[i] = r; s_tgts[i] = t; }
+            }
+        }
+        __syncthreads();
+        float tj = 0.f;
+        bool have_tj = false;
+        for (int i = 0; i < k; ++i) {
+            const int pick = s_runs[i];
+            if (pick < 0) {
+                if (tid == 0) {
+                    out[i] = -1;
+                    if (P.status) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
+                }
+                continue;
+            }
+            if (pick != warp) continue;
+            if (!have_tj) { tj = step_totals<kMaxSteps>(g, lane); have_tj = true; }
+            int ps, l, found = -1;
+            float rem;
+            if (search_run<kMaxSteps>(g, tj, s_tgts[i], lane, ps, l, rem)) {
+                int pe = -1;
+                if (lane == l) {
+                    float w[GV];
+                    weights(x_lo + ps * kStep + lane * GV, ps, w);
+                    pe = pick_element<GV>(w, rem);
+                }
+                found = __shfl_sync(0xffffffffu, pe < 0 ? -1 : x_lo + ps * kStep + lane * GV + pe, l);
+            }
+            if (lane == 0) {
+                out[i] = found;
+                if (found < 0 && P.status) atomicOr(P.status + b, MCSD_STATUS_NO_MASS);
+            }
+        }
+        return;
+    }
+
+    // Without replacement (Eq. 1) every draw changes the distribution of the next: one draw at a time.
     int n_rem = 0;  // tokens taken out so far (Eq. 1); the same in every thread
     for (int i = 0; i < k; ++i) {
         // warp 0 finds the run that holds the quantile ...
