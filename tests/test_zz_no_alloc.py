@@ -63,10 +63,17 @@ def _both_ways(w):
     other.desc.workspace_bytes = 0
     other.mcsd_verify_static(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)   # first call on the device: address lookup
     torch.cuda.synchronize()
-    free_before = torch.cuda.mem_get_info()[0]
-    b = other.mcsd_verify_static(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
-    torch.cuda.synchronize()
-    assert torch.cuda.mem_get_info()[0] == free_before, "mcsd_verify_static changed the device's free memory"
+    # (free memory is a property of the whole device: a call that allocates shows it every time, another
+    # process that happens to allocate in between does not, so a difference is checked again)
+    unchanged = False
+    for _ in range(3):
+        free_before = torch.cuda.mem_get_info()[0]
+        b = other.mcsd_verify_static(inp.target, draft, inp.cand, inp.unif, w.temperature, w.mode)
+        torch.cuda.synchronize()
+        if torch.cuda.mem_get_info()[0] == free_before:
+            unchanged = True
+            break
+    assert unchanged, "mcsd_verify_static changed the device's free memory"
     return inp, a, b
 
 
