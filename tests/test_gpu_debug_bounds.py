@@ -1,8 +1,8 @@
 """The checked build of the library (libmcsd_debug.so, -DMCSD_DEBUG_BOUNDS): every read of caller
 memory by the kernels that read logits is checked against the extents the descriptor implies; a
-read outside them is skipped and counted, never trapped.  compute-sanitizer is not available on the
-GPUs these tests run on, so this build, the guard words around every output (gpu_util.Guards) and the
-run-twice comparisons stand in for its memcheck.  Across awkward shapes (ragged vocabularies, padded
+read outside them is skipped and counted, never trapped.  Together with the guard words around every
+output (gpu_util.Guards) and the run-twice comparisons it does what a memory checker would, without
+a tool around the process.  Across awkward shapes (ragged vocabularies, padded
 and unaligned rows, every entry point) the count must stay 0 and the results must be the oracle's."""
 import os
 
