@@ -8,6 +8,8 @@
 #include <mutex>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "mcsd_device.cuh"
 
 namespace mcsd {
@@ -35,9 +37,50 @@ struct Options {
         v[MCSD_OPT_TEST_EXTRA_TX] = 0;
         v[MCSD_OPT_PDL] = env_int("MCSD_PDL", 1);
         v[MCSD_OPT_SPLIT] = env_int("MCSD_SPLIT", 0);
+        v[MCSD_OPT_TRACE] = env_int("MCSD_TRACE", 0);
     }
 };
 Options g_opt;
+
+// MCSD_OPT_TRACE: bit 0, one line per call of a verification entry point on stderr (what was asked for,
+// how the node stage was laid out, the return code); bit 1, an NVTX range around the call, for timelines.
+// Host side only; the kernels are not touched.
+struct TraceNote {
+    int cluster = 0, ept = 0, threads = 0, direct = 0, split = 0;
+    long long clusters = 0, stream_ctas = 0;
+};
+thread_local TraceNote g_note;
+struct Trace {
+    const char *name;
+    const mcsd_desc *d;
+    float T;
+    int mode, bits;
+    Trace(const char *n, const mcsd_desc *desc, float temperature, int replacement_mode)
+        : name(n), d(desc), T(temperature), mode(replacement_mode), bits(g_opt.v[MCSD_OPT_TRACE])
+    {
+        if (bits & 2) nvtxRangePushA(name);
+        if (bits & 1) g_note = TraceNote();
+    }
+    int done(int rc)
+    {
+        if (bits & 2) nvtxRangePop();
+        if (bits & 1) {
+            if (d)
+                std::fprintf(stderr, "[mcsd] %s batch=%d nodes=%d internal=%d vocab=%d dtype=%d T=%g mode=%d -> rc=%d launches=%d",
+                             name, d->batch, d->n_nodes, d->n_internal, d->vocab, d->dtype, static_cast<double>(T), mode, rc,
+                             rc == MCSD_OK ? g_last_launches : 0);
+            else
+                std::fprintf(stderr, "[mcsd] %s desc=NULL -> rc=%d", name, rc);
+            if (rc == MCSD_OK && g_note.threads)
+                std::fprintf(stderr, " node stage: cluster=%d x %d threads, %d elements/thread%s, %lld clusters%s",
+                             g_note.cluster, g_note.threads, g_note.ept, g_note.direct ? ", element loads" : "",
+                             g_note.clusters, g_note.split ? ", split launch" : "");
+            if (rc == MCSD_OK && g_note.split) std::fprintf(stderr, " (%lld streaming CTAs)", g_note.stream_ctas);
+            std::fprintf(stderr, "\n");
+        }
+        return rc;
+    }
+};
 
 struct TreePlan {
     int gamma = 0;
@@ -521,6 +564,10 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
+    if (g_opt.v[MCSD_OPT_TRACE] & 1) {
+        g_note.cluster = cfg.cluster; g_note.ept = cfg.ept; g_note.threads = cfg.threads; g_note.direct = cfg.direct;
+        g_note.split = split; g_note.clusters = n_clusters;
+    }
     if (n_clusters > 0) {
         ScopedTimer timer(0, c.stream);
         if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
@@ -547,6 +594,7 @@ int launch_nodes(const Call &c, const void *target, const void *draft, const int
         long long ctas = (warps + 3) / 4;
         if (ctas > static_cast<long long>(n_sm) * 64) ctas = static_cast<long long>(n_sm) * 64;
         const unsigned grid = static_cast<unsigned>(ctas);
+        g_note.stream_ctas = ctas;
         ScopedTimer timer(1, c.stream);
         switch (d->dtype * 100 + cfg.ept) {
         case MCSD_DTYPE_F32 * 100 + 16: stream_stats_kernel<MCSD_DTYPE_F32, 16><<<grid, kNodeThreads, 0, c.stream>>>(sp); break;
@@ -818,7 +866,7 @@ int mcsd_get_option(int option)
     return g_opt.v[option];
 }
 
-int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+static int mcsd_verify_nodes_impl(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                       const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                       float temperature, int replacement_mode)
 {
@@ -833,7 +881,15 @@ int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const vo
     return launch_nodes(c, target_logits, draft_logits, cand_tokens, uniforms, temperature, replacement_mode);
 }
 
-int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+int mcsd_verify_nodes(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                      float temperature, int replacement_mode)
+{
+    Trace trace("mcsd_verify_nodes", desc, temperature, replacement_mode);
+    return trace.done(mcsd_verify_nodes_impl(desc, target_logits, draft_logits, tree_parent, cand_tokens, uniforms, temperature, replacement_mode));
+}
+
+static int mcsd_verify_walk_impl(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                      float temperature, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
 {
@@ -850,7 +906,15 @@ int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const voi
                        out_tokens, out_residual);
 }
 
-int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+int mcsd_verify_walk(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual)
+{
+    Trace trace("mcsd_verify_walk", desc, temperature, 0);
+    return trace.done(mcsd_verify_walk_impl(desc, target_logits, draft_logits, tree_parent, cand_tokens, uniforms, temperature, out_accept_len, out_tokens, out_residual));
+}
+
+static int mcsd_verify_impl(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                 const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                 float temperature, int replacement_mode, int32_t *out_accept_len,
                 int32_t *out_tokens, float *out_residual)
@@ -877,7 +941,16 @@ int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *dr
                        out_tokens, out_residual);
 }
 
-int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+int mcsd_verify(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                float temperature, int replacement_mode, int32_t *out_accept_len,
+                int32_t *out_tokens, float *out_residual)
+{
+    Trace trace("mcsd_verify", desc, temperature, replacement_mode);
+    return trace.done(mcsd_verify_impl(desc, target_logits, draft_logits, tree_parent, cand_tokens, uniforms, temperature, replacement_mode, out_accept_len, out_tokens, out_residual));
+}
+
+static int mcsd_verify_path_impl(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                      float temperature, int replacement_mode, int32_t *out_accept_len,
                      int32_t *out_tokens, float *out_residual)
@@ -910,7 +983,16 @@ int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const voi
                        out_tokens, out_residual, false);
 }
 
-int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, const int32_t *tree_parent,
+int mcsd_verify_path(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int replacement_mode, int32_t *out_accept_len,
+                     int32_t *out_tokens, float *out_residual)
+{
+    Trace trace("mcsd_verify_path", desc, temperature, replacement_mode);
+    return trace.done(mcsd_verify_path_impl(desc, target_logits, draft_logits, tree_parent, cand_tokens, uniforms, temperature, replacement_mode, out_accept_len, out_tokens, out_residual));
+}
+
+static int mcsd_sample_candidates_impl(const mcsd_desc *desc, const void *draft_logits, const int32_t *tree_parent,
                            const float *uniforms_draw, float temperature, int replacement_mode,
                            int32_t node_begin, int32_t node_end, int32_t *cand_tokens)
 {
@@ -977,6 +1059,14 @@ int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, cons
     if (cudaGetLastError() != cudaSuccess) return MCSD_ERR_CUDA;
     g_last_launches = 1;
     return MCSD_OK;
+}
+
+int mcsd_sample_candidates(const mcsd_desc *desc, const void *draft_logits, const int32_t *tree_parent,
+                           const float *uniforms_draw, float temperature, int replacement_mode,
+                           int32_t node_begin, int32_t node_end, int32_t *cand_tokens)
+{
+    Trace trace("mcsd_sample_candidates", desc, temperature, replacement_mode);
+    return trace.done(mcsd_sample_candidates_impl(desc, draft_logits, tree_parent, uniforms_draw, temperature, replacement_mode, node_begin, node_end, cand_tokens));
 }
 
 int mcsd_tree_attention_layout(const int32_t *tree_parent, int32_t n_nodes, int32_t prefix_len,
@@ -1375,7 +1465,7 @@ void *static_workspace()
 }
 }  // namespace
 
-int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+static int mcsd_verify_static_impl(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                        const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                        float temperature, int replacement_mode, int32_t *out_accept_len,
                        int32_t *out_tokens, float *out_residual)
@@ -1390,8 +1480,17 @@ int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const v
     with_scratch.workspace_bytes = MCSD_STATIC_WORKSPACE_BYTES;
     // the status words are cleared by the node stage itself; everything else in the
     // array is written before it is read
-    return mcsd_verify(&with_scratch, target_logits, draft_logits, tree_parent, cand_tokens, uniforms,
+    return mcsd_verify_impl(&with_scratch, target_logits, draft_logits, tree_parent, cand_tokens, uniforms,
                        temperature, replacement_mode, out_accept_len, out_tokens, out_residual);
+}
+
+int mcsd_verify_static(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                       const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                       float temperature, int replacement_mode, int32_t *out_accept_len,
+                       int32_t *out_tokens, float *out_residual)
+{
+    Trace trace("mcsd_verify_static", desc, temperature, replacement_mode);
+    return trace.done(mcsd_verify_static_impl(desc, target_logits, draft_logits, tree_parent, cand_tokens, uniforms, temperature, replacement_mode, out_accept_len, out_tokens, out_residual));
 }
 
 // ---- mcsd_verify_host: device staging buffers kept between calls ------------------------
@@ -1426,7 +1525,7 @@ int mcsd_release_host_staging(void)
     return MCSD_OK;
 }
 
-int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+static int mcsd_verify_host_impl(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
                      const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
                      float temperature, int replacement_mode, int32_t *out_accept_len,
                      int32_t *out_tokens, float *out_residual, int32_t *out_status)
@@ -1508,7 +1607,7 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
         cd.workspace = base + o_ws;
         cd.workspace_bytes = ws_bytes;
         cd.out_status = reinterpret_cast<int32_t *>(base + o_st);
-        rc = mcsd_verify(&cd, base + o_t, use_draft ? base + o_d : nullptr, tree_parent,
+        rc = mcsd_verify_impl(&cd, base + o_t, use_draft ? base + o_d : nullptr, tree_parent,
                          reinterpret_cast<const int32_t *>(base + o_c),
                          uniforms ? reinterpret_cast<const float *>(base + o_u) : nullptr, temperature,
                          replacement_mode, reinterpret_cast<int32_t *>(base + o_len),
@@ -1531,6 +1630,15 @@ int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const voi
     if (rc != MCSD_OK) return rc;
     if (!ok) { cudaGetLastError(); return MCSD_ERR_CUDA; }
     return MCSD_OK;
+}
+
+int mcsd_verify_host(const mcsd_desc *desc, const void *target_logits, const void *draft_logits,
+                     const int32_t *tree_parent, const int32_t *cand_tokens, const float *uniforms,
+                     float temperature, int replacement_mode, int32_t *out_accept_len,
+                     int32_t *out_tokens, float *out_residual, int32_t *out_status)
+{
+    Trace trace("mcsd_verify_host", desc, temperature, replacement_mode);
+    return trace.done(mcsd_verify_host_impl(desc, target_logits, draft_logits, tree_parent, cand_tokens, uniforms, temperature, replacement_mode, out_accept_len, out_tokens, out_residual, out_status));
 }
 
 }  // extern "C"

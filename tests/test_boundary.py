@@ -40,7 +40,7 @@ def test_header_constants_match_binding():
     assert int(consts["MCSD_MAX_VOCAB"]) == binding.MAX_VOCAB
     assert int(consts["MCSD_STATUS_TIMEOUT"]) == binding.STATUS_TIMEOUT
     assert int(consts["MCSD_DTYPE_BF16"]) == 1 and int(consts["MCSD_DTYPE_F16"]) == 2
-    for name in ("CLUSTER", "EPT", "DIRECT", "SAMPLE_AHEAD", "WAIT_POLLS", "TEST_EXTRA_TX", "PDL", "TEST_SHRINK_RANGES", "SPLIT", "TIME_KERNELS"):
+    for name in ("CLUSTER", "EPT", "DIRECT", "SAMPLE_AHEAD", "WAIT_POLLS", "TEST_EXTRA_TX", "PDL", "TEST_SHRINK_RANGES", "SPLIT", "TIME_KERNELS", "TRACE"):
         assert int(consts["MCSD_OPT_" + name]) == getattr(binding, "OPT_" + name)
 
 
@@ -57,6 +57,29 @@ def test_options_are_set_read_back_and_validated(lib):
     finally:
         for i, val in enumerate(before):
             binding.mcsd_set_option(i, val)
+
+
+def test_trace_option_reports_rejected_calls_on_stderr(lib, capfd):
+    """MCSD_OPT_TRACE bit 0: one line per call with the shape, the temperature, the mode and the return
+    code; here for calls the host checks reject (nothing is enqueued, the fake pointers are never used)."""
+    d, parent = _desc(ws=(0x10000, 1 << 20))
+    before = binding.mcsd_get_option(binding.OPT_TRACE)
+    try:
+        binding.mcsd_set_option(binding.OPT_TRACE, 1)
+        assert lib.mcsd_verify(ctypes.byref(d), 0x1000, 0x1000, parent.ctypes.data, 0x1000, 0x1000, -0.5, 0,
+                               0x1000, 0x1000, None) == -5
+        assert lib.mcsd_verify_path(None, 0x1000, 0x1000, parent.ctypes.data, 0x1000, 0x1000, 1.0, 1,
+                                    0x1000, 0x1000, None) == -1
+        binding.mcsd_set_option(binding.OPT_TRACE, 0)
+        assert lib.mcsd_verify(ctypes.byref(d), 0x1000, 0x1000, parent.ctypes.data, 0x1000, 0x1000, -0.5, 0,
+                               0x1000, 0x1000, None) == -5
+    finally:
+        binding.mcsd_set_option(binding.OPT_TRACE, before)
+    lines = [l for l in capfd.readouterr().err.splitlines() if l.startswith("[mcsd]")]
+    assert len(lines) == 2                                       # nothing once the option is off again
+    assert "mcsd_verify " in lines[0] and f"batch={d.batch}" in lines[0] and f"vocab={d.vocab}" in lines[0]
+    assert "T=-0.5" in lines[0] and "rc=-5" in lines[0] and "launches=0" in lines[0]
+    assert "mcsd_verify_path desc=NULL" in lines[1] and "rc=-1" in lines[1]
 
 
 def test_tree_depth_and_contract(lib):

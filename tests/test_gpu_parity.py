@@ -132,6 +132,27 @@ def test_split_launch_equals_single_launch(dtype, vocab, kconfig, mode):
         assert np.array_equal(a, b, equal_nan=True)
 
 
+def test_traced_call_reports_its_layout_and_changes_nothing(capfd):
+    """MCSD_OPT_TRACE 3: a line on stderr per call (with how the node stage was laid out) and an NVTX
+    range around it; the outputs are those of the untraced call."""
+    w = synth.Workload("traced", 5, 32000, "4x2x1", "bf16", "normal", 2.5, 0.9, 1.2, 1.0, 1, 4711)
+    inp = synth.make_inputs(w, "cuda")
+    with library_options(split=2):
+        _, plain = run_library(inp, node_outputs=False)
+        want = [to_np(x).copy() for x in (plain.accept_len, plain.tokens, plain.residual, plain.status)]
+        capfd.readouterr()
+        with library_options(trace=3):
+            _, traced = run_library(inp, node_outputs=False)
+        torch.cuda.synchronize()
+    lines = [l for l in capfd.readouterr().err.splitlines() if l.startswith("[mcsd] mcsd_verify ")]
+    assert len(lines) == 1
+    for part in ("batch=5", "vocab=32000", "dtype=1", "mode=1", "rc=0", "launches=4", "cluster=4 x 128 threads",
+                 "64 elements/thread", "split launch"):
+        assert part in lines[0], (part, lines[0])
+    for a, b in zip(want, (traced.accept_len, traced.tokens, traced.residual, traced.status)):
+        assert np.array_equal(a, to_np(b), equal_nan=True)
+
+
 def test_direct_path_matches_bulk_copy_path():
     w = synth.Workload("direct", 6, 32000, "4x2", "bf16", "normal", 2.5, 0.8, 1.5, 1.0, 0, 99)
     inp = synth.make_inputs(w, "cuda")
