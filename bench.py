@@ -604,6 +604,19 @@ def run_e2e(args, w, inp, dist, world, dev):
 
 
 # ----------------------------------------------------------------------------- sweep
+def sweep_points_done(path: str):
+    """Names of the sweep points a (possibly cut-off) output file already holds; a last line that is
+    not whole JSON is ignored."""
+    names = set()
+    with open(path) as f:
+        for line in f:
+            try:
+                names.add(json.loads(line)["workload"])
+            except (ValueError, KeyError):
+                pass
+    return names
+
+
 def run_sweep(args):
     """The 300-point throughput sweep (dtype x batch x k-config x sigma x mode at vocabulary
     32000, temperature 1).  Every call is timed on its own between CUDA events with L2
@@ -623,7 +636,14 @@ def run_sweep(args):
         points = [w for name, w in synth.named_workloads().items() if name != "cfg5_largest" and args.sweep_filter in name]
     else:
         points = [w for w in synth.sweep_workloads() if args.sweep_filter in w.name]
-    out = open(args.sweep_out, "w") if args.sweep_out else None
+    # --sweep-resume: points already in the output file (one JSON line each, written as they finish) are
+    # skipped, so an interrupted sweep goes on where it stopped
+    done = set()
+    if args.sweep_out and args.sweep_resume and os.path.exists(args.sweep_out):
+        done = sweep_points_done(args.sweep_out)
+        points = [w for w in points if w.name not in done]
+        print(f"resuming: {len(done)} points found in {args.sweep_out}, {len(points)} left", flush=True)
+    out = open(args.sweep_out, "a" if done else "w") if args.sweep_out else None
     for w in points:
         inp = synth.make_inputs(w, dev)
         st = inp.stats
@@ -819,6 +839,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the bench line")
     ap.add_argument("--sweep-filter", default="", help="only sweep points whose name contains this text")
     ap.add_argument("--sweep-out", default="", help="file for one JSON line per sweep point")
+    ap.add_argument("--sweep-resume", action="store_true", help="skip the points --sweep-out already holds")
     ap.add_argument("--named", action="store_true",
                     help="with --sweep: the named configurations 1 to 4 instead of the sweep points, parity on every sequence")
     ap.add_argument("--sweep-calls", type=int, default=20)

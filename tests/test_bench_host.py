@@ -84,3 +84,10 @@ def test_gpus_n_without_a_launcher_starts_its_own_ranks():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     cmd = bench.spawn_command(["--gpus", "2"], 2, 29999)
     assert "torch.distributed.run" in cmd and "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd
+
+
+def test_sweep_resume_reads_the_points_a_cut_off_file_holds(tmp_path):
+    import bench
+    path = tmp_path / "sweep.jsonl"
+    path.write_text('{"workload": "a", "us_median": 1.0}\n{"workload": "b"}\n{"workload": "c", "us_med')   # cut off in the third line
+    assert bench.sweep_points_done(str(path)) == {"a", "b"}
