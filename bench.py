@@ -565,7 +565,7 @@ def run_e2e(args, w, inp, dist, world, dev):
     if args.e2e_batch > 0:
         nb, why = min(w.batch, args.e2e_batch), "--e2e-batch"
     else:
-        avail = host_mem_available()
+        avail = host_mem_available() // max(world, 1)      # the ranks of one node pin at the same time
         while nb > 1 and avail and 2 * per_seq * nb + (8 << 30) > avail:     # an unpinned copy exists while pinning
             nb //= 2
             why = f"host memory: {avail / 2**30:.0f} GiB available"
