@@ -11,8 +11,8 @@ Rules
     near-tie decision; these must stay below NEAR_TIE_SHARE of all decisions (small
     samples: at most NEAR_TIE_MIN_EVENTS events).
   * A sequence whose oracle path crosses a flipped node is excluded from the path
-    and residual comparison (and counted).  All other sequences must have the same
-    accepted length and accepted tokens.
+    and residual comparison (and counted); its outputs must still be a valid walk of the
+    tree.  All other sequences must have the same accepted length and accepted tokens.
   * Endpoint tokens are draws by inverse CDF; a different token is tolerated only
     if it has positive oracle probability and u lies within NEAR_TIE (in CDF
     units) of that token's oracle CDF interval.  Such cases are counted.
@@ -260,6 +260,25 @@ def compare(target, draft, parent, cand, unif, T: float, mode: int, dtype_name: 
                 fail(f"seq {b}: residual max abs error {err:.3e} > {tol:.1e}")
         if status is not None and int(status[b]) != int(ref_status[b]):
             fail(f"seq {b}: status {int(status[b])}, oracle (sequential form) {int(ref_status[b])}")
+    # A sequence left out above took the other branch of a near-tie: its outputs are not the oracle's,
+    # but they still have to be a walk of this tree — a length within the depth, -1 padding, and, where
+    # the nodes of the walk are reported, a chain of children from the root carrying the emitted tokens.
+    gamma_p1 = tokens.shape[1]
+    for b in rep.excluded:
+        Lg = int(accept_len[b])
+        if not 0 <= Lg < gamma_p1:
+            fail(f"seq {b} (near-tie branch): accepted length {Lg} outside [0, {gamma_p1 - 1}]")
+            continue
+        if not (tokens[b, Lg + 1:] == -1).all():
+            fail(f"seq {b} (near-tie branch): padding after the endpoint token is not -1")
+        if path_nodes is not None:
+            pg = [int(x) for x in path_nodes[b, :Lg]]
+            prev = 0
+            for i, node in enumerate(pg):
+                if not (0 < node < n_nodes) or int(parent[node]) != prev or int(tokens[b, i]) != int(cand[b, node]):
+                    fail(f"seq {b} (near-tie branch): accepted path {pg} is not a walk of the tree carrying its tokens")
+                    break
+                prev = node
     if rep.n_bonus_tolerated > boundary_draw_limit(V, max(rep.n_bonus_draws, 1)):
         fail(f"{rep.n_bonus_tolerated} of {rep.n_bonus_draws} endpoint draws differ inside the tolerance: "
              f"more than the {boundary_draw_limit(V, max(rep.n_bonus_draws, 1)):.1f} float rounding explains")
