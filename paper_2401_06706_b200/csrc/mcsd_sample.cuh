@@ -89,6 +89,29 @@ sample_kernel(const __grid_constant__ SampleParams P)
             for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
         }
     };
+    // The same, left packed (2-byte types only): 4 registers for 8 elements while the load is in flight.
+    [[maybe_unused]] auto load_raw_clamped = [&](int x0) -> uint4 {
+        uint4 r = make_uint4(0u, 0u, 0u, 0u);
+        if constexpr (E::kBytes == 2) {
+            float v[GV];
+            if (P.vector_ok) {
+                const int xc = x0 < x_last ? x0 : x_last;
+                r = ldg_v4(row + static_cast<size_t>(xc) * E::kBytes);
+                if (!(tail_mask && xc == x_last)) return r;
+                E::unpack(r, v);   // the row's last, incomplete group: its padding becomes -inf
+#pragma unroll
+                for (int e = 0; e < GV; ++e) v[e] = xc + e < P.V ? v[e] : -INFINITY;
+            } else {
+#pragma unroll
+                for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
+            }
+            r.x = E::to_bits(v[0]) | (E::to_bits(v[1]) << 16);
+            r.y = E::to_bits(v[2]) | (E::to_bits(v[3]) << 16);
+            r.z = E::to_bits(v[4]) | (E::to_bits(v[5]) << 16);
+            r.w = E::to_bits(v[6]) | (E::to_bits(v[7]) << 16);
+        }
+        return r;
+    };
     // The CTA that takes this one's place when it has finished is about `prefetch_ahead` blocks
     // further on: its row is asked into L2 now, so that HBM streams while this CTA computes and
     // that CTA's two passes both read from L2.
@@ -119,20 +142,35 @@ sample_kernel(const __grid_constant__ SampleParams P)
         float best = -INFINITY;
         int best_i = 0x7fffffff;
         {
-            constexpr int UT = 4 < kMaxSteps ? 4 : kMaxSteps;
+            // (2-byte groups stay packed until they are looked at, so eight loads in flight cost the
+            // registers of four unpacked 4-byte groups)
+            constexpr int kAhead = E::kBytes == 2 ? 8 : 4;
+            constexpr int UT = kAhead < kMaxSteps ? kAhead : kMaxSteps;
+            constexpr int VW = E::kBytes == 2 ? 1 : GV;
 #pragma unroll 1
             for (int s0 = 0; s0 < kMaxSteps; s0 += UT) {
                 if (x_lo + s0 * kStep >= x_hi) break;
-                float v[UT][GV];
+                float v[UT][VW];
+                [[maybe_unused]] uint4 raw[E::kBytes == 2 ? UT : 1];
 #pragma unroll
-                for (int u = 0; u < UT; ++u) load_group_clamped(x_lo + (s0 + u) * kStep + lane * GV, v[u]);
+                for (int u = 0; u < UT; ++u) {
+                    if constexpr (E::kBytes == 2) raw[u] = load_raw_clamped(x_lo + (s0 + u) * kStep + lane * GV);
+                    else load_group_clamped(x_lo + (s0 + u) * kStep + lane * GV, v[u]);
+                }
 #pragma unroll
                 for (int u = 0; u < UT; ++u) {
                     const int x0 = x_lo + (s0 + u) * kStep + lane * GV;
                     if (x0 < x_hi) {   // (a group read in place of one past the run is not this thread's)
+                        float f[GV];
+                        if constexpr (E::kBytes == 2) {
+                            E::unpack(raw[u], f);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < GV; ++e) f[e] = v[u][e];
+                        }
 #pragma unroll
                         for (int e = 0; e < GV; ++e)
-                            if (v[u][e] > best) { best = v[u][e]; best_i = x0 + e; }   // ascending index: ties keep the lowest
+                            if (f[e] > best) { best = f[e]; best_i = x0 + e; }   // ascending index: ties keep the lowest
                     }
                 }
             }
@@ -205,27 +243,6 @@ sample_kernel(const __grid_constant__ SampleParams P)
     float g[kMaxSteps];
     float rb[NB];   // reference of each batch (-inf: nothing there)
     if constexpr (E::kBytes == 2) {
-        // the packed form of load_group_clamped
-        auto load_raw_clamped = [&](int x0) -> uint4 {
-            float v[GV];
-            if (P.vector_ok) {
-                const int xc = x0 < x_last ? x0 : x_last;
-                const uint4 r = ldg_v4(row + static_cast<size_t>(xc) * E::kBytes);
-                if (!(tail_mask && xc == x_last)) return r;
-                E::unpack(r, v);   // the row's last, incomplete group: its padding becomes -inf
-#pragma unroll
-                for (int e = 0; e < GV; ++e) v[e] = xc + e < P.V ? v[e] : -INFINITY;
-            } else {
-#pragma unroll
-                for (int e = 0; e < GV; ++e) v[e] = x0 + e < P.V ? E::load(row, x0 + e) : -INFINITY;
-            }
-            uint4 r;
-            r.x = E::to_bits(v[0]) | (E::to_bits(v[1]) << 16);
-            r.y = E::to_bits(v[2]) | (E::to_bits(v[3]) << 16);
-            r.z = E::to_bits(v[4]) | (E::to_bits(v[5]) << 16);
-            r.w = E::to_bits(v[6]) | (E::to_bits(v[7]) << 16);
-            return r;
-        };
 #pragma unroll
         for (int bi = 0; bi < NB; ++bi) {
             uint4 raw[U];
