@@ -113,7 +113,7 @@ extern "C" {
 
 /* Options of mcsd_set_option: process-wide tuning and test overrides, 0 = library default.
  * Some also take their initial value from the environment variable of the same
- * name (MCSD_CLUSTER, MCSD_EPT, MCSD_DIRECT, MCSD_SAMPLE_AHEAD, MCSD_PDL, MCSD_SPLIT, MCSD_TRACE), read once when
+ * name (MCSD_CLUSTER, MCSD_EPT, MCSD_DIRECT, MCSD_SAMPLE_AHEAD, MCSD_PDL, MCSD_SPLIT, MCSD_TRACE, MCSD_WALK_CLUSTER), read once when
  * the library is loaded. */
 #define MCSD_OPT_CLUSTER 0       /* CTAs per thread-block cluster of the node kernel (1..8)          */
 #define MCSD_OPT_EPT 1           /* vocabulary elements per thread and row of the node kernel         */
@@ -138,7 +138,9 @@ extern "C" {
 #define MCSD_OPT_TRACE 10        /* host-side tracing of the verification entry points and mcsd_sample_candidates:
                                     bit 0: one line per call on stderr (shape, temperature, mode, return code, kernel
                                     launches, layout of the node stage); bit 1: an NVTX range around every call     */
-#define MCSD_OPT_COUNT 11
+#define MCSD_OPT_WALK_CLUSTER 11 /* walk stage with a thread-block cluster of eight CTAs per sequence instead of one
+                                    CTA (same results): 0 = library's choice (small batches), 1 = never, 2 = always  */
+#define MCSD_OPT_COUNT 12
 
 typedef struct mcsd_desc {
     int32_t batch;      /* B: number of trees                                         */

@@ -29,7 +29,7 @@ EXPORTS = ("mcsd_verify", "mcsd_verify_nodes", "mcsd_verify_walk", "mcsd_verify_
            "mcsd_version", "mcsd_set_option", "mcsd_get_option", "mcsd_release_host_staging",
            "mcsd_shard_columns", "mcsd_shard_workspace_bytes", "mcsd_shard_rounds", "mcsd_shard_partials",
            "mcsd_shard_decide", "mcsd_shard_endpoint", "mcsd_shard_finish", "mcsd_shard_commit", "mcsd_debug_bounds_hits", "mcsd_last_kernel_times")
-OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL, OPT_TEST_SHRINK_RANGES, OPT_SPLIT, OPT_TIME_KERNELS, OPT_TRACE = range(11)
+OPT_CLUSTER, OPT_EPT, OPT_DIRECT, OPT_SAMPLE_AHEAD, OPT_WAIT_POLLS, OPT_TEST_EXTRA_TX, OPT_PDL, OPT_TEST_SHRINK_RANGES, OPT_SPLIT, OPT_TIME_KERNELS, OPT_TRACE, OPT_WALK_CLUSTER = range(12)
 
 
 class McsdDesc(ctypes.Structure):

@@ -38,6 +38,7 @@ struct Options {
         v[MCSD_OPT_PDL] = env_int("MCSD_PDL", 1);
         v[MCSD_OPT_SPLIT] = env_int("MCSD_SPLIT", 0);
         v[MCSD_OPT_TRACE] = env_int("MCSD_TRACE", 0);
+        v[MCSD_OPT_WALK_CLUSTER] = env_int("MCSD_WALK_CLUSTER", 0);
     }
 };
 Options g_opt;
@@ -688,6 +689,9 @@ int launch_naive(const Call &c, const void *target, const int32_t *cand, const f
     return MCSD_OK;
 }
 
+// Batches up to this many sequences per eight SMs take the clustered walk kernel (measured).
+constexpr int kWalkClusterUpTo = 2;
+
 int launch_walk(const Call &c, const void *target, const void *draft, const int32_t *cand,
                 const float *unif, float T, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual,
                 bool all_nodes_allowed = true)
@@ -740,7 +744,16 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     }
     const bool want_all_early = all_nodes_allowed && ((T > 0.f && d->node_bonus) || d->node_residual);
-    if (d->vocab <= MCSD_MAX_VOCAB / 2 && (d->batch > n_sm || want_all_early)) {
+    // a small batch: a cluster of eight CTAs of 128 threads per sequence, so that eight SMs share its
+    // exponentials (MCSD_OPT_WALK_CLUSTER: 1 never, 2 always)
+    const int wc_opt = g_opt.v[MCSD_OPT_WALK_CLUSTER];
+    int walk_cluster = 1;
+    if (wc_opt == 2 || (wc_opt == 0 && !want_all_early && d->batch * 8 <= kWalkClusterUpTo * n_sm)) {
+        walk_cluster = 8;
+        threads = 128;
+        fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 128, 8>
+           : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 128, 8> : walk_kernel<MCSD_DTYPE_F16, 128, 8>;
+    } else if (d->vocab <= MCSD_MAX_VOCAB / 2 && (d->batch > n_sm || want_all_early)) {
         threads = 512;
         fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 512>
            : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 512> : walk_kernel<MCSD_DTYPE_F16, 512>;
@@ -755,14 +768,25 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
     for (int all = want_all ? 1 : 0; all >= 0; --all) {
         p.all_nodes = all;
         cudaLaunchConfig_t lc = {};
-        lc.gridDim = dim3(static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch));
+        lc.gridDim = dim3(static_cast<unsigned>((all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch) * walk_cluster));
         lc.blockDim = dim3(static_cast<unsigned>(threads));
         lc.stream = c.stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchAttribute attr[2];
+        int n_attr = 0;
+        if (p.pdl) {
+            attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+            ++n_attr;
+        }
+        if (walk_cluster > 1) {
+            attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+            attr[n_attr].val.clusterDim.x = static_cast<unsigned>(walk_cluster);
+            attr[n_attr].val.clusterDim.y = 1;
+            attr[n_attr].val.clusterDim.z = 1;
+            ++n_attr;
+        }
         lc.attrs = attr;
-        lc.numAttrs = p.pdl ? 1 : 0;
+        lc.numAttrs = static_cast<unsigned>(n_attr);
         ScopedTimer timer(3, c.stream);
         if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
             cudaGetLastError();

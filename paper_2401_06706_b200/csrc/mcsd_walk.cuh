@@ -48,11 +48,18 @@ constexpr int kWalkWarps = kWalkThreads / 32;
 // the lane and the element from the group sums it kept (the helpers of mcsd_common.cuh).
 // NT threads per CTA: 512 (two CTAs per SM) when the vocabulary is at most half the maximum,
 // else 1024; a warp's run is at most MCSD_MAX_VOCAB / 32 elements either way.
-template <int DT, int NT>
+// CL > 1 (small batches, which leave most SMs idle): a thread-block cluster of CL CTAs works on one
+// sequence, so that its 2 V exponentials are spread over CL SMs instead of queueing at the special-
+// function unit of one (at batch 1 that queue alone is 2 us per sweep).  The CL * NT / 32 warps of the
+// cluster own the runs exactly as the warps of one large CTA would (the results are the same bit for
+// bit); every warp sends its run's total into the shared memory of all CTAs, one cluster barrier, and
+// every CTA goes on alone.  The walk itself is followed by every CTA; CTA 0 writes it.
+template <int DT, int NT, int CL = 1>
 __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
 walk_kernel(const __grid_constant__ WalkParams P)
 {
     using E = Elem<DT>;
+    static_assert(CL * NT <= 1024, "the cluster's warps are the at most 32 runs of the search");
     constexpr int GV = E::kVec;
     __shared__ int s_term, s_len, s_stat;
     __shared__ int32_t s_acc[MCSD_MAX_NODES], s_tok[MCSD_MAX_NODES];
@@ -60,16 +67,19 @@ walk_kernel(const __grid_constant__ WalkParams P)
     // up front in parallel, so that nothing the walk decides has to wait for another trip to memory
     __shared__ NodeStats s_stats[MCSD_MAX_NODES];
     __shared__ float s_uend[MCSD_MAX_NODES];
-    constexpr int kW = NT / 32;  // warps
+    constexpr int kW = CL * NT / 32;  // warps (of the whole cluster)
     __shared__ double s_wtot[32];
     __shared__ float s_leaf[2];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int crank = CL > 1 ? static_cast<int>(cluster_ctarank()) : 0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = crank * (NT / 32) + (tid >> 5);   // warp: index in the cluster
+    const bool writer = crank == 0;   // the CTA that writes what all CTAs of the cluster compute alike
+    const int unit = CL > 1 ? static_cast<int>(blockIdx.x) / CL : static_cast<int>(blockIdx.x);
     int b, n;
     if (P.all_nodes) {
-        b = blockIdx.x / P.n_nodes;
-        n = blockIdx.x - b * P.n_nodes;
+        b = unit / P.n_nodes;
+        n = unit - b * P.n_nodes;
     } else {
-        b = blockIdx.x;
+        b = unit;
         n = 0;
     }
     const long long nb = static_cast<long long>(b) * P.n_nodes;
@@ -98,15 +108,19 @@ walk_kernel(const __grid_constant__ WalkParams P)
                 const int nx = s_acc[n];
                 if (nx <= n || nx >= P.n_nodes) break;
                 n = nx;
-                tok[len] = s_tok[n];
-                if (P.out_path_nodes) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + len] = n;
+                if (writer) {
+                    tok[len] = s_tok[n];
+                    if (P.out_path_nodes) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + len] = n;
+                }
                 ++len;
             }
             if (P.scale != 0.f && n < P.n_internal) st |= s_stats[n].status;
-            for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
-            if (P.out_path_nodes)
-                for (int i = len; i <= P.gamma; ++i) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + i] = -1;
-            P.out_accept_len[b] = len;
+            if (writer) {
+                for (int i = len + 1; i <= P.gamma; ++i) tok[i] = -1;
+                if (P.out_path_nodes)
+                    for (int i = len; i <= P.gamma; ++i) P.out_path_nodes[static_cast<long long>(b) * (P.gamma + 1) + i] = -1;
+                P.out_accept_len[b] = len;
+            }
             s_term = n;
             s_len = len;
             s_stat = st;
@@ -117,7 +131,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
     } else {
         if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (P.node_accept[nb + n] >= 0) {
-            if (tid == 0) P.node_bonus[nb + n] = -1;  // a walk never stops here
+            if (tid == 0 && writer) P.node_bonus[nb + n] = -1;  // a walk never stops here
             return;
         }
     }
@@ -137,9 +151,9 @@ walk_kernel(const __grid_constant__ WalkParams P)
         // argmax rule: the endpoint is the target argmax of the stopping node, the
         // distribution is one-hot (all-nodes mode has nothing to add here)
         const int a = P.node_bonus[nb + n];
-        if (tid == 0 && !P.all_nodes) finish(a, 0);
+        if (tid == 0 && writer && !P.all_nodes) finish(a, 0);
         if (out)
-            for (int x = tid; x < P.V; x += NT) out[x] = (x == a) ? 1.f : 0.f;
+            for (int x = crank * NT + tid; x < P.V; x += CL * NT) out[x] = (x == a) ? 1.f : 0.f;
         return;
     }
 
@@ -150,7 +164,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
         const NodeStats st = P.all_nodes ? P.stats[nb + n] : s_stats[n];
         r_t = st.r_t; r_d = st.r_d; z_t = st.z_t; z_d = st.z_d; c = st.c; c_prev = st.c_prev;
     } else {
-        if (warp == 0) {
+        if ((tid >> 5) == 0) {
             const float2 *part = P.leaf_part +
                 (static_cast<long long>(b) * (P.n_nodes - P.n_internal) + (n - P.n_internal)) * kLeafEntries;
             float2 e = make_float2(-INFINITY, 0.f);
@@ -236,9 +250,19 @@ walk_kernel(const __grid_constant__ WalkParams P)
             }
         }
         const double mass = run_total<kMaxSteps>(g);
-        __syncthreads();   // (second attempt: everybody has read the totals of the first)
-        if (lane == 0) s_wtot[warp] = mass;
-        __syncthreads();
+        if constexpr (CL > 1) {
+            // (second attempt: every CTA has read the totals of the first before they are overwritten)
+            if (attempt) cluster_sync_all();
+            if (lane < CL) {
+                const uint32_t dst = map_to_rank(smem_u32(&s_wtot[warp]), static_cast<uint32_t>(lane));
+                asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(dst), "d"(mass) : "memory");
+            }
+            cluster_sync_all();   // release / acquire: the totals of all CTAs are in this CTA's shared memory
+        } else {
+            __syncthreads();   // (second attempt: everybody has read the totals of the first)
+            if (lane == 0) s_wtot[warp] = mass;
+            __syncthreads();
+        }
         // the run that holds the quantile (every warp finds the same one)
         pick = pick_run(lane < kW ? s_wtot[lane] : 0.0, u_end, lane, tgt);
         if (pick >= 0 || !internal) break;
@@ -248,7 +272,7 @@ walk_kernel(const __grid_constant__ WalkParams P)
         kappa = fminf(c_prev * dq, 3.0e38f);
     }
     if (pick < 0) {
-        if (tid == 0) finish(-1, extra_bits | MCSD_STATUS_NO_MASS);
+        if (tid == 0 && writer) finish(-1, extra_bits | MCSD_STATUS_NO_MASS);
         return;   // (`out` keeps the unnormalised weights: zeros or NaN, there is no distribution)
     }
     // sweep 2: every thread scales what it wrote by 1 / S

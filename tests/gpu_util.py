@@ -61,7 +61,7 @@ def library_options(**opts):
     ids = {"cluster": binding.OPT_CLUSTER, "ept": binding.OPT_EPT, "direct": binding.OPT_DIRECT,
            "sample_ahead": binding.OPT_SAMPLE_AHEAD, "wait_polls": binding.OPT_WAIT_POLLS,
            "test_extra_tx": binding.OPT_TEST_EXTRA_TX, "pdl": binding.OPT_PDL,
-           "test_shrink_ranges": binding.OPT_TEST_SHRINK_RANGES, "split": binding.OPT_SPLIT, "trace": binding.OPT_TRACE}
+           "test_shrink_ranges": binding.OPT_TEST_SHRINK_RANGES, "split": binding.OPT_SPLIT, "trace": binding.OPT_TRACE, "walk_cluster": binding.OPT_WALK_CLUSTER}
     before = {k: binding.mcsd_get_option(ids[k]) for k in opts}
     try:
         for k, val in opts.items():

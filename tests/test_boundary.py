@@ -40,7 +40,7 @@ def test_header_constants_match_binding():
     assert int(consts["MCSD_MAX_VOCAB"]) == binding.MAX_VOCAB
     assert int(consts["MCSD_STATUS_TIMEOUT"]) == binding.STATUS_TIMEOUT
     assert int(consts["MCSD_DTYPE_BF16"]) == 1 and int(consts["MCSD_DTYPE_F16"]) == 2
-    for name in ("CLUSTER", "EPT", "DIRECT", "SAMPLE_AHEAD", "WAIT_POLLS", "TEST_EXTRA_TX", "PDL", "TEST_SHRINK_RANGES", "SPLIT", "TIME_KERNELS", "TRACE"):
+    for name in ("CLUSTER", "EPT", "DIRECT", "SAMPLE_AHEAD", "WAIT_POLLS", "TEST_EXTRA_TX", "PDL", "TEST_SHRINK_RANGES", "SPLIT", "TIME_KERNELS", "TRACE", "WALK_CLUSTER"):
         assert int(consts["MCSD_OPT_" + name]) == getattr(binding, "OPT_" + name)
 
 

@@ -132,6 +132,29 @@ def test_split_launch_equals_single_launch(dtype, vocab, kconfig, mode):
         assert np.array_equal(a, b, equal_nan=True)
 
 
+@pytest.mark.parametrize("dtype,vocab,kconfig,mode,T", [("bf16", 32000, "4x2x2x1", 1, 1.0), ("fp32", 32000, "2", 0, 0.7),
+                                                       ("fp16", 50272, "2x2", 1, 1.3), ("fp32", 1000, "3x2x1", 0, 1.0),
+                                                       ("bf16", 7, "2x2", 0, 1.0), ("fp32", 65536, "1x1", 0, 1.0),
+                                                       ("fp16", 4099, "8x1", 1, 0.0)])
+def test_clustered_walk_equals_single_cta_walk(dtype, vocab, kconfig, mode, T):
+    """Small batches give every sequence a cluster of eight CTAs in the walk stage; its 32 warps own the
+    runs the 32 warps of the one-CTA form of 1024 threads own and sum in the same order, so every output
+    agrees bit for bit, and with the oracle.  (With per-node outputs the one-CTA form has 16 warps and
+    other runs: there both are held against the oracle.)"""
+    w = synth.Workload("cwalk", 5, vocab, kconfig, dtype, "normal", 2.5, 0.9, 1.2, T, mode, 5100 + vocab)
+    inp = synth.make_inputs(w, "cuda")
+    outs = []
+    for wc in (1, 2):                         # 1: never, 2: always
+        with library_options(walk_cluster=wc):
+            _, out = run_library(inp, node_outputs=False)
+            outs.append([to_np(x).copy() for x in (out.accept_len, out.tokens, out.residual, out.status, out.path_nodes)])
+            assert_parity(inp, out)
+            _, out = run_library(inp, node_outputs=True)
+            assert_parity(inp, out)
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b, equal_nan=True)
+
+
 def test_traced_call_reports_its_layout_and_changes_nothing(capfd):
     """MCSD_OPT_TRACE 3: a line on stderr per call (with how the node stage was laid out) and an NVTX
     range around it; the outputs are those of the untraced call."""
