@@ -689,8 +689,11 @@ int launch_naive(const Call &c, const void *target, const int32_t *cand, const f
     return MCSD_OK;
 }
 
-// Batches up to this many sequences per eight SMs take the clustered walk kernel (measured).
-constexpr int kWalkClusterUpTo = 2;
+// Batches up to this size take the clustered walk kernel, the smallest ones its form without a register
+// budget (measured on 148 SMs: one wave of 8-CTA clusters holds 18 sequences at 2 CTAs per SM; at 64
+// sequences the clustered form is no faster with a vocabulary of 32000 and slower with 50272).
+constexpr int kWalkClusterFewBatch = 18;
+constexpr int kWalkClusterMaxBatch = 37;
 
 int launch_walk(const Call &c, const void *target, const void *draft, const int32_t *cand,
                 const float *unif, float T, int32_t *out_accept_len, int32_t *out_tokens, float *out_residual,
@@ -748,11 +751,15 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
     // exponentials (MCSD_OPT_WALK_CLUSTER: 1 never, 2 always)
     const int wc_opt = g_opt.v[MCSD_OPT_WALK_CLUSTER];
     int walk_cluster = 1;
-    if (wc_opt == 2 || (wc_opt == 0 && !want_all_early && d->batch * 8 <= kWalkClusterUpTo * n_sm)) {
+    if (wc_opt == 2 || (wc_opt == 0 && !want_all_early && d->batch <= kWalkClusterMaxBatch)) {
         walk_cluster = 8;
         threads = 128;
-        fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 128, 8>
-           : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 128, 8> : walk_kernel<MCSD_DTYPE_F16, 128, 8>;
+        if (d->batch <= kWalkClusterFewBatch)
+            fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 128, 8, 1>
+               : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 128, 8, 1> : walk_kernel<MCSD_DTYPE_F16, 128, 8, 1>;
+        else
+            fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 128, 8, 4>
+               : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 128, 8, 4> : walk_kernel<MCSD_DTYPE_F16, 128, 8, 4>;
     } else if (d->vocab <= MCSD_MAX_VOCAB / 2 && (d->batch > n_sm || want_all_early)) {
         threads = 512;
         fn = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 512>

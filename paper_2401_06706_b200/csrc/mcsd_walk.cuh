@@ -54,8 +54,11 @@ constexpr int kWalkWarps = kWalkThreads / 32;
 // cluster own the runs exactly as the warps of one large CTA would (the results are the same bit for
 // bit); every warp sends its run's total into the shared memory of all CTAs, one cluster barrier, and
 // every CTA goes on alone.  The walk itself is followed by every CTA; CTA 0 writes it.
-template <int DT, int NT, int CL = 1>
-__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
+// MB: CTAs per SM the register budget is held to.  The clustered form exists with 1 (the compiler then has
+// all row loads of a sweep in flight: the fastest form for a handful of sequences) and with 4 (128
+// registers: 74 clusters resident at once, for batches up to that).
+template <int DT, int NT, int CL = 1, int MB = (NT == 512 ? 2 : 1)>
+__global__ void __launch_bounds__(NT, MB)
 walk_kernel(const __grid_constant__ WalkParams P)
 {
     using E = Elem<DT>;
