@@ -795,7 +795,18 @@ int launch_walk(const Call &c, const void *target, const void *draft, const int3
         lc.attrs = attr;
         lc.numAttrs = static_cast<unsigned>(n_attr);
         ScopedTimer timer(3, c.stream);
-        if (cudaLaunchKernelEx(&lc, fn, p) != cudaSuccess) {
+        cudaError_t err = cudaLaunchKernelEx(&lc, fn, p);
+        if (err != cudaSuccess && walk_cluster > 1) {
+            // a device (or partition of one) that cannot place clusters of eight: the one-CTA form does the same
+            cudaGetLastError();
+            WalkKernel one = d->dtype == MCSD_DTYPE_F32 ? walk_kernel<MCSD_DTYPE_F32, 1024>
+                           : d->dtype == MCSD_DTYPE_BF16 ? walk_kernel<MCSD_DTYPE_BF16, 1024> : walk_kernel<MCSD_DTYPE_F16, 1024>;
+            lc.gridDim = dim3(static_cast<unsigned>(all ? static_cast<long long>(d->batch) * d->n_nodes : d->batch));
+            lc.blockDim = dim3(1024);
+            lc.numAttrs = p.pdl ? 1 : 0;   // (the attribute of the dependent launch comes first)
+            err = cudaLaunchKernelEx(&lc, one, p);
+        }
+        if (err != cudaSuccess) {
             cudaGetLastError();
             return MCSD_ERR_CUDA;
         }
